@@ -1,0 +1,175 @@
+/*
+ * peqa.h -- C ABI of the B200 (sm_100a) PEQA quantized-linear library.
+ *
+ * PEQA (arXiv 2305.14152) freezes a b-bit integer matrix Q and a zero-point z
+ * and trains only the quantization scale s; the effective weight of a linear
+ * layer is W_hat = s * (Q - z) (Eq. 2, Sec. 3.2).  This library is the layer's
+ * hot path: quantize once (Eq. 1), forward, backward (dX and the scale
+ * gradient dS, without ever materialising dW), small-batch decode, and AdamW
+ * on the scales.
+ *
+ * Conventions for every entry point
+ *   - All tensor pointers are DEVICE pointers owned by the caller, dense and
+ *     row-major, 16-byte aligned, unless an argument says "host".  The library
+ *     allocates no device memory.
+ *   - N = out_features (rows of W, the paper's n), K = in_features (columns,
+ *     the paper's m), T = tokens.  group_size g: 0 or K means one (s, z) per
+ *     output row ("per-channel", Sec. 3.2); otherwise g is a multiple of 32
+ *     that divides K and (s, z) are shared by runs of g input columns within
+ *     a row (Sec. 4.2, "Group-wise Quantization").  G = K / g.
+ *   - bits b is 3 or 4.
+ *   - Packed layout of Q: each row is a little-endian bit string in which
+ *     column j occupies bits [b*j, b*j+b), stored as uint32 words; a row has
+ *     K*b/32 words (8 codes per word for b=4, 32 codes per 3 words for b=3).
+ *   - Activations and their gradients are bf16; scales and dS are fp32;
+ *     zero-points are uint8 integers in [0, 2^b-1].
+ *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).
+ *     Calls validate their arguments on the host, enqueue work and return
+ *     without synchronising (peqa_train_step_host and peqa_check_status
+ *     synchronise, as documented).
+ *   - Return value: PEQA_OK or a negative peqa_status code.  Nothing is
+ *     enqueued when an argument check fails.
+ *   - Kernels that wait on hardware barriers give every wait a bound; a wait
+ *     that runs out records PEQA_ERR_DEVICE_TIMEOUT in a device status word
+ *     that peqa_check_status() reads back.  Outputs are undefined after it.
+ */
+#ifndef PEQA_H_
+#define PEQA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  PEQA_OK = 0,
+  PEQA_ERR_NULL = -1,           /* a required pointer is NULL */
+  PEQA_ERR_BAD_BITS = -2,       /* bits not in {3, 4} */
+  PEQA_ERR_BAD_SHAPE = -3,      /* non-positive size, K % 32, bad group size, unsupported tile constraint */
+  PEQA_ERR_ALIGNMENT = -4,      /* a pointer is not aligned as required */
+  PEQA_ERR_WORKSPACE = -5,      /* workspace missing or smaller than peqa_workspace_bytes() */
+  PEQA_ERR_ARCH = -6,           /* current device is not compute capability 10.x */
+  PEQA_ERR_CUDA = -7,           /* a CUDA runtime/driver call failed; see peqa_last_cuda_error() */
+  PEQA_ERR_DEVICE_TIMEOUT = -8, /* a bounded device-side wait expired */
+  PEQA_ERR_TOO_LARGE = -9       /* size exceeds a documented fixed capacity */
+} peqa_status;
+
+/* Frozen part (Q, z) and trainable scale s of one PEQA linear layer. */
+typedef struct {
+  int32_t bits;            /* 3 or 4 */
+  int32_t out_features;    /* N */
+  int32_t in_features;     /* K, multiple of 32 */
+  int32_t group_size;      /* 0 or K: per-channel; else multiple of 32 dividing K */
+  const uint32_t* qweight; /* [N, K*bits/32] packed codes */
+  const uint8_t* zeros;    /* [N, G] */
+  const float* scales;     /* [N, G] */
+} peqa_qweight_t;
+
+typedef enum { PEQA_OP_FWD = 0, PEQA_OP_BWD = 1, PEQA_OP_DECODE = 2 } peqa_op;
+
+/* Library version, major*10000 + minor*100 + patch. */
+int peqa_version(void);
+
+/* cudaError_t of the most recent failing CUDA call made by this library on
+ * the calling thread (0 if none). */
+int peqa_last_cuda_error(void);
+
+/*
+ * Asymmetric round-to-nearest quantization, Eq. 1 (Sec. 3.2), per (row, group):
+ *   mn, mx = min/max of the group;  s = (mx - mn) / (2^b - 1)  (s = 1 if mx == mn)
+ *   z = clamp(rint(-mn / s), 0, 2^b - 1);   Q = clamp(rint(W / s) + z, 0, 2^b - 1)
+ * evaluated in IEEE binary32, round-half-to-even, true division, no FMA.
+ *   W        in   fp32 [N, K]
+ *   qweight  out  uint32 [N, K*bits/32]  packed Q
+ *   zeros    out  uint8 [N, G]
+ *   scales   out  fp32 [N, G]
+ * W must be finite.  K % 32 == 0 and K <= 65536 (else PEQA_ERR_TOO_LARGE).
+ */
+int peqa_quantize_rtn(const float* W, int N, int K, int bits, int group_size,
+                      uint32_t* qweight, uint8_t* zeros, float* scales, void* stream);
+
+/* Pack one code per byte (values in [0, 2^bits-1], upper bits ignored) into the
+ * packed layout above, and the inverse.  codes is uint8 [N, K]; K % 32 == 0.
+ * (The paper only states that the weights are a b-bit integer matrix, Sec. 3.3.) */
+int peqa_pack(const uint8_t* codes, int N, int K, int bits, uint32_t* qweight, void* stream);
+int peqa_unpack(const uint32_t* qweight, int N, int K, int bits, uint8_t* codes, void* stream);
+
+/* Bytes of caller-provided scratch the given operation (peqa_op) needs for T
+ * tokens (0 if none).  The workspace must be 256-byte aligned.  Its contents
+ * are overwritten by each call; calls that may overlap need distinct workspaces. */
+size_t peqa_workspace_bytes(int op, int T, const peqa_qweight_t* w);
+
+/*
+ * Forward of the PEQA layer, Y = X * W_hat^T with W_hat = s*(Q - z) (Eq. 2):
+ *   Y[t,i] = sum_j X[t,j] * s[i,g(j)] * (Q[i,j] - z[i,g(j)])
+ *   X  in   bf16 [T, K]
+ *   Y  out  bf16 [T, N]  (fp32 accumulation, rounded to nearest even)
+ * Requires K % 64 == 0, N % 8 == 0, T >= 1.  workspace may be NULL.
+ */
+int peqa_qlinear_fwd(const peqa_qweight_t* w, const void* X_bf16, int T, void* Y_bf16,
+                     void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Backward of the PEQA layer (chain rule on Eq. 2; Q and z are frozen, s is
+ * the only trainable tensor, Sec. 3.2):
+ *   dX[t,j]  = sum_i dY[t,i] * s[i,g(j)] * (Q[i,j] - z[i,g(j)])
+ *   dS[i,gi] = sum_{j in group gi} (Q[i,j] - z[i,gi]) * sum_t dY[t,i] * X[t,j]
+ *   X   in   bf16 [T, K]  (only needed for dS)      dY  in  bf16 [T, N]
+ *   dX  out  bf16 [T, K]      (may be NULL: skipped)
+ *   dS  out  fp32 [N, G]      (may be NULL: skipped) OVERWRITTEN, not accumulated
+ * dW = dY^T X exists only tile by tile in tensor memory and registers.
+ * Requires K % 64 == 0, N % 8 == 0, T >= 1.  Needs a workspace of
+ * peqa_workspace_bytes(PEQA_OP_BWD, T, w) bytes when that is non-zero.
+ */
+int peqa_qlinear_bwd(const peqa_qweight_t* w, const void* X_bf16, const void* dY_bf16, int T,
+                     void* dX_bf16, float* dS, void* workspace, size_t workspace_bytes,
+                     void* stream);
+
+/*
+ * Small-batch forward for token generation (the memory-bound matrix-vector
+ * regime of Sec. 3.1 / 3.3): same definition as peqa_qlinear_fwd with
+ * T = M in [1, 16], implemented as a streaming fused dequant GEMV / skinny GEMM.
+ * Requires K % 128 == 0 and N % 8 == 0.
+ */
+int peqa_qlinear_decode(const peqa_qweight_t* w, const void* X_bf16, int M, void* Y_bf16,
+                        void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * One AdamW step on the scales, in place (App. A names AdamW; decoupled weight
+ * decay, bias-corrected moments, step counted from 1):
+ *   s <- s*(1 - lr*wd);  m <- b1*m + (1-b1)*dS;  v <- b2*v + (1-b2)*dS^2
+ *   s <- s - lr * (m/(1-b1^step)) / (sqrt(v/(1-b2^step)) + eps)
+ * scales, dS, m, v are fp32 [numel].
+ */
+int peqa_scale_adamw(float* scales, const float* dS, float* m, float* v, int64_t numel,
+                     float lr, float beta1, float beta2, float eps, float weight_decay,
+                     int64_t step, void* stream);
+
+/*
+ * One training step of a PEQA layer with HOST activations (composition of
+ * Eq. 2's forward/backward with App. A's optimizer): copies h_X [T,K] and
+ * h_dY [T,N] (host bf16, pinned or pageable) into the caller's device staging
+ * buffers d_X, d_dY, runs forward, backward and AdamW on the stream, and
+ * copies Y [T,N], dX [T,K] (host bf16) and dS [N,G] (host fp32) back.  Every
+ * d_* pointer is device memory of the size of its host counterpart; d_m, d_v
+ * are the optimizer state [N,G].  w->scales is updated in place (it must be
+ * writable).  Synchronises the stream before returning.
+ */
+int peqa_train_step_host(const peqa_qweight_t* w, int T,
+                         const void* h_X_bf16, const void* h_dY_bf16,
+                         void* h_Y_bf16, void* h_dX_bf16, float* h_dS,
+                         void* d_X, void* d_dY, void* d_Y, void* d_dX, float* d_dS,
+                         float* d_m, float* d_v,
+                         float lr, float beta1, float beta2, float eps, float weight_decay,
+                         int64_t step, void* workspace, size_t workspace_bytes, void* stream);
+
+/* Synchronises `stream`, reads and clears the device status word.  Returns
+ * PEQA_OK, PEQA_ERR_DEVICE_TIMEOUT, or PEQA_ERR_CUDA. */
+int peqa_check_status(void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PEQA_H_ */

@@ -1,0 +1,163 @@
+// C-ABI entry points that only validate and dispatch, plus the library's
+// small amount of per-device state (architecture check, status word).
+#include "common.cuh"
+
+namespace peqa {
+
+thread_local int g_last_cuda_error = 0;
+
+// Written by kernels whose bounded waits expire: [0] = status code, [1..3] = where.
+__device__ int g_status_word[4];
+
+int status_word(int** dev_ptr) {
+  void* p = nullptr;
+  PEQA_CUDA(cudaGetSymbolAddress(&p, g_status_word));
+  *dev_ptr = static_cast<int*>(p);
+  return PEQA_OK;
+}
+
+int check_arch() {
+  static thread_local int cached_dev = -1;
+  static thread_local int cached_ok = 0;
+  int dev = 0;
+  PEQA_CUDA(cudaGetDevice(&dev));
+  if (dev != cached_dev) {
+    int major = 0;
+    PEQA_CUDA(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
+    cached_dev = dev;
+    cached_ok = (major == 10);
+  }
+  return cached_ok ? PEQA_OK : PEQA_ERR_ARCH;
+}
+
+int check_qweight(const peqa_qweight_t* w, int* g, int* G) {
+  if (!w) return PEQA_ERR_NULL;
+  if (!w->qweight || !w->zeros || !w->scales) return PEQA_ERR_NULL;
+  PEQA_TRY(check_bits_shape(w->out_features, w->in_features, w->bits, w->group_size));
+  if (!aligned16(w->qweight) || !aligned16(w->scales)) return PEQA_ERR_ALIGNMENT;
+  *g = effective_group(w->in_features, w->group_size);
+  *G = w->in_features / *g;
+  return PEQA_OK;
+}
+
+}  // namespace peqa
+
+using namespace peqa;
+
+extern "C" int peqa_version(void) { return 100; }
+
+extern "C" int peqa_last_cuda_error(void) { return g_last_cuda_error; }
+
+extern "C" size_t peqa_workspace_bytes(int op, int T, const peqa_qweight_t* w) {
+  if (!w || T <= 0) return 0;
+  if (check_bits_shape(w->out_features, w->in_features, w->bits, w->group_size) != PEQA_OK)
+    return 0;
+  const int g = effective_group(w->in_features, w->group_size);
+  switch (op) {
+    case PEQA_OP_BWD: return ds_workspace_bytes(w, g, T);
+    case PEQA_OP_DECODE: return decode_workspace_bytes(w, g, T);
+    default: return 0;
+  }
+}
+
+static int check_gemm_shape(const peqa_qweight_t* w, int T) {
+  if (T <= 0) return PEQA_ERR_BAD_SHAPE;
+  if (w->in_features % 64 != 0 || w->out_features % 8 != 0) return PEQA_ERR_BAD_SHAPE;
+  return PEQA_OK;
+}
+
+extern "C" int peqa_qlinear_fwd(const peqa_qweight_t* w, const void* X, int T, void* Y,
+                                void* workspace, size_t workspace_bytes, void* stream) {
+  (void)workspace; (void)workspace_bytes;
+  int g = 0, G = 0;
+  PEQA_TRY(check_qweight(w, &g, &G));
+  if (!X || !Y) return PEQA_ERR_NULL;
+  PEQA_TRY(check_gemm_shape(w, T));
+  if (!aligned16(X) || !aligned16(Y)) return PEQA_ERR_ALIGNMENT;
+  PEQA_TRY(check_arch());
+  return launch_fwd(w, g, X, T, Y, as_stream(stream));
+}
+
+extern "C" int peqa_qlinear_bwd(const peqa_qweight_t* w, const void* X, const void* dY, int T,
+                                void* dX, float* dS, void* workspace, size_t workspace_bytes,
+                                void* stream) {
+  int g = 0, G = 0;
+  PEQA_TRY(check_qweight(w, &g, &G));
+  if (!dY) return PEQA_ERR_NULL;
+  if (dS && !X) return PEQA_ERR_NULL;
+  PEQA_TRY(check_gemm_shape(w, T));
+  if (!aligned16(dY) || (X && !aligned16(X)) || (dX && !aligned16(dX)) || (dS && !aligned16(dS)))
+    return PEQA_ERR_ALIGNMENT;
+  PEQA_TRY(check_arch());
+  if (dS) {
+    const size_t need = ds_workspace_bytes(w, g, T);
+    if (need > 0) {
+      if (!workspace || workspace_bytes < need) return PEQA_ERR_WORKSPACE;
+      if (reinterpret_cast<uintptr_t>(workspace) & 255u) return PEQA_ERR_ALIGNMENT;
+    }
+  }
+  if (dX) PEQA_TRY(launch_dx(w, g, dY, T, dX, as_stream(stream)));
+  if (dS) PEQA_TRY(launch_ds(w, g, X, dY, T, dS, workspace, workspace_bytes, as_stream(stream)));
+  return PEQA_OK;
+}
+
+extern "C" int peqa_qlinear_decode(const peqa_qweight_t* w, const void* X, int M, void* Y,
+                                   void* workspace, size_t workspace_bytes, void* stream) {
+  int g = 0, G = 0;
+  PEQA_TRY(check_qweight(w, &g, &G));
+  if (!X || !Y) return PEQA_ERR_NULL;
+  if (M < 1 || M > 16) return PEQA_ERR_BAD_SHAPE;
+  if (w->in_features % 128 != 0 || w->out_features % 8 != 0) return PEQA_ERR_BAD_SHAPE;
+  if (!aligned16(X) || !aligned16(Y)) return PEQA_ERR_ALIGNMENT;
+  PEQA_TRY(check_arch());
+  const size_t need = decode_workspace_bytes(w, g, M);
+  if (need > 0) {
+    if (!workspace || workspace_bytes < need) return PEQA_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(workspace) & 255u) return PEQA_ERR_ALIGNMENT;
+  }
+  return launch_decode(w, g, X, M, Y, workspace, workspace_bytes, as_stream(stream));
+}
+
+extern "C" int peqa_train_step_host(const peqa_qweight_t* w, int T,
+                                    const void* h_X, const void* h_dY,
+                                    void* h_Y, void* h_dX, float* h_dS,
+                                    void* d_X, void* d_dY, void* d_Y, void* d_dX, float* d_dS,
+                                    float* d_m, float* d_v,
+                                    float lr, float beta1, float beta2, float eps,
+                                    float weight_decay, int64_t step,
+                                    void* workspace, size_t workspace_bytes, void* stream) {
+  int g = 0, G = 0;
+  PEQA_TRY(check_qweight(w, &g, &G));
+  if (!h_X || !h_dY || !h_Y || !h_dX || !h_dS || !d_X || !d_dY || !d_Y || !d_dX || !d_dS ||
+      !d_m || !d_v)
+    return PEQA_ERR_NULL;
+  if (T <= 0) return PEQA_ERR_BAD_SHAPE;
+  cudaStream_t st = as_stream(stream);
+  const size_t N = w->out_features, K = w->in_features;
+  PEQA_CUDA(cudaMemcpyAsync(d_X, h_X, (size_t)T * K * 2, cudaMemcpyHostToDevice, st));
+  PEQA_CUDA(cudaMemcpyAsync(d_dY, h_dY, (size_t)T * N * 2, cudaMemcpyHostToDevice, st));
+  PEQA_TRY(peqa_qlinear_fwd(w, d_X, T, d_Y, workspace, workspace_bytes, stream));
+  PEQA_CUDA(cudaMemcpyAsync(h_Y, d_Y, (size_t)T * N * 2, cudaMemcpyDeviceToHost, st));
+  PEQA_TRY(peqa_qlinear_bwd(w, d_X, d_dY, T, d_dX, d_dS, workspace, workspace_bytes, stream));
+  PEQA_CUDA(cudaMemcpyAsync(h_dX, d_dX, (size_t)T * K * 2, cudaMemcpyDeviceToHost, st));
+  PEQA_CUDA(cudaMemcpyAsync(h_dS, d_dS, N * (size_t)G * 4, cudaMemcpyDeviceToHost, st));
+  PEQA_TRY(peqa_scale_adamw(const_cast<float*>(w->scales), d_dS, d_m, d_v, (int64_t)(N * G), lr,
+                            beta1, beta2, eps, weight_decay, step, stream));
+  PEQA_CUDA(cudaStreamSynchronize(st));
+  return PEQA_OK;
+}
+
+extern "C" int peqa_check_status(void* stream) {
+  int* dev = nullptr;
+  PEQA_TRY(status_word(&dev));
+  int host[4] = {0, 0, 0, 0};
+  cudaStream_t st = as_stream(stream);
+  PEQA_CUDA(cudaMemcpyAsync(host, dev, sizeof(host), cudaMemcpyDeviceToHost, st));
+  PEQA_CUDA(cudaStreamSynchronize(st));
+  if (host[0] != 0) {
+    PEQA_CUDA(cudaMemsetAsync(dev, 0, sizeof(host), st));
+    PEQA_CUDA(cudaStreamSynchronize(st));
+    return PEQA_ERR_DEVICE_TIMEOUT;
+  }
+  return PEQA_OK;
+}

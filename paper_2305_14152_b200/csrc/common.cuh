@@ -1,0 +1,68 @@
+// Shared host-side helpers of the PEQA sm_100a library: argument checks,
+// CUDA error capture and the device status word.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "peqa.h"
+
+namespace peqa {
+
+extern thread_local int g_last_cuda_error;
+
+inline int cuda_fail(cudaError_t e) {
+  g_last_cuda_error = (int)e;
+  return PEQA_ERR_CUDA;
+}
+
+#define PEQA_CUDA(expr)                                   \
+  do {                                                    \
+    cudaError_t _e = (expr);                              \
+    if (_e != cudaSuccess) return ::peqa::cuda_fail(_e);  \
+  } while (0)
+
+#define PEQA_TRY(expr)              \
+  do {                              \
+    int _s = (expr);                \
+    if (_s != PEQA_OK) return _s;   \
+  } while (0)
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Effective group size (per-channel when 0 or K) or 0 when invalid.
+inline int effective_group(int K, int group_size) {
+  if (group_size == 0 || group_size == K) return K;
+  if (group_size < 0 || group_size % 32 != 0 || K % group_size != 0) return 0;
+  return group_size;
+}
+
+inline int check_bits_shape(int N, int K, int bits, int group_size) {
+  if (bits != 3 && bits != 4) return PEQA_ERR_BAD_BITS;
+  if (N <= 0 || K <= 0 || K % 32 != 0) return PEQA_ERR_BAD_SHAPE;
+  if (effective_group(K, group_size) == 0) return PEQA_ERR_BAD_SHAPE;
+  return PEQA_OK;
+}
+
+// Validates a layer descriptor; fills g (effective group) and G.
+int check_qweight(const peqa_qweight_t* w, int* g, int* G);
+
+// The current device must be compute capability 10.x (cached per device).
+int check_arch();
+
+// Device address of the library's status word (int[4]) on the current device.
+int status_word(int** dev_ptr);
+
+inline cudaStream_t as_stream(void* s) { return reinterpret_cast<cudaStream_t>(s); }
+
+// Entry points implemented in the individual translation units.
+int launch_fwd(const peqa_qweight_t* w, int g, const void* X, int T, void* Y, cudaStream_t st);
+int launch_dx(const peqa_qweight_t* w, int g, const void* dY, int T, void* dX, cudaStream_t st);
+int launch_ds(const peqa_qweight_t* w, int g, const void* X, const void* dY, int T, float* dS,
+              void* workspace, size_t workspace_bytes, cudaStream_t st);
+size_t ds_workspace_bytes(const peqa_qweight_t* w, int g, int T);
+int launch_decode(const peqa_qweight_t* w, int g, const void* X, int M, void* Y,
+                  void* workspace, size_t workspace_bytes, cudaStream_t st);
+size_t decode_workspace_bytes(const peqa_qweight_t* w, int g, int M);
+
+}  // namespace peqa

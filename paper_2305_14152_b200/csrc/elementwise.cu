@@ -1,0 +1,228 @@
+// HBM-bound kernels of the PEQA path: RTN quantization (Eq. 1), the packed
+// b-bit layout, and AdamW on the scales (App. A).
+#include <math.h>
+
+#include "common.cuh"
+
+namespace peqa {
+
+namespace {
+
+constexpr int kQuantThreads = 256;
+constexpr int kQuantWarps = kQuantThreads / 32;
+constexpr int kMaxChunks = 2048;  // 32-column chunks per row -> K <= 65536
+
+// Lane `lane` of a warp holds code c for column (32*chunk + lane).  The row is
+// a little-endian bit string with column j at bits [bits*j, bits*j + bits), so
+// the 32 codes of a chunk fill exactly `bits` consecutive words.  Each lane
+// shifts its code to its place and the words are OR-reduced across the warp.
+template <int BITS>
+__device__ __forceinline__ void warp_pack_store(uint32_t code, int lane, uint32_t* dst) {
+  const int pos = BITS * lane;
+  const int word = pos >> 5;
+  const int sh = pos & 31;
+  const uint32_t lo = code << sh;
+  const uint32_t hi = (sh + BITS > 32) ? (code >> (32 - sh)) : 0u;
+#pragma unroll
+  for (int wi = 0; wi < BITS; ++wi) {
+    uint32_t contrib = (word == wi ? lo : 0u) | (word + 1 == wi ? hi : 0u);
+    uint32_t v = __reduce_or_sync(0xffffffffu, contrib);
+    if (lane == wi) dst[wi] = v;
+  }
+}
+
+template <int BITS>
+__device__ __forceinline__ uint32_t warp_unpack(const uint32_t* src, int lane) {
+  const int pos = BITS * lane;
+  const int word = pos >> 5;
+  const int sh = pos & 31;
+  uint32_t v = src[word] >> sh;
+  if (sh + BITS > 32) v |= src[word + 1] << (32 - sh);
+  return v & ((1u << BITS) - 1u);
+}
+
+// One CTA per output row.  Pass 1: per 32-column chunk min/max.  Pass 2: per
+// group (s, z) in strict binary32 (division and rounding as single IEEE
+// operations, no FMA).  Pass 3: codes, packed with the warp OR-reduction.
+// The row is read twice; the second read is served by L2.
+template <int BITS>
+__global__ void __launch_bounds__(kQuantThreads)
+quantize_rtn_kernel(const float* __restrict__ W, int K, int g,
+                    uint32_t* __restrict__ qweight, uint8_t* __restrict__ zeros,
+                    float* __restrict__ scales) {
+  __shared__ float cmin[kMaxChunks];
+  __shared__ float cmax[kMaxChunks];
+  __shared__ float gscale[kMaxChunks];
+  __shared__ float gzero[kMaxChunks];
+
+  const int row = blockIdx.x;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int chunks = K >> 5;
+  const int G = K / g;
+  const int cpg = g >> 5;  // chunks per group
+  const float* w = W + (size_t)row * K;
+  const float qmax = (float)((1 << BITS) - 1);
+
+  for (int c = warp; c < chunks; c += kQuantWarps) {
+    float v = w[c * 32 + lane];
+    float mn = v, mx = v;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    }
+    if (lane == 0) { cmin[c] = mn; cmax[c] = mx; }
+  }
+  __syncthreads();
+
+  for (int gi = warp; gi < G; gi += kQuantWarps) {
+    float mn = INFINITY, mx = -INFINITY;
+    for (int c = lane; c < cpg; c += 32) {
+      mn = fminf(mn, cmin[gi * cpg + c]);
+      mx = fmaxf(mx, cmax[gi * cpg + c]);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    }
+    if (lane == 0) {
+      float s = __fdiv_rn(__fsub_rn(mx, mn), qmax);
+      if (mx == mn) s = 1.0f;
+      float z = rintf(__fdiv_rn(-mn, s));
+      z = fminf(fmaxf(z, 0.0f), qmax);
+      gscale[gi] = s;
+      gzero[gi] = z;
+      scales[(size_t)row * G + gi] = s;
+      zeros[(size_t)row * G + gi] = (uint8_t)z;
+    }
+  }
+  __syncthreads();
+
+  uint32_t* qrow = qweight + (size_t)row * chunks * BITS;
+  for (int c = warp; c < chunks; c += kQuantWarps) {
+    const int gi = c / cpg;
+    const float s = gscale[gi], z = gzero[gi];
+    float q = __fadd_rn(rintf(__fdiv_rn(w[c * 32 + lane], s)), z);
+    q = fminf(fmaxf(q, 0.0f), qmax);
+    warp_pack_store<BITS>((uint32_t)q, lane, qrow + c * BITS);
+  }
+}
+
+template <int BITS>
+__global__ void pack_kernel(const uint8_t* __restrict__ codes, long long total_chunks,
+                            uint32_t* __restrict__ qweight) {
+  const int lane = threadIdx.x & 31;
+  long long c = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const long long stride = ((long long)gridDim.x * blockDim.x) >> 5;
+  for (; c < total_chunks; c += stride) {
+    uint32_t code = codes[c * 32 + lane] & ((1u << BITS) - 1u);
+    warp_pack_store<BITS>(code, lane, qweight + c * BITS);
+  }
+}
+
+template <int BITS>
+__global__ void unpack_kernel(const uint32_t* __restrict__ qweight, long long total_chunks,
+                              uint8_t* __restrict__ codes) {
+  const int lane = threadIdx.x & 31;
+  long long c = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const long long stride = ((long long)gridDim.x * blockDim.x) >> 5;
+  for (; c < total_chunks; c += stride)
+    codes[c * 32 + lane] = (uint8_t)warp_unpack<BITS>(qweight + c * BITS, lane);
+}
+
+// Elementwise AdamW in binary32.  The bias corrections 1-b^t are formed on the
+// host in double and passed in as reciprocals.
+__global__ void adamw_kernel(float* __restrict__ s, const float* __restrict__ grad,
+                             float* __restrict__ m, float* __restrict__ v, long long n,
+                             float lr, float b1, float b2, float eps, float decay,
+                             float inv_c1, float inv_c2) {
+  long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  for (; i < n; i += stride) {
+    const float gr = grad[i];
+    const float mn = b1 * m[i] + (1.0f - b1) * gr;
+    const float vn = b2 * v[i] + (1.0f - b2) * gr * gr;
+    const float denom = sqrtf(vn * inv_c2) + eps;
+    s[i] = s[i] * decay - lr * (mn * inv_c1) / denom;
+    m[i] = mn;
+    v[i] = vn;
+  }
+}
+
+int grid_for(long long work_items, int threads, int max_blocks = 148 * 16) {
+  long long b = (work_items + threads - 1) / threads;
+  if (b < 1) b = 1;
+  if (b > max_blocks) b = max_blocks;
+  return (int)b;
+}
+
+}  // namespace
+
+}  // namespace peqa
+
+using namespace peqa;
+
+extern "C" int peqa_quantize_rtn(const float* W, int N, int K, int bits, int group_size,
+                                 uint32_t* qweight, uint8_t* zeros, float* scales, void* stream) {
+  if (!W || !qweight || !zeros || !scales) return PEQA_ERR_NULL;
+  PEQA_TRY(check_bits_shape(N, K, bits, group_size));
+  if ((K >> 5) > kMaxChunks) return PEQA_ERR_TOO_LARGE;
+  if (!aligned16(W) || !aligned16(qweight) || !aligned16(scales)) return PEQA_ERR_ALIGNMENT;
+  PEQA_TRY(check_arch());
+  const int g = effective_group(K, group_size);
+  cudaStream_t st = as_stream(stream);
+  if (bits == 4)
+    quantize_rtn_kernel<4><<<N, kQuantThreads, 0, st>>>(W, K, g, qweight, zeros, scales);
+  else
+    quantize_rtn_kernel<3><<<N, kQuantThreads, 0, st>>>(W, K, g, qweight, zeros, scales);
+  PEQA_CUDA(cudaGetLastError());
+  return PEQA_OK;
+}
+
+extern "C" int peqa_pack(const uint8_t* codes, int N, int K, int bits, uint32_t* qweight,
+                         void* stream) {
+  if (!codes || !qweight) return PEQA_ERR_NULL;
+  PEQA_TRY(check_bits_shape(N, K, bits, 0));
+  if (!aligned16(qweight)) return PEQA_ERR_ALIGNMENT;
+  PEQA_TRY(check_arch());
+  const long long chunks = (long long)N * (K >> 5);
+  const int grid = grid_for(chunks * 32, 256);
+  cudaStream_t st = as_stream(stream);
+  if (bits == 4) pack_kernel<4><<<grid, 256, 0, st>>>(codes, chunks, qweight);
+  else pack_kernel<3><<<grid, 256, 0, st>>>(codes, chunks, qweight);
+  PEQA_CUDA(cudaGetLastError());
+  return PEQA_OK;
+}
+
+extern "C" int peqa_unpack(const uint32_t* qweight, int N, int K, int bits, uint8_t* codes,
+                           void* stream) {
+  if (!codes || !qweight) return PEQA_ERR_NULL;
+  PEQA_TRY(check_bits_shape(N, K, bits, 0));
+  if (!aligned16(qweight)) return PEQA_ERR_ALIGNMENT;
+  PEQA_TRY(check_arch());
+  const long long chunks = (long long)N * (K >> 5);
+  const int grid = grid_for(chunks * 32, 256);
+  cudaStream_t st = as_stream(stream);
+  if (bits == 4) unpack_kernel<4><<<grid, 256, 0, st>>>(qweight, chunks, codes);
+  else unpack_kernel<3><<<grid, 256, 0, st>>>(qweight, chunks, codes);
+  PEQA_CUDA(cudaGetLastError());
+  return PEQA_OK;
+}
+
+extern "C" int peqa_scale_adamw(float* scales, const float* dS, float* m, float* v, int64_t numel,
+                                float lr, float beta1, float beta2, float eps, float weight_decay,
+                                int64_t step, void* stream) {
+  if (!scales || !dS || !m || !v) return PEQA_ERR_NULL;
+  if (numel <= 0 || step < 1) return PEQA_ERR_BAD_SHAPE;
+  PEQA_TRY(check_arch());
+  const double c1 = 1.0 - pow((double)beta1, (double)step);
+  const double c2 = 1.0 - pow((double)beta2, (double)step);
+  const float decay = (float)(1.0 - (double)lr * (double)weight_decay);
+  const int grid = grid_for(numel, 256);
+  adamw_kernel<<<grid, 256, 0, as_stream(stream)>>>(scales, dS, m, v, (long long)numel, lr, beta1,
+                                                   beta2, eps, decay, (float)(1.0 / c1),
+                                                   (float)(1.0 / c2));
+  PEQA_CUDA(cudaGetLastError());
+  return PEQA_OK;
+}
