@@ -1,0 +1,234 @@
+"""ctypes binding of libpeqa_b200.so: argument marshalling only.
+
+Every function has the name of the C entry point it calls (see include/peqa.h)
+minus the ``peqa_`` prefix.  torch provides device memory and the current
+stream; all arithmetic runs in the library's CUDA kernels.  There is no CPU
+fallback: a missing library or a non-zero status raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libpeqa_b200.so")
+_lib = None
+
+OP_FWD, OP_BWD, OP_DECODE = 0, 1, 2
+
+STATUS_NAMES = {
+    0: "PEQA_OK", -1: "PEQA_ERR_NULL", -2: "PEQA_ERR_BAD_BITS", -3: "PEQA_ERR_BAD_SHAPE",
+    -4: "PEQA_ERR_ALIGNMENT", -5: "PEQA_ERR_WORKSPACE", -6: "PEQA_ERR_ARCH", -7: "PEQA_ERR_CUDA",
+    -8: "PEQA_ERR_DEVICE_TIMEOUT", -9: "PEQA_ERR_TOO_LARGE",
+}
+
+
+class PeqaError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        extra = ""
+        if status == -7 and _lib is not None:
+            extra = f" (cudaError {_lib.peqa_last_cuda_error()})"
+        super().__init__(f"{where}: {STATUS_NAMES.get(status, status)}{extra}")
+
+
+class _QWeight(ctypes.Structure):
+    _fields_ = [("bits", ctypes.c_int32), ("out_features", ctypes.c_int32),
+                ("in_features", ctypes.c_int32), ("group_size", ctypes.c_int32),
+                ("qweight", ctypes.c_void_p), ("zeros", ctypes.c_void_p),
+                ("scales", ctypes.c_void_p)]
+
+
+def lib() -> ctypes.CDLL:
+    """Load the shared library (built by paper_2305_14152_b200.build); never falls back."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                f"{LIB_PATH} is missing: run `python -m paper_2305_14152_b200.build` first; "
+                "there is no CPU fallback")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i32, i64, f32, sz = (ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_float,
+                                 ctypes.c_size_t)
+        qp = ctypes.POINTER(_QWeight)
+        L.peqa_version.restype = ctypes.c_int
+        L.peqa_last_cuda_error.restype = ctypes.c_int
+        L.peqa_quantize_rtn.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, vp]
+        L.peqa_pack.argtypes = [vp, i32, i32, i32, vp, vp]
+        L.peqa_unpack.argtypes = [vp, i32, i32, i32, vp, vp]
+        L.peqa_workspace_bytes.argtypes = [i32, i32, qp]
+        L.peqa_workspace_bytes.restype = sz
+        L.peqa_qlinear_fwd.argtypes = [qp, vp, i32, vp, vp, sz, vp]
+        L.peqa_qlinear_bwd.argtypes = [qp, vp, vp, i32, vp, vp, vp, sz, vp]
+        L.peqa_qlinear_decode.argtypes = [qp, vp, i32, vp, vp, sz, vp]
+        L.peqa_scale_adamw.argtypes = [vp, vp, vp, vp, i64, f32, f32, f32, f32, f32, i64, vp]
+        L.peqa_train_step_host.argtypes = [qp, i32] + [vp] * 12 + [f32] * 5 + [i64, vp, sz, vp]
+        L.peqa_check_status.argtypes = [vp]
+        for name in ("peqa_quantize_rtn", "peqa_pack", "peqa_unpack", "peqa_qlinear_fwd",
+                     "peqa_qlinear_bwd", "peqa_qlinear_decode", "peqa_scale_adamw",
+                     "peqa_train_step_host", "peqa_check_status"):
+            getattr(L, name).restype = ctypes.c_int
+        _lib = L
+    return _lib
+
+
+def _check(status: int, where: str) -> None:
+    if status != 0:
+        raise PeqaError(status, where)
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _ptr(t) -> int:
+    return 0 if t is None else t.data_ptr()
+
+
+def _dev(t: torch.Tensor, dtype, name: str) -> torch.Tensor:
+    if not t.is_cuda or t.dtype != dtype or not t.is_contiguous():
+        raise ValueError(f"{name}: expected a contiguous CUDA tensor of {dtype}")
+    return t
+
+
+@dataclass
+class QWeight:
+    """Device tensors of one PEQA layer: packed Q (int32 bit patterns), z (uint8), s (fp32)."""
+    bits: int
+    N: int
+    K: int
+    group_size: int          # 0 = per-channel
+    qweight: torch.Tensor    # int32 [N, K*bits/32]
+    zeros: torch.Tensor      # uint8 [N, G]
+    scales: torch.Tensor     # float32 [N, G]
+
+    @property
+    def G(self) -> int:
+        return 1 if self.group_size in (0, self.K) else self.K // self.group_size
+
+    def c_struct(self) -> _QWeight:
+        return _QWeight(self.bits, self.N, self.K, self.group_size, self.qweight.data_ptr(),
+                        self.zeros.data_ptr(), self.scales.data_ptr())
+
+
+def version() -> int:
+    return lib().peqa_version()
+
+
+def quantize_rtn(W: torch.Tensor, bits: int, group_size: int = 0) -> QWeight:
+    _dev(W, torch.float32, "W")
+    N, K = W.shape
+    G = 1 if group_size in (0, K) else max(K // max(group_size, 1), 1)
+    words = max(K * bits // 32, 1)
+    q = torch.empty((N, words), dtype=torch.int32, device=W.device)
+    z = torch.empty((N, G), dtype=torch.uint8, device=W.device)
+    s = torch.empty((N, G), dtype=torch.float32, device=W.device)
+    _check(lib().peqa_quantize_rtn(W.data_ptr(), N, K, bits, group_size, q.data_ptr(), z.data_ptr(),
+                                   s.data_ptr(), _stream()), "peqa_quantize_rtn")
+    return QWeight(bits, N, K, group_size, q, z, s)
+
+
+def pack(codes: torch.Tensor, bits: int) -> torch.Tensor:
+    _dev(codes, torch.uint8, "codes")
+    N, K = codes.shape
+    q = torch.empty((N, max(K * bits // 32, 1)), dtype=torch.int32, device=codes.device)
+    _check(lib().peqa_pack(codes.data_ptr(), N, K, bits, q.data_ptr(), _stream()), "peqa_pack")
+    return q
+
+
+def unpack(qweight: torch.Tensor, K: int, bits: int) -> torch.Tensor:
+    _dev(qweight, torch.int32, "qweight")
+    N = qweight.shape[0]
+    codes = torch.empty((N, K), dtype=torch.uint8, device=qweight.device)
+    _check(lib().peqa_unpack(qweight.data_ptr(), N, K, bits, codes.data_ptr(), _stream()),
+           "peqa_unpack")
+    return codes
+
+
+def workspace_bytes(op: int, T: int, w: QWeight) -> int:
+    cs = w.c_struct()
+    return int(lib().peqa_workspace_bytes(op, T, ctypes.byref(cs)))
+
+
+def alloc_workspace(op: int, T: int, w: QWeight):
+    n = workspace_bytes(op, T, w)
+    if n == 0:
+        return None
+    return torch.empty(n, dtype=torch.uint8, device=w.qweight.device)
+
+
+def _ws(ws):
+    return (0, 0) if ws is None else (ws.data_ptr(), ws.numel() * ws.element_size())
+
+
+def qlinear_fwd(w: QWeight, X: torch.Tensor, Y: torch.Tensor | None = None, workspace=None):
+    _dev(X, torch.bfloat16, "X")
+    T = X.shape[0]
+    if Y is None:
+        Y = torch.empty((T, w.N), dtype=torch.bfloat16, device=X.device)
+    cs = w.c_struct()
+    wp, wb = _ws(workspace)
+    _check(lib().peqa_qlinear_fwd(ctypes.byref(cs), X.data_ptr(), T, Y.data_ptr(), wp, wb,
+                                  _stream()), "peqa_qlinear_fwd")
+    return Y
+
+
+def qlinear_bwd(w: QWeight, X, dY: torch.Tensor, dX=None, dS=None, workspace=None,
+                need_dx: bool = True, need_ds: bool = True):
+    _dev(dY, torch.bfloat16, "dY")
+    T = dY.shape[0]
+    if need_dx and dX is None:
+        dX = torch.empty((T, w.K), dtype=torch.bfloat16, device=dY.device)
+    if need_ds and dS is None:
+        dS = torch.empty((w.N, w.G), dtype=torch.float32, device=dY.device)
+    if need_ds and workspace is None:
+        workspace = alloc_workspace(OP_BWD, T, w)
+    cs = w.c_struct()
+    wp, wb = _ws(workspace)
+    _check(lib().peqa_qlinear_bwd(ctypes.byref(cs), _ptr(X), dY.data_ptr(), T,
+                                  _ptr(dX) if need_dx else 0, _ptr(dS) if need_ds else 0,
+                                  wp, wb, _stream()), "peqa_qlinear_bwd")
+    return dX, dS
+
+
+def qlinear_decode(w: QWeight, X: torch.Tensor, Y: torch.Tensor | None = None, workspace=None):
+    _dev(X, torch.bfloat16, "X")
+    M = X.shape[0]
+    if Y is None:
+        Y = torch.empty((M, w.N), dtype=torch.bfloat16, device=X.device)
+    if workspace is None:
+        workspace = alloc_workspace(OP_DECODE, M, w)
+    cs = w.c_struct()
+    wp, wb = _ws(workspace)
+    _check(lib().peqa_qlinear_decode(ctypes.byref(cs), X.data_ptr(), M, Y.data_ptr(), wp, wb,
+                                     _stream()), "peqa_qlinear_decode")
+    return Y
+
+
+def scale_adamw(scales, dS, m, v, lr, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.0, step=1):
+    for t, n in ((scales, "scales"), (dS, "dS"), (m, "m"), (v, "v")):
+        _dev(t, torch.float32, n)
+    _check(lib().peqa_scale_adamw(scales.data_ptr(), dS.data_ptr(), m.data_ptr(), v.data_ptr(),
+                                  scales.numel(), lr, beta1, beta2, eps, weight_decay, step,
+                                  _stream()), "peqa_scale_adamw")
+
+
+def train_step_host(w: QWeight, h_X, h_dY, h_Y, h_dX, h_dS, d_X, d_dY, d_Y, d_dX, d_dS, d_m, d_v,
+                    lr, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.0, step=1,
+                    workspace=None):
+    """Host-buffer training step: h_* are CPU tensors (pinned preferred), d_* device staging."""
+    T = h_X.shape[0]
+    cs = w.c_struct()
+    wp, wb = _ws(workspace)
+    _check(lib().peqa_train_step_host(
+        ctypes.byref(cs), T, h_X.data_ptr(), h_dY.data_ptr(), h_Y.data_ptr(), h_dX.data_ptr(),
+        h_dS.data_ptr(), d_X.data_ptr(), d_dY.data_ptr(), d_Y.data_ptr(), d_dX.data_ptr(),
+        d_dS.data_ptr(), d_m.data_ptr(), d_v.data_ptr(), lr, beta1, beta2, eps, weight_decay, step,
+        wp, wb, _stream()), "peqa_train_step_host")
+
+
+def check_status() -> None:
+    _check(lib().peqa_check_status(_stream()), "peqa_check_status")

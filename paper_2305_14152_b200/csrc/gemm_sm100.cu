@@ -1,0 +1,678 @@
+// Tensor-core kernels of the PEQA layer for sm_100a.
+//
+//   qgemm_kernel<TRANS=false>  Y[t,i]  = sum_j X[t,j]  * W_hat[i,j]     (forward, Eq. 2)
+//   qgemm_kernel<TRANS=true>   dX[t,j] = sum_i dY[t,i] * W_hat[i,j]     (backward wrt input)
+//   ds_kernel                  dS[i,g] = sum_{j in g} (Q-z)[i,j] * (dY^T X)[i,j]
+//
+// All three are persistent, warp-specialised kernels: one CTA per SM walks a
+// static list of 128x256 output tiles.  Activations arrive by TMA into
+// 128-byte-swizzled shared memory, tcgen05.mma accumulates fp32 in tensor
+// memory (two 256-column accumulators, so the epilogue of one tile overlaps
+// the main loop of the next), and every mbarrier wait is bounded.
+//
+// In qgemm the weight operand never exists in HBM as bf16: dedicated warps
+// read the packed codes, rebuild (Q - z) [times bf16(s) when the scale varies
+// along the contraction] in registers and write the bf16 tile straight into
+// the swizzled layout the tensor core reads.  The weight tile is the MMA "A"
+// operand (M = 128 weight rows/columns), the activation tile the "B" operand
+// (N = 256 tokens), so each weight is dequantised once per 256 tokens.
+//   forward : A is K-major   (row = out channel i, 64 contraction columns j)
+//   dX      : A is MN-major  (row = contraction index i, 128 columns j) --
+//             the same row-wise unpack, only the descriptor differs, so Q is
+//             "read transposed" without any transposed copy.
+//
+// In ds_kernel both operands are activations (dY^T and X, MN-major straight
+// from their row-major storage); the 128x256 dW tile stays in tensor memory,
+// and the epilogue multiplies it by (Q - z) and sums over column pieces that
+// lie inside one group.  dW never reaches HBM.
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include "common.cuh"
+#include "dequant.cuh"
+#include "sm100_ptx.cuh"
+
+namespace peqa {
+
+namespace {
+
+using namespace ptx;
+
+constexpr int BM = 128;      // weight rows per tile (MMA M, TMEM lanes)
+constexpr int BN = 256;      // tokens (qgemm) / weight columns (ds) per tile (MMA N)
+constexpr int BK = 64;       // contraction elements per pipeline stage
+constexpr int UMMA_K = 16;   // contraction elements per tcgen05.mma
+constexpr int STAGES = 4;
+constexpr int A_BYTES = BM * BK * 2;   // 16 KiB
+constexpr int B_BYTES = BN * BK * 2;   // 32 KiB
+constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int TMEM_COLS = 512;         // two fp32 accumulators of 256 columns
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/;
+
+constexpr int kQgemmThreads = 512;     // warps: 0 TMA, 1 MMA, 2 TMEM alloc, 4-7 epilogue, 8-15 dequant
+constexpr int kDequantThreads = 256;
+constexpr int kDsThreads = 384;        // warps: 0 TMA, 1 MMA, 2 TMEM alloc, 4-11 epilogue
+
+struct Barriers {
+  uint64_t full_a[STAGES];   // dequantised weight tile written (qgemm only)
+  uint64_t full_b[STAGES];   // TMA bytes landed
+  uint64_t empty[STAGES];    // MMAs that read the stage have completed
+  uint64_t acc_full[2];      // accumulator ready for the epilogue
+  uint64_t acc_empty[2];     // accumulator drained by the epilogue
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+struct SmemView {
+  uint8_t* a[STAGES];
+  uint8_t* b[STAGES];
+  Barriers* bars;
+};
+
+__device__ __forceinline__ SmemView carve_smem(uint8_t* raw) {
+  uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(raw) + 1023) &
+                                             ~static_cast<uintptr_t>(1023));
+  SmemView v;
+#pragma unroll
+  for (int s = 0; s < STAGES; ++s) {
+    v.a[s] = base + s * STAGE_BYTES;
+    v.b[s] = base + s * STAGE_BYTES + A_BYTES;
+  }
+  v.bars = reinterpret_cast<Barriers*>(base + STAGES * STAGE_BYTES);
+  return v;
+}
+
+// After a bounded wait gave up: let copies and MMAs already in flight finish
+// before shared and tensor memory are released.
+__device__ __forceinline__ void drain_after_abort() {
+  for (int i = 0; i < 64; ++i) __nanosleep(1000);
+}
+
+struct QGemmParams {
+  const uint32_t* qw;
+  const uint8_t* zeros;
+  const float* scales;
+  __nv_bfloat16* out;   // [T, R]
+  int N, K, G, g, T;
+  int wpr;              // packed words per weight row
+  int R, C;             // output features, contraction length
+  int r_tiles, t_tiles, k_blocks;
+  int* status;
+};
+
+// Packed words, zero-point and scale of one 32-column unit of one weight row.
+template <int BITS>
+struct Unit {
+  uint32_t w[BITS];
+  uint32_t z;
+  float s;
+};
+
+template <int BITS, bool TRANS>
+__device__ __forceinline__ Unit<BITS> load_unit(const QGemmParams& p, int r0, int c0, int dq) {
+  int i, col0;
+  if (!TRANS) {
+    i = r0 + (dq & 127);
+    col0 = c0 + 32 * (dq >> 7);
+  } else {
+    i = c0 + (dq & 63);
+    col0 = r0 + 32 * (dq >> 6);
+  }
+  Unit<BITS> u;
+  if (i < p.N && col0 < p.K) {
+    const uint32_t* src = p.qw + (size_t)i * p.wpr + (col0 >> 5) * BITS;
+    if constexpr (BITS == 4) {
+      const uint4 v = __ldg(reinterpret_cast<const uint4*>(src));
+      u.w[0] = v.x; u.w[1] = v.y; u.w[2] = v.z; u.w[3] = v.w;
+    } else {
+      u.w[0] = __ldg(src); u.w[1] = __ldg(src + 1); u.w[2] = __ldg(src + 2);
+    }
+    const size_t gidx = (size_t)i * p.G + col0 / p.g;
+    u.z = __ldg(p.zeros + gidx);
+    u.s = __ldg(p.scales + gidx);
+  } else {
+    // Outside the matrix: codes equal to the zero-point dequantise to exactly 0.
+#pragma unroll
+    for (int q = 0; q < BITS; ++q) u.w[q] = 0u;
+    u.z = 0u;
+    u.s = 0.0f;
+  }
+  return u;
+}
+
+template <int BITS, bool TRANS, bool FOLD>
+__global__ void __launch_bounds__(kQgemmThreads, 1)
+qgemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const QGemmParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  SmemView sm = carve_smem(smem_raw);
+  Barriers* bars = sm.bars;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  volatile int* abort_flag = &bars->abort_flag;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(smem_u32(&bars->full_a[s]), kDequantThreads);
+      mbar_init(smem_u32(&bars->full_b[s]), 1);
+      mbar_init(smem_u32(&bars->empty[s]), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(smem_u32(&bars->acc_full[b]), 1);
+      mbar_init(smem_u32(&bars->acc_empty[b]), 128);
+    }
+    bars->abort_flag = 0;
+    fence_mbar_init();
+    prefetch_tmap(&tmap_act);
+  }
+  if (warp == 2) {
+    tmem_alloc(smem_u32(&bars->tmem_base), TMEM_COLS);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = bars->tmem_base;
+
+  const int total_tiles = p.r_tiles * p.t_tiles;
+
+  if (warp == 0) {
+    // ------------------------------------------------ TMA producer (one lane)
+    if (lane == 0) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+        const int t0 = (tile / p.r_tiles) * BN;
+        for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
+          const int s = it % STAGES;
+          const uint32_t ph = (it / STAGES) & 1u;
+          if (!mbar_wait(smem_u32(&bars->empty[s]), ph ^ 1u, abort_flag)) { ok = false; break; }
+          const uint32_t bar = smem_u32(&bars->full_b[s]);
+          mbar_arrive_expect_tx(bar, B_BYTES);
+          tma_load_2d(smem_u32(sm.b[s]), &tmap_act, bar, kb * BK, t0);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------- MMA issuer (one lane)
+    if (lane == 0) {
+      constexpr uint32_t idesc = idesc_bf16_f32(BM, BN, TRANS ? 1 : 0, 0);
+      uint32_t it = 0;
+      int local = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++local) {
+        const int buf = local & 1;
+        const uint32_t acc_ph = (local >> 1) & 1u;
+        if (!mbar_wait(smem_u32(&bars->acc_empty[buf]), acc_ph ^ 1u, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + buf * BN;
+        for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
+          const int s = it % STAGES;
+          const uint32_t ph = (it / STAGES) & 1u;
+          if (!mbar_wait(smem_u32(&bars->full_a[s]), ph, abort_flag) ||
+              !mbar_wait(smem_u32(&bars->full_b[s]), ph, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t a_addr = smem_u32(sm.a[s]);
+          const uint32_t b_addr = smem_u32(sm.b[s]);
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k) {
+            const uint64_t adesc = TRANS
+                ? smem_desc_sw128(a_addr + k * (UMMA_K * 128), 64 * 128, 1024)
+                : smem_desc_sw128(a_addr + k * (UMMA_K * 2), 16, 1024);
+            const uint64_t bdesc = smem_desc_sw128(b_addr + k * (UMMA_K * 2), 16, 1024);
+            mma_bf16_ss(d_tmem, adesc, bdesc, idesc, (kb | k) != 0 ? 1u : 0u);
+          }
+          mma_commit(smem_u32(&bars->empty[s]));
+        }
+        if (ok) mma_commit(smem_u32(&bars->acc_full[buf]));
+      }
+    }
+  } else if (warp >= 4 && warp < 8) {
+    // ------------------------------------------------------------- epilogue
+    const int ew = warp - 4;  // == warp % 4: the TMEM lane quarter this warp may read
+    int local = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++local) {
+      const int r0 = (tile % p.r_tiles) * BM;
+      const int t0 = (tile / p.r_tiles) * BN;
+      const int buf = local & 1;
+      const uint32_t acc_ph = (local >> 1) & 1u;
+      if (!mbar_wait(smem_u32(&bars->acc_full[buf]), acc_ph, abort_flag)) { ok = false; break; }
+      tc_fence_after();
+      const int r = r0 + ew * 32 + lane;
+      float scale = 1.0f;
+      if (!FOLD && r < p.R) scale = __ldg(p.scales + r);  // per-channel forward: s[i] applied here
+#pragma unroll 1
+      for (int cc = 0; cc < BN / 32; ++cc) {
+        const int tc0 = t0 + cc * 32;
+        if (tc0 >= p.T) break;
+        uint32_t v[32];
+        tmem_ld_32x32(tmem_base + ((uint32_t)(ew * 32) << 16) + buf * BN + cc * 32, v);
+        tmem_ld_wait();
+        if (r < p.R) {
+          __nv_bfloat16* dst = p.out + (size_t)tc0 * p.R + r;
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            if (tc0 + j < p.T) dst[(size_t)j * p.R] = __float2bfloat16_rn(__uint_as_float(v[j]) * scale);
+          }
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(smem_u32(&bars->acc_empty[buf]));
+    }
+  } else if (warp >= 8) {
+    // ------------------------------------------------------- weight dequant
+    const int dq = threadIdx.x - 256;
+    // Destination of this thread's 32 columns (64 bytes = four 16-byte chunks)
+    // inside the 128-byte-swizzled tile: 16-byte chunk index XOR (row & 7).
+    int row_off, chunk0, swz;
+    if (!TRANS) {
+      const int row = dq & 127;
+      row_off = row * 128;
+      chunk0 = (dq >> 7) * 4;
+      swz = row & 7;
+    } else {
+      const int crow = dq & 63;
+      const int quarter = dq >> 6;
+      row_off = (quarter >> 1) * (64 * 128) + crow * 128;
+      chunk0 = (quarter & 1) * 4;
+      swz = crow & 7;
+    }
+    const int my_tiles = (total_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+    const uint32_t total_it = (uint32_t)my_tiles * (uint32_t)p.k_blocks;
+    // Flattened (tile, k-block) walk with a two-deep register prefetch of the
+    // packed words so that global latency hides behind the conversions.
+    auto coords = [&](uint32_t it, int& r0, int& c0) {
+      const int tile = blockIdx.x + (int)(it / (uint32_t)p.k_blocks) * gridDim.x;
+      r0 = (tile % p.r_tiles) * BM;
+      c0 = (int)(it % (uint32_t)p.k_blocks) * BK;
+    };
+    Unit<BITS> u0, u1;
+    {
+      int r0, c0;
+      if (total_it > 0) { coords(0, r0, c0); u0 = load_unit<BITS, TRANS>(p, r0, c0, dq); }
+      if (total_it > 1) { coords(1, r0, c0); u1 = load_unit<BITS, TRANS>(p, r0, c0, dq); }
+    }
+    for (uint32_t it = 0; it < total_it; ++it) {
+      const Unit<BITS> cur = u0;
+      u0 = u1;
+      if (it + 2 < total_it) {
+        int r0, c0;
+        coords(it + 2, r0, c0);
+        u1 = load_unit<BITS, TRANS>(p, r0, c0, dq);
+      }
+      const int s = it % STAGES;
+      const uint32_t ph = (it / STAGES) & 1u;
+      uint32_t o[16];
+      dq::unit32_natural<BITS, FOLD>(cur.w, cur.z, cur.s, o);
+      if (!mbar_wait(smem_u32(&bars->empty[s]), ph ^ 1u, abort_flag)) break;
+      uint8_t* dst = sm.a[s] + row_off;
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        *reinterpret_cast<uint4*>(dst + (((chunk0 + q) ^ swz) << 4)) =
+            make_uint4(o[4 * q], o[4 * q + 1], o[4 * q + 2], o[4 * q + 3]);
+      }
+      fence_proxy_async_smem();
+      mbar_arrive(smem_u32(&bars->full_a[s]));
+    }
+  }
+
+  // ---------------------------------------------------------------- teardown
+  if (*abort_flag) drain_after_abort();
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 2) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, TMEM_COLS);
+  }
+  if (threadIdx.x == 0 && bars->abort_flag) {
+    atomicExch(p.status, (int)PEQA_ERR_DEVICE_TIMEOUT);
+    p.status[1] = (int)blockIdx.x;
+  }
+}
+
+// ------------------------------------------------------------------- dS ---
+struct DsParams {
+  const uint32_t* qw;
+  const uint8_t* zeros;
+  float* out;        // [N, K / piece]: dS itself when piece == g, else partial sums
+  int N, K, G, g, T;
+  int wpr;
+  int piece;         // columns per output piece: 32, 64 or 128; divides g
+  int i_tiles, j_tiles, k_blocks;
+  int* status;
+};
+
+template <int BITS>
+__global__ void __launch_bounds__(kDsThreads, 1)
+ds_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_constant__ CUtensorMap tmap_x,
+          const DsParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  SmemView sm = carve_smem(smem_raw);
+  Barriers* bars = sm.bars;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  volatile int* abort_flag = &bars->abort_flag;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(smem_u32(&bars->full_a[s]), 1);   // unused here
+      mbar_init(smem_u32(&bars->full_b[s]), 1);
+      mbar_init(smem_u32(&bars->empty[s]), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(smem_u32(&bars->acc_full[b]), 1);
+      mbar_init(smem_u32(&bars->acc_empty[b]), 256);
+    }
+    bars->abort_flag = 0;
+    fence_mbar_init();
+    prefetch_tmap(&tmap_dy);
+    prefetch_tmap(&tmap_x);
+  }
+  if (warp == 2) {
+    tmem_alloc(smem_u32(&bars->tmem_base), TMEM_COLS);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = bars->tmem_base;
+  const int total_tiles = p.i_tiles * p.j_tiles;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+        const int i0 = (tile % p.i_tiles) * BM;
+        const int j0 = (tile / p.i_tiles) * BN;
+        for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
+          const int s = it % STAGES;
+          const uint32_t ph = (it / STAGES) & 1u;
+          if (!mbar_wait(smem_u32(&bars->empty[s]), ph ^ 1u, abort_flag)) { ok = false; break; }
+          const uint32_t bar = smem_u32(&bars->full_b[s]);
+          mbar_arrive_expect_tx(bar, STAGE_BYTES);
+          // Each box is 64 contiguous features x 64 tokens = one 8 KiB MN-major chunk.
+#pragma unroll
+          for (int m = 0; m < BM / 64; ++m)
+            tma_load_2d(smem_u32(sm.a[s]) + m * 8192, &tmap_dy, bar, i0 + 64 * m, kb * BK);
+#pragma unroll
+          for (int m = 0; m < BN / 64; ++m)
+            tma_load_2d(smem_u32(sm.b[s]) + m * 8192, &tmap_x, bar, j0 + 64 * m, kb * BK);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      constexpr uint32_t idesc = idesc_bf16_f32(BM, BN, 1, 1);
+      uint32_t it = 0;
+      int local = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++local) {
+        const int buf = local & 1;
+        const uint32_t acc_ph = (local >> 1) & 1u;
+        if (!mbar_wait(smem_u32(&bars->acc_empty[buf]), acc_ph ^ 1u, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + buf * BN;
+        for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
+          const int s = it % STAGES;
+          const uint32_t ph = (it / STAGES) & 1u;
+          if (!mbar_wait(smem_u32(&bars->full_b[s]), ph, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t a_addr = smem_u32(sm.a[s]);
+          const uint32_t b_addr = smem_u32(sm.b[s]);
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k) {
+            const uint64_t adesc = smem_desc_sw128(a_addr + k * (UMMA_K * 128), 8192, 1024);
+            const uint64_t bdesc = smem_desc_sw128(b_addr + k * (UMMA_K * 128), 8192, 1024);
+            mma_bf16_ss(d_tmem, adesc, bdesc, idesc, (kb | k) != 0 ? 1u : 0u);
+          }
+          mma_commit(smem_u32(&bars->empty[s]));
+        }
+        if (ok) mma_commit(smem_u32(&bars->acc_full[buf]));
+      }
+    }
+  } else if (warp >= 4) {
+    // Epilogue: thread = one weight row i (TMEM lane) and one 128-column half.
+    const int quarter = warp & 3;
+    const int half = (warp - 4) >> 2;
+    const int npieces = p.K / p.piece;
+    const int chunks_per_piece = p.piece >> 5;
+    int local = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++local) {
+      const int i0 = (tile % p.i_tiles) * BM;
+      const int j0 = (tile / p.i_tiles) * BN;
+      const int buf = local & 1;
+      const uint32_t acc_ph = (local >> 1) & 1u;
+      if (!mbar_wait(smem_u32(&bars->acc_full[buf]), acc_ph, abort_flag)) { ok = false; break; }
+      tc_fence_after();
+      const int i = i0 + quarter * 32 + lane;
+      float acc = 0.0f;
+#pragma unroll 1
+      for (int cc = 0; cc < 4; ++cc) {
+        const int col0 = j0 + half * 128 + cc * 32;
+        if (col0 >= p.K) break;
+        uint32_t v[32];
+        tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * BN + half * 128 + cc * 32, v);
+        const bool row_ok = i < p.N;
+        uint32_t w[BITS];
+        uint32_t z = 0u;
+#pragma unroll
+        for (int q = 0; q < BITS; ++q) w[q] = 0u;
+        if (row_ok) {
+          const uint32_t* src = p.qw + (size_t)i * p.wpr + (col0 >> 5) * BITS;
+          if constexpr (BITS == 4) {
+            const uint4 q4 = __ldg(reinterpret_cast<const uint4*>(src));
+            w[0] = q4.x; w[1] = q4.y; w[2] = q4.z; w[3] = q4.w;
+          } else {
+            w[0] = __ldg(src); w[1] = __ldg(src + 1); w[2] = __ldg(src + 2);
+          }
+          z = __ldg(p.zeros + (size_t)i * p.G + col0 / p.g);
+        }
+        uint32_t o[16];
+        dq::unit32_natural<BITS, false>(w, z, 0.0f, o);
+        tmem_ld_wait();   // warp-wide: every lane executes it, ragged rows included
+#pragma unroll
+        for (int q = 0; q < 16; ++q) {
+          acc = fmaf(__uint_as_float(v[2 * q]), __uint_as_float(o[q] << 16), acc);
+          acc = fmaf(__uint_as_float(v[2 * q + 1]), __uint_as_float(o[q] & 0xFFFF0000u), acc);
+        }
+        if (((cc + 1) % chunks_per_piece) == 0) {
+          if (row_ok) p.out[(size_t)i * npieces + col0 / p.piece] = acc;
+          acc = 0.0f;
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(smem_u32(&bars->acc_empty[buf]));
+    }
+  }
+
+  if (*abort_flag) drain_after_abort();
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 2) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, TMEM_COLS);
+  }
+  if (threadIdx.x == 0 && bars->abort_flag) {
+    atomicExch(p.status, (int)PEQA_ERR_DEVICE_TIMEOUT);
+    p.status[1] = (int)blockIdx.x;
+  }
+}
+
+// dS[i, gi] = sum of the group's partial pieces, in index order (deterministic).
+__global__ void ds_reduce_kernel(const float* __restrict__ partial, float* __restrict__ dS,
+                                 long long n_out, int pieces_per_group) {
+  long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= n_out) return;
+  const float* src = partial + e * pieces_per_group;
+  float acc = 0.0f;
+  for (int q = 0; q < pieces_per_group; ++q) acc += src[q];
+  dS[e] = acc;
+}
+
+// --------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+int get_encode_fn(EncodeTiledFn* out) {
+  static EncodeTiledFn cached = nullptr;
+  if (!cached) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    PEQA_CUDA(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
+    if (!fn || qres != cudaDriverEntryPointSuccess) return cuda_fail(cudaErrorUnknown);
+    cached = reinterpret_cast<EncodeTiledFn>(fn);
+  }
+  *out = cached;
+  return PEQA_OK;
+}
+
+// bf16 row-major [outer, inner] tensor, box = [box_outer rows, 64 elements], 128B swizzle,
+// out-of-bounds elements read as zero.
+int make_tmap_bf16(CUtensorMap* m, const void* base, uint64_t inner, uint64_t outer,
+                   uint32_t box_outer) {
+  EncodeTiledFn enc = nullptr;
+  PEQA_TRY(get_encode_fn(&enc));
+  cuuint64_t dims[2] = {inner, outer};
+  cuuint64_t strides[1] = {inner * 2};
+  cuuint32_t box[2] = {64, box_outer};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides,
+                   box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return cuda_fail(cudaErrorInvalidValue);
+  return PEQA_OK;
+}
+
+int sm_count(int* n) {
+  static thread_local int cached_dev = -1, cached_n = 0;
+  int dev = 0;
+  PEQA_CUDA(cudaGetDevice(&dev));
+  if (dev != cached_dev) {
+    PEQA_CUDA(cudaDeviceGetAttribute(&cached_n, cudaDevAttrMultiProcessorCount, dev));
+    cached_dev = dev;
+  }
+  *n = cached_n;
+  return PEQA_OK;
+}
+
+template <typename Kern>
+int set_smem(Kern k) {
+  PEQA_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
+  return PEQA_OK;
+}
+
+template <int BITS, bool TRANS, bool FOLD>
+int launch_qgemm_t(const CUtensorMap& tmap, const QGemmParams& p, int grid, cudaStream_t st) {
+  auto kern = qgemm_kernel<BITS, TRANS, FOLD>;
+  PEQA_TRY(set_smem(kern));
+  kern<<<grid, kQgemmThreads, SMEM_BYTES, st>>>(tmap, p);
+  PEQA_CUDA(cudaGetLastError());
+  return PEQA_OK;
+}
+
+int launch_qgemm(const peqa_qweight_t* w, int g, const void* act, int T, void* out, bool trans,
+                 cudaStream_t st) {
+  QGemmParams p;
+  p.qw = w->qweight;
+  p.zeros = w->zeros;
+  p.scales = w->scales;
+  p.out = static_cast<__nv_bfloat16*>(out);
+  p.N = w->out_features;
+  p.K = w->in_features;
+  p.g = g;
+  p.G = p.K / g;
+  p.T = T;
+  p.wpr = p.K * w->bits / 32;
+  p.R = trans ? p.K : p.N;
+  p.C = trans ? p.N : p.K;
+  p.r_tiles = (p.R + BM - 1) / BM;
+  p.t_tiles = (T + BN - 1) / BN;
+  p.k_blocks = (p.C + BK - 1) / BK;
+  PEQA_TRY(status_word(&p.status));
+  CUtensorMap tmap;
+  PEQA_TRY(make_tmap_bf16(&tmap, act, (uint64_t)p.C, (uint64_t)T, BN));
+  int sms = 0;
+  PEQA_TRY(sm_count(&sms));
+  const int tiles = p.r_tiles * p.t_tiles;
+  const int grid = tiles < sms ? tiles : sms;
+  const bool fold = trans || p.G > 1;
+  if (w->bits == 4) {
+    if (trans) return launch_qgemm_t<4, true, true>(tmap, p, grid, st);
+    return fold ? launch_qgemm_t<4, false, true>(tmap, p, grid, st)
+                : launch_qgemm_t<4, false, false>(tmap, p, grid, st);
+  }
+  if (trans) return launch_qgemm_t<3, true, true>(tmap, p, grid, st);
+  return fold ? launch_qgemm_t<3, false, true>(tmap, p, grid, st)
+              : launch_qgemm_t<3, false, false>(tmap, p, grid, st);
+}
+
+int gcd_int(int a, int b) { return b == 0 ? a : gcd_int(b, a % b); }
+
+// Columns per dS output piece: the largest of {32, 64, 128} that divides g, so
+// that a piece never crosses a group or a 128-column epilogue half.
+int ds_piece(int g) { return gcd_int(g, 128); }
+
+}  // namespace
+
+int launch_fwd(const peqa_qweight_t* w, int g, const void* X, int T, void* Y, cudaStream_t st) {
+  return launch_qgemm(w, g, X, T, Y, false, st);
+}
+
+int launch_dx(const peqa_qweight_t* w, int g, const void* dY, int T, void* dX, cudaStream_t st) {
+  return launch_qgemm(w, g, dY, T, dX, true, st);
+}
+
+size_t ds_workspace_bytes(const peqa_qweight_t* w, int g, int T) {
+  (void)T;
+  const int piece = ds_piece(g);
+  if (piece == g) return 0;
+  return (size_t)w->out_features * (size_t)(w->in_features / piece) * sizeof(float);
+}
+
+int launch_ds(const peqa_qweight_t* w, int g, const void* X, const void* dY, int T, float* dS,
+              void* workspace, size_t workspace_bytes, cudaStream_t st) {
+  (void)workspace_bytes;
+  DsParams p;
+  p.qw = w->qweight;
+  p.zeros = w->zeros;
+  p.N = w->out_features;
+  p.K = w->in_features;
+  p.g = g;
+  p.G = p.K / g;
+  p.T = T;
+  p.wpr = p.K * w->bits / 32;
+  p.piece = ds_piece(g);
+  const bool direct = (p.piece == g);
+  p.out = direct ? dS : static_cast<float*>(workspace);
+  p.i_tiles = (p.N + BM - 1) / BM;
+  p.j_tiles = (p.K + BN - 1) / BN;
+  p.k_blocks = (T + BK - 1) / BK;
+  PEQA_TRY(status_word(&p.status));
+  CUtensorMap tmap_dy, tmap_x;
+  PEQA_TRY(make_tmap_bf16(&tmap_dy, dY, (uint64_t)p.N, (uint64_t)T, BK));
+  PEQA_TRY(make_tmap_bf16(&tmap_x, X, (uint64_t)p.K, (uint64_t)T, BK));
+  int sms = 0;
+  PEQA_TRY(sm_count(&sms));
+  const int tiles = p.i_tiles * p.j_tiles;
+  const int grid = tiles < sms ? tiles : sms;
+  if (w->bits == 4) {
+    PEQA_TRY(set_smem(ds_kernel<4>));
+    ds_kernel<4><<<grid, kDsThreads, SMEM_BYTES, st>>>(tmap_dy, tmap_x, p);
+  } else {
+    PEQA_TRY(set_smem(ds_kernel<3>));
+    ds_kernel<3><<<grid, kDsThreads, SMEM_BYTES, st>>>(tmap_dy, tmap_x, p);
+  }
+  PEQA_CUDA(cudaGetLastError());
+  if (!direct) {
+    const long long n_out = (long long)p.N * p.G;
+    const int ppg = g / p.piece;
+    const int blocks = (int)((n_out + 255) / 256);
+    ds_reduce_kernel<<<blocks, 256, 0, st>>>(p.out, dS, n_out, ppg);
+    PEQA_CUDA(cudaGetLastError());
+  }
+  return PEQA_OK;
+}
+
+}  // namespace peqa

@@ -1,0 +1,68 @@
+"""Host-side checks: the shared library builds, exports every declared symbol, and rejects
+bad arguments before touching the GPU."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2305_14152_b200 import binding, build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def L():
+    build.build()
+    return binding.lib()
+
+
+def _declared():
+    text = open(os.path.join(ROOT, "include", "peqa.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(peqa_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(L):
+    names = _declared()
+    assert "peqa_qlinear_fwd" in names and "peqa_scale_adamw" in names and len(names) >= 12
+    for n in names:
+        assert hasattr(L, n), n
+
+
+def test_version(L):
+    assert L.peqa_version() >= 100
+
+
+def test_argument_validation_needs_no_gpu(L):
+    buf = ctypes.create_string_buffer(4096)
+    p = ctypes.addressof(buf)
+    p16 = (p + 15) & ~15
+    assert L.peqa_quantize_rtn(0, 4, 64, 4, 0, p16, p16, p16, 0) == -1
+    assert L.peqa_quantize_rtn(p16, 4, 64, 5, 0, p16, p16, p16, 0) == -2
+    assert L.peqa_quantize_rtn(p16, 4, 48, 4, 0, p16, p16, p16, 0) == -3
+    assert L.peqa_quantize_rtn(p16, 4, 64, 4, 24, p16, p16, p16, 0) == -3
+    assert L.peqa_quantize_rtn(p16, 0, 64, 4, 0, p16, p16, p16, 0) == -3
+    assert L.peqa_quantize_rtn(p16 + 4, 4, 64, 4, 0, p16, p16, p16, 0) == -4
+    assert L.peqa_quantize_rtn(p16, 4, 1 << 17, 4, 0, p16, p16, p16, 0) == -9
+    assert L.peqa_pack(0, 1, 32, 4, p16, 0) == -1
+    assert L.peqa_unpack(p16, 1, 32, 2, p16, 0) == -2
+    assert L.peqa_scale_adamw(p16, p16, p16, 0, 4, 1e-3, 0.9, 0.999, 1e-8, 0.0, 1, 0) == -1
+    assert L.peqa_scale_adamw(p16, p16, p16, p16, 4, 1e-3, 0.9, 0.999, 1e-8, 0.0, 0, 0) == -3
+    w = binding._QWeight(4, 128, 256, 0, p16, p16, p16)
+    assert L.peqa_qlinear_fwd(ctypes.byref(w), 0, 8, p16, 0, 0, 0) == -1
+    assert L.peqa_qlinear_fwd(ctypes.byref(w), p16, 0, p16, 0, 0, 0) == -3
+    w2 = binding._QWeight(4, 128, 96, 0, p16, p16, p16)
+    assert L.peqa_qlinear_fwd(ctypes.byref(w2), p16, 8, p16, 0, 0, 0) == -3      # K % 64
+    w3 = binding._QWeight(4, 100, 256, 0, p16, p16, p16)
+    assert L.peqa_qlinear_fwd(ctypes.byref(w3), p16, 8, p16, 0, 0, 0) == -3      # N % 8
+    assert L.peqa_qlinear_decode(ctypes.byref(w), p16, 17, p16, 0, 0, 0) == -3
+    assert L.peqa_qlinear_bwd(ctypes.byref(w), p16, 0, 8, p16, 0, 0, 0, 0) == -1
+
+
+def test_workspace_query(L):
+    w = binding._QWeight(4, 4096, 4096, 0, 16, 16, 16)
+    assert L.peqa_workspace_bytes(binding.OP_BWD, 2048, ctypes.byref(w)) == 4096 * (4096 // 128) * 4
+    w = binding._QWeight(3, 4096, 4096, 128, 16, 16, 16)
+    assert L.peqa_workspace_bytes(binding.OP_BWD, 2048, ctypes.byref(w)) == 0
+    assert L.peqa_workspace_bytes(binding.OP_FWD, 2048, ctypes.byref(w)) == 0
