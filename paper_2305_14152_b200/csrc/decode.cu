@@ -1,8 +1,376 @@
-// placeholder until the decode kernel lands
+// Small-batch forward (token generation): Y[m,i] = sum_j X[m,j] * s[i,g(j)] * (Q[i,j] - z[i,g(j)])
+// for M <= 16 tokens.  The packed weights are streamed from HBM exactly once
+// with 128-bit loads; everything else is sized so that the stream is the bound.
+//
+// Work split: a CTA owns 128 weight rows and one slice of the K range; the
+// CTAs that share the same rows form a thread-block cluster along K and add
+// their partial sums through distributed shared memory in rank order, so the
+// result is deterministic and needs neither atomics nor a workspace.
+//
+// Inside a CTA each warp owns 32 rows.  The multiply-accumulate runs on the
+// warp-level tensor-core instruction mma.m16n8k16 with the *weights* as the
+// 16-row operand and the tokens as the 8-wide operand (M <= 8: one MMA per 16
+// rows; M <= 16: two).  Lane (g, c) = (lane/4, lane%4) streams 128 consecutive
+// codes of rows g and g+8 per step (48 B for 3-bit, 64 B for 4-bit), so the
+// four lanes of a row read one contiguous 192/256-byte run.  Codes become bf16
+// pairs (column k, column k+4) with one shift/funnel-shift, one logic op and
+// one bf16x2 subtract (see dequant.cuh); the contraction order inside an MMA is
+// free, so the activations are simply stored in shared memory in that same
+// pair order and no register permutation is needed.
+#include <cooperative_groups.h>
+#include <cuda_bf16.h>
+
 #include "common.cuh"
+#include "dequant.cuh"
+
+namespace cg = cooperative_groups;
+
 namespace peqa {
+
+namespace {
+
+constexpr int kDecWarps = 4;
+constexpr int kDecThreads = kDecWarps * 32;
+constexpr int kRowsPerWarp = 32;
+constexpr int kRowsPerCta = kDecWarps * kRowsPerWarp;   // 128
+constexpr int kStepCols = 512;                          // columns per warp step (4 lanes x 128)
+constexpr int kBlockBytes = 288;                        // 128 activations (256 B) + 32 B bank skew
+constexpr int kMaxSplit = 8;                            // portable cluster size
+
+struct DecodeParams {
+  const uint32_t* qw;
+  const uint8_t* zeros;
+  const float* scales;
+  const __nv_bfloat16* X;   // [M, K]
+  __nv_bfloat16* Y;         // [M, N]
+  int N, K, G, g, M;
+  int wpr;                  // packed words per row
+  int total_steps;          // ceil(K / 512)
+  int split;                // CTAs per cluster along K
+  int x_pitch;              // bytes between token rows of the staged activations
+};
+
+__device__ __forceinline__ void mma_16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0,
+                                          uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 "
+      "{%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+// 128 consecutive codes of one row: WORDS = 4 * BITS packed words.
+template <int BITS>
+struct RowChunk {
+  uint4 v[BITS];
+};
+
+template <int BITS>
+__device__ __forceinline__ RowChunk<BITS> load_chunk(const DecodeParams& p, int row, int col) {
+  RowChunk<BITS> r;
+  if (row < p.N && col < p.K) {
+    const uint4* src = reinterpret_cast<const uint4*>(p.qw + (size_t)row * p.wpr + (col >> 5) * BITS);
+#pragma unroll
+    for (int q = 0; q < BITS; ++q) r.v[q] = __ldg(src + q);
+  } else {
+#pragma unroll
+    for (int q = 0; q < BITS; ++q) r.v[q] = make_uint4(0u, 0u, 0u, 0u);
+  }
+  return r;
+}
+
+template <int BITS>
+__device__ __forceinline__ void unit_words(const RowChunk<BITS>& r, int u, uint32_t (&w)[BITS]) {
+  const uint32_t* flat = reinterpret_cast<const uint32_t*>(r.v);
+#pragma unroll
+  for (int q = 0; q < BITS; ++q) w[q] = flat[u * BITS + q];
+}
+
+// The two bf16x2 registers one lane contributes to one MMA for one weight row:
+// pairs (8*BLK + E, +4) and (8*BLK + E + 1, +4).
+template <int BITS, int BLK, int E, bool FOLD>
+__device__ __forceinline__ void two_pairs(const uint32_t (&w)[BITS], uint32_t zc, uint32_t s2,
+                                          uint32_t& p0, uint32_t& p1) {
+  p0 = dq::bf162_sub(dq::pair_raw<BITS, 8 * BLK + E>(w), zc);
+  p1 = dq::bf162_sub(dq::pair_raw<BITS, 8 * BLK + E + 1>(w), zc);
+  if (FOLD) {
+    p0 = dq::bf162_mul(p0, s2);
+    p1 = dq::bf162_mul(p1, s2);
+  }
+}
+
+template <int BITS, int NT, bool FOLD>
+__global__ void __launch_bounds__(kDecThreads)
+decode_kernel(const DecodeParams p) {
+  extern __shared__ __align__(16) uint8_t dec_smem[];
+  // layout: [staged activations: M rows of x_pitch bytes][partials: 128 rows x (8*NT) fp32]
+  const int rank = blockIdx.y;   // position along K inside the cluster
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g8 = lane >> 2, c4 = lane & 3;
+
+  const int steps_lo = (int)(((long long)p.total_steps * rank) / p.split);
+  const int steps_hi = (int)(((long long)p.total_steps * (rank + 1)) / p.split);
+  const int kbeg = steps_lo * kStepCols;
+  const int nsteps = steps_hi - steps_lo;
+
+  uint8_t* xs = dec_smem;
+  float* partial = reinterpret_cast<float*>(dec_smem + (((size_t)p.M * p.x_pitch + 15) & ~(size_t)15));
+
+  // ---- stage the activation slice: blocks of 8 columns stored as (0,4,1,5,2,6,3,7)
+  {
+    const int blocks8 = nsteps * (kStepCols / 8);
+    for (int idx = threadIdx.x; idx < p.M * blocks8; idx += kDecThreads) {
+      const int m = idx / blocks8;
+      const int b8 = idx - m * blocks8;
+      const int col = kbeg + b8 * 8;
+      uint4 v = make_uint4(0u, 0u, 0u, 0u);
+      if (col < p.K) v = __ldg(reinterpret_cast<const uint4*>(p.X + (size_t)m * p.K + col));
+      const int lcol = b8 * 8;
+      uint8_t* dst = xs + (size_t)m * p.x_pitch + (lcol >> 7) * kBlockBytes + (lcol & 127) * 2;
+      *reinterpret_cast<uint2*>(dst) =
+          make_uint2(dq::prmt(v.x, v.z, 0x5410u), dq::prmt(v.x, v.z, 0x7632u));
+      *reinterpret_cast<uint2*>(dst + 8) =
+          make_uint2(dq::prmt(v.y, v.w, 0x5410u), dq::prmt(v.y, v.w, 0x7632u));
+    }
+  }
+  __syncthreads();
+
+  const int row_base = blockIdx.x * kRowsPerCta + warp * kRowsPerWarp;
+  // rows of this lane: fragment rows g and g+8 of the two 16-row blocks
+  int rows[4] = {row_base + g8, row_base + g8 + 8, row_base + 16 + g8, row_base + 24 + g8};
+
+  float acc[2][NT][4];
+#pragma unroll
+  for (int rb = 0; rb < 2; ++rb)
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) acc[rb][nt][e] = 0.0f;
+
+  uint32_t zc_row[4] = {0u, 0u, 0u, 0u};
+  if (!FOLD) {
+#pragma unroll
+    for (int r = 0; r < 4; ++r)
+      if (rows[r] < p.N) zc_row[r] = dq::zero_const<BITS>(__ldg(p.zeros + rows[r]));
+      else zc_row[r] = dq::zero_const<BITS>(0u);
+  }
+
+  // token rows this lane reads as the MMA "B" operand (token index = lane / 4);
+  // lanes beyond M read row 0: their accumulator columns are never stored.
+  const uint8_t* xrow0 = xs + (size_t)(g8 < p.M ? g8 : 0) * p.x_pitch;
+  const uint8_t* xrow1 = xs + (size_t)(g8 + 8 < p.M ? g8 + 8 : 0) * p.x_pitch;
+
+  RowChunk<BITS> cur[4], nxt[4];
+  if (nsteps > 0) {
+#pragma unroll
+    for (int r = 0; r < 4; ++r) cur[r] = load_chunk<BITS>(p, rows[r], kbeg + c4 * 128);
+  }
+  for (int st = 0; st < nsteps; ++st) {
+    const int col0 = kbeg + st * kStepCols + c4 * 128;   // first column of this lane's chunk
+    if (st + 1 < nsteps) {
+#pragma unroll
+      for (int r = 0; r < 4; ++r) nxt[r] = load_chunk<BITS>(p, rows[r], col0 + kStepCols);
+    }
+    const int xoff = (st * 4 + c4) * kBlockBytes;
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      uint32_t w[4][BITS];
+      uint32_t zc[4], s2[4];
+#pragma unroll
+      for (int r = 0; r < 4; ++r) {
+        unit_words<BITS>(cur[r], u, w[r]);
+        if (FOLD) {
+          const int col = col0 + u * 32;
+          uint32_t z = 0u;
+          float s = 0.0f;
+          if (rows[r] < p.N && col < p.K) {
+            const size_t gi = (size_t)rows[r] * p.G + col / p.g;
+            z = __ldg(p.zeros + gi);
+            s = __ldg(p.scales + gi);
+          }
+          zc[r] = dq::zero_const<BITS>(z);
+          s2[r] = dq::bf162_broadcast(s);
+        } else {
+          zc[r] = zc_row[r];
+          s2[r] = 0u;
+        }
+      }
+#pragma unroll
+      for (int blk = 0; blk < 4; ++blk) {
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) {
+          // activations of pairs (2*hh, 2*hh+1) of this 8-column block
+          const int xo = xoff + u * 64 + blk * 16 + hh * 8;
+          const uint2 b0 = *reinterpret_cast<const uint2*>(xrow0 + xo);
+          uint2 b1 = make_uint2(0u, 0u);
+          if (NT == 2) b1 = *reinterpret_cast<const uint2*>(xrow1 + xo);
+#pragma unroll
+          for (int rb = 0; rb < 2; ++rb) {
+            uint32_t a[4];
+            if (hh == 0) {
+              if (blk == 0) { two_pairs<BITS, 0, 0, FOLD>(w[2 * rb], zc[2 * rb], s2[2 * rb], a[0], a[2]);
+                              two_pairs<BITS, 0, 0, FOLD>(w[2 * rb + 1], zc[2 * rb + 1], s2[2 * rb + 1], a[1], a[3]); }
+              if (blk == 1) { two_pairs<BITS, 1, 0, FOLD>(w[2 * rb], zc[2 * rb], s2[2 * rb], a[0], a[2]);
+                              two_pairs<BITS, 1, 0, FOLD>(w[2 * rb + 1], zc[2 * rb + 1], s2[2 * rb + 1], a[1], a[3]); }
+              if (blk == 2) { two_pairs<BITS, 2, 0, FOLD>(w[2 * rb], zc[2 * rb], s2[2 * rb], a[0], a[2]);
+                              two_pairs<BITS, 2, 0, FOLD>(w[2 * rb + 1], zc[2 * rb + 1], s2[2 * rb + 1], a[1], a[3]); }
+              if (blk == 3) { two_pairs<BITS, 3, 0, FOLD>(w[2 * rb], zc[2 * rb], s2[2 * rb], a[0], a[2]);
+                              two_pairs<BITS, 3, 0, FOLD>(w[2 * rb + 1], zc[2 * rb + 1], s2[2 * rb + 1], a[1], a[3]); }
+            } else {
+              if (blk == 0) { two_pairs<BITS, 0, 2, FOLD>(w[2 * rb], zc[2 * rb], s2[2 * rb], a[0], a[2]);
+                              two_pairs<BITS, 0, 2, FOLD>(w[2 * rb + 1], zc[2 * rb + 1], s2[2 * rb + 1], a[1], a[3]); }
+              if (blk == 1) { two_pairs<BITS, 1, 2, FOLD>(w[2 * rb], zc[2 * rb], s2[2 * rb], a[0], a[2]);
+                              two_pairs<BITS, 1, 2, FOLD>(w[2 * rb + 1], zc[2 * rb + 1], s2[2 * rb + 1], a[1], a[3]); }
+              if (blk == 2) { two_pairs<BITS, 2, 2, FOLD>(w[2 * rb], zc[2 * rb], s2[2 * rb], a[0], a[2]);
+                              two_pairs<BITS, 2, 2, FOLD>(w[2 * rb + 1], zc[2 * rb + 1], s2[2 * rb + 1], a[1], a[3]); }
+              if (blk == 3) { two_pairs<BITS, 3, 2, FOLD>(w[2 * rb], zc[2 * rb], s2[2 * rb], a[0], a[2]);
+                              two_pairs<BITS, 3, 2, FOLD>(w[2 * rb + 1], zc[2 * rb + 1], s2[2 * rb + 1], a[1], a[3]); }
+            }
+            mma_16816(acc[rb][0], a, b0.x, b0.y);
+            if (NT == 2) mma_16816(acc[rb][1], a, b1.x, b1.y);
+          }
+        }
+      }
+    }
+    if (st + 1 < nsteps) {
+#pragma unroll
+      for (int r = 0; r < 4; ++r) cur[r] = nxt[r];
+    }
+  }
+
+  // ---- partial sums of this CTA: [128 rows][8*NT tokens]
+  constexpr int TOK = 8 * NT;
+#pragma unroll
+  for (int rb = 0; rb < 2; ++rb)
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+      const int lr = warp * kRowsPerWarp + rb * 16 + g8;
+      const int tk = nt * 8 + c4 * 2;
+      partial[lr * TOK + tk] = acc[rb][nt][0];
+      partial[lr * TOK + tk + 1] = acc[rb][nt][1];
+      partial[(lr + 8) * TOK + tk] = acc[rb][nt][2];
+      partial[(lr + 8) * TOK + tk + 1] = acc[rb][nt][3];
+    }
+
+  // ---- add the K-slices of the cluster in rank order and write Y
+  const int rows_per_rank = kRowsPerCta / p.split;
+  if (p.split > 1) {
+    cg::cluster_group cluster = cg::this_cluster();
+    cluster.sync();
+    for (int idx = threadIdx.x; idx < rows_per_rank * p.M; idx += kDecThreads) {
+      const int m = idx / rows_per_rank;
+      const int lr = rank * rows_per_rank + (idx - m * rows_per_rank);
+      const int row = blockIdx.x * kRowsPerCta + lr;
+      float sum = 0.0f;
+      for (int r = 0; r < p.split; ++r) {
+        const float* remote = cluster.map_shared_rank(partial, r);
+        sum += remote[lr * TOK + m];
+      }
+      if (row < p.N) {
+        if (!FOLD) sum *= __ldg(p.scales + row);
+        p.Y[(size_t)m * p.N + row] = __float2bfloat16_rn(sum);
+      }
+    }
+    cluster.sync();   // keep every CTA's shared memory alive until all ranks have read it
+  } else {
+    __syncthreads();
+    for (int idx = threadIdx.x; idx < kRowsPerCta * p.M; idx += kDecThreads) {
+      const int m = idx / kRowsPerCta;
+      const int lr = idx - m * kRowsPerCta;
+      const int row = blockIdx.x * kRowsPerCta + lr;
+      if (row < p.N) {
+        float sum = partial[lr * TOK + m];
+        if (!FOLD) sum *= __ldg(p.scales + row);
+        p.Y[(size_t)m * p.N + row] = __float2bfloat16_rn(sum);
+      }
+    }
+  }
+}
+
+int sm_count_cached(int* n) {
+  static thread_local int cached_dev = -1, cached_n = 0;
+  int dev = 0;
+  PEQA_CUDA(cudaGetDevice(&dev));
+  if (dev != cached_dev) {
+    PEQA_CUDA(cudaDeviceGetAttribute(&cached_n, cudaDevAttrMultiProcessorCount, dev));
+    cached_dev = dev;
+  }
+  *n = cached_n;
+  return PEQA_OK;
+}
+
+template <int BITS, int NT, bool FOLD>
+int launch_decode_t(const DecodeParams& p, int row_blocks, size_t smem, cudaStream_t st) {
+  auto kern = decode_kernel<BITS, NT, FOLD>;
+  PEQA_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(row_blocks, p.split, 1);
+  cfg.blockDim = dim3(kDecThreads, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 1;
+  attr[0].val.clusterDim.y = p.split;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  PEQA_CUDA(cudaLaunchKernelEx(&cfg, kern, p));
+  return PEQA_OK;
+}
+
+}  // namespace
+
 size_t decode_workspace_bytes(const peqa_qweight_t*, int, int) { return 0; }
-int launch_decode(const peqa_qweight_t*, int, const void*, int, void*, void*, size_t, cudaStream_t) {
-  return PEQA_ERR_BAD_SHAPE;
+
+int launch_decode(const peqa_qweight_t* w, int g, const void* X, int M, void* Y,
+                  void* workspace, size_t workspace_bytes, cudaStream_t st) {
+  (void)workspace; (void)workspace_bytes;
+  DecodeParams p;
+  p.qw = w->qweight;
+  p.zeros = w->zeros;
+  p.scales = w->scales;
+  p.X = static_cast<const __nv_bfloat16*>(X);
+  p.Y = static_cast<__nv_bfloat16*>(Y);
+  p.N = w->out_features;
+  p.K = w->in_features;
+  p.g = g;
+  p.G = p.K / g;
+  p.M = M;
+  p.wpr = p.K * w->bits / 32;
+  p.total_steps = (p.K + kStepCols - 1) / kStepCols;
+
+  int sms = 0;
+  PEQA_TRY(sm_count_cached(&sms));
+  const int row_blocks = (p.N + kRowsPerCta - 1) / kRowsPerCta;
+  // Enough CTAs for about three waves of the machine, split a power of two <= 8.
+  int split = 1;
+  while (split < kMaxSplit && row_blocks * split < 3 * sms && split * 2 <= p.total_steps) split *= 2;
+  const int NT = M <= 8 ? 1 : 2;
+  size_t smem = 0;
+  for (;;) {
+    p.split = split;
+    const int max_steps = (p.total_steps + split - 1) / split;
+    const int nblk = max_steps * (kStepCols / 128);
+    // pitch = nblk*288 + pad with pitch % 128 == 8: consecutive tokens land 2 banks apart
+    const int pad = ((8 - (nblk * kBlockBytes) % 128) % 128 + 128) % 128;
+    p.x_pitch = nblk * kBlockBytes + pad;
+    smem = (((size_t)M * p.x_pitch + 15) & ~(size_t)15) + (size_t)kRowsPerCta * 8 * NT * sizeof(float);
+    if (smem <= 200 * 1024 || split == kMaxSplit) break;
+    split *= 2;
+  }
+  if (smem > 227 * 1024) return PEQA_ERR_TOO_LARGE;
+  const bool fold = p.G > 1;
+  if (w->bits == 4) {
+    if (NT == 1) return fold ? launch_decode_t<4, 1, true>(p, row_blocks, smem, st)
+                             : launch_decode_t<4, 1, false>(p, row_blocks, smem, st);
+    return fold ? launch_decode_t<4, 2, true>(p, row_blocks, smem, st)
+                : launch_decode_t<4, 2, false>(p, row_blocks, smem, st);
+  }
+  if (NT == 1) return fold ? launch_decode_t<3, 1, true>(p, row_blocks, smem, st)
+                           : launch_decode_t<3, 1, false>(p, row_blocks, smem, st);
+  return fold ? launch_decode_t<3, 2, true>(p, row_blocks, smem, st)
+              : launch_decode_t<3, 2, false>(p, row_blocks, smem, st);
 }
-}
+
+}  // namespace peqa

@@ -132,17 +132,18 @@ __global__ void unpack_kernel(const uint32_t* __restrict__ qweight, long long to
 }
 
 // Elementwise AdamW in binary32.  The bias corrections 1-b^t are formed on the
-// host in double and passed in as reciprocals.
+// host in double and passed in as reciprocals, as are 1-b1 and 1-b2 (the
+// arguments are the binary32 values of lr, b1, b2, eps the caller passed).
 __global__ void adamw_kernel(float* __restrict__ s, const float* __restrict__ grad,
                              float* __restrict__ m, float* __restrict__ v, long long n,
-                             float lr, float b1, float b2, float eps, float decay,
-                             float inv_c1, float inv_c2) {
+                             float lr, float b1, float b2, float omb1, float omb2, float eps,
+                             float decay, float inv_c1, float inv_c2) {
   long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   const long long stride = (long long)gridDim.x * blockDim.x;
   for (; i < n; i += stride) {
     const float gr = grad[i];
-    const float mn = b1 * m[i] + (1.0f - b1) * gr;
-    const float vn = b2 * v[i] + (1.0f - b2) * gr * gr;
+    const float mn = b1 * m[i] + omb1 * gr;
+    const float vn = b2 * v[i] + omb2 * gr * gr;
     const float denom = sqrtf(vn * inv_c2) + eps;
     s[i] = s[i] * decay - lr * (mn * inv_c1) / denom;
     m[i] = mn;
@@ -221,8 +222,9 @@ extern "C" int peqa_scale_adamw(float* scales, const float* dS, float* m, float*
   const float decay = (float)(1.0 - (double)lr * (double)weight_decay);
   const int grid = grid_for(numel, 256);
   adamw_kernel<<<grid, 256, 0, as_stream(stream)>>>(scales, dS, m, v, (long long)numel, lr, beta1,
-                                                   beta2, eps, decay, (float)(1.0 / c1),
-                                                   (float)(1.0 / c2));
+                                                   beta2, (float)(1.0 - (double)beta1),
+                                                   (float)(1.0 - (double)beta2), eps, decay,
+                                                   (float)(1.0 / c1), (float)(1.0 / c2));
   PEQA_CUDA(cudaGetLastError());
   return PEQA_OK;
 }

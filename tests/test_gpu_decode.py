@@ -1,0 +1,60 @@
+"""GPU parity: the small-batch decode path (Sec. 3.1/3.3 matrix-vector regime) against the oracle."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2305_14152_b200 import binding, synth
+from gpu_util import assert_close, bf16_to_dev, dev_to_f64, oracle_layer, to_qweight
+
+pytestmark = pytest.mark.gpu
+
+
+def _check(d, bits, g, M, also_fwd=False):
+    codes, zeros, scales, packed = oracle_layer(d, bits, g)
+    K = d["W"].shape[1]
+    qw = to_qweight(packed, zeros, scales, bits, g, K)
+    Xb = d["X"][:M]
+    X = bf16_to_dev(Xb)
+    Y = binding.qlinear_decode(qw, X)
+    torch.cuda.synchronize()
+    ref = oracle.fwd(Xb, packed, zeros, scales, bits, g)
+    assert_close(dev_to_f64(Y), ref, f"decode M={M}")
+    if also_fwd:
+        Y2 = binding.qlinear_fwd(qw, X)
+        binding.check_status()
+        assert_close(dev_to_f64(Y), dev_to_f64(Y2), "decode vs fwd kernel")
+
+
+@pytest.mark.parametrize("M", [1, 2, 4, 8, 9, 16])
+@pytest.mark.parametrize("bits,g", [(3, 0), (4, 0), (3, 128), (4, 64), (3, 32)])
+def test_small_shapes(M, bits, g):
+    # N=200: ragged 128-row block; K=1408 = 2.75 steps of 512 columns
+    d = synth.custom(7 * M + bits + g, 200, 1408, 16, bits, g, outliers=True)
+    _check(d, bits, g, M, also_fwd=(M in (1, 16)))
+
+
+def test_single_step_and_tiny_rows():
+    d = synth.custom(2, 8, 128, 16, 3, 0)
+    _check(d, 3, 0, 1)
+    _check(d, 3, 0, 16)
+
+
+@pytest.mark.parametrize("M", [1, 4, 16])
+def test_c4_llama65b_shapes(M):
+    """BASELINE config 4 at full size: 3-bit per-channel, three layer shapes."""
+    for d in synth.generate("c4"):
+        _check(d, 3, 0, M)
+
+
+def test_unit_scale_integer_inputs_are_exact():
+    rng = np.random.default_rng(0)
+    N, K, M = 256, 1024, 5
+    codes = rng.integers(0, 8, size=(N, K), dtype=np.uint8)
+    packed = oracle.pack(codes, 3)
+    qw = to_qweight(packed, np.zeros((N, 1), np.uint8), np.ones((N, 1), np.float32), 3, 0, K)
+    Xi = rng.integers(-4, 5, size=(M, K))
+    Y = binding.qlinear_decode(qw, bf16_to_dev(synth.f32_to_bf16_bits(Xi.astype(np.float32))))
+    ref = (Xi @ codes.astype(np.int64).T).astype(np.float32)
+    exp = synth.bf16_bits_to_f32(synth.f32_to_bf16_bits(ref)).astype(np.float64)
+    assert np.array_equal(dev_to_f64(Y), exp)
