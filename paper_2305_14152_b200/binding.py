@@ -118,17 +118,21 @@ def version() -> int:
     return lib().peqa_version()
 
 
-def quantize_rtn(W: torch.Tensor, bits: int, group_size: int = 0) -> QWeight:
+def quantize_rtn(W: torch.Tensor, bits: int, group_size: int = 0, out: QWeight | None = None) -> QWeight:
+    """Quantize W; with ``out`` the results are written into its existing tensors."""
     _dev(W, torch.float32, "W")
     N, K = W.shape
-    G = 1 if group_size in (0, K) else max(K // max(group_size, 1), 1)
-    words = max(K * bits // 32, 1)
-    q = torch.empty((N, words), dtype=torch.int32, device=W.device)
-    z = torch.empty((N, G), dtype=torch.uint8, device=W.device)
-    s = torch.empty((N, G), dtype=torch.float32, device=W.device)
+    if out is not None:
+        q, z, s = out.qweight, out.zeros, out.scales
+    else:
+        G = 1 if group_size in (0, K) else max(K // max(group_size, 1), 1)
+        words = max(K * bits // 32, 1)
+        q = torch.empty((N, words), dtype=torch.int32, device=W.device)
+        z = torch.empty((N, G), dtype=torch.uint8, device=W.device)
+        s = torch.empty((N, G), dtype=torch.float32, device=W.device)
     _check(lib().peqa_quantize_rtn(W.data_ptr(), N, K, bits, group_size, q.data_ptr(), z.data_ptr(),
                                    s.data_ptr(), _stream()), "peqa_quantize_rtn")
-    return QWeight(bits, N, K, group_size, q, z, s)
+    return out if out is not None else QWeight(bits, N, K, group_size, q, z, s)
 
 
 def pack(codes: torch.Tensor, bits: int) -> torch.Tensor:
