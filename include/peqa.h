@@ -165,6 +165,30 @@ int peqa_train_step_host(const peqa_qweight_t* w, int T,
                          float lr, float beta1, float beta2, float eps, float weight_decay,
                          int64_t step, void* workspace, size_t workspace_bytes, void* stream);
 
+/*
+ * Scale gradient dS alone, for callers that cannot allocate device memory and
+ * therefore cannot hand peqa_qlinear_bwd a workspace: code that runs where
+ * cudaMalloc is off limits, or that is given nothing but its input and output
+ * buffers.  (The paper has no counterpart to this call; it is the dS half of
+ * peqa_qlinear_bwd with the scratch moved inside the library.)
+ *   X in bf16 [T, K];  dY in bf16 [T, N];  dS out fp32 [N, G], overwritten.
+ * The partial sums go to a fixed 8 MiB array that is part of the library's
+ * device image (each GPU that loads the library holds it until the process
+ * ends); peqa_bwd_ds_static_capacity_bytes() returns that size.  A layer
+ * whose peqa_workspace_bytes(PEQA_OP_BWD, T, w) exceeds it is refused with
+ * PEQA_ERR_TOO_LARGE and nothing is enqueued.  The call performs no
+ * allocation of any kind.  The first call on each device looks the array's
+ * device address up (with that device current) and caches it; make that
+ * first call outside any stream capture.  All calls on a device share the one
+ * array: it keeps whatever the previous call left, every value that is read
+ * is rewritten first, and two calls whose kernels may overlap on the GPU
+ * (different streams) race on it -- serialise them.  Same shape rules and
+ * return codes as peqa_qlinear_bwd.
+ */
+int peqa_qlinear_bwd_ds_static(const peqa_qweight_t* w, const void* X_bf16, const void* dY_bf16,
+                               int T, float* dS, void* stream);
+size_t peqa_bwd_ds_static_capacity_bytes(void);
+
 /* Synchronises `stream`, reads and clears the device status word.  Returns
  * PEQA_OK, PEQA_ERR_DEVICE_TIMEOUT, or PEQA_ERR_CUDA. */
 int peqa_check_status(void* stream);

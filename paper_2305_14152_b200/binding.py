@@ -67,6 +67,9 @@ def lib() -> ctypes.CDLL:
         L.peqa_scale_adamw.argtypes = [vp, vp, vp, vp, i64, f32, f32, f32, f32, f32, i64, vp]
         L.peqa_train_step_host.argtypes = [qp, i32] + [vp] * 12 + [f32] * 5 + [i64, vp, sz, vp]
         L.peqa_check_status.argtypes = [vp]
+        L.peqa_qlinear_bwd_ds_static.argtypes = [qp, vp, vp, i32, vp, vp]
+        L.peqa_qlinear_bwd_ds_static.restype = ctypes.c_int
+        L.peqa_bwd_ds_static_capacity_bytes.restype = sz
         for name in ("peqa_quantize_rtn", "peqa_pack", "peqa_unpack", "peqa_qlinear_fwd",
                      "peqa_qlinear_bwd", "peqa_qlinear_decode", "peqa_scale_adamw",
                      "peqa_train_step_host", "peqa_check_status"):
@@ -232,6 +235,23 @@ def train_step_host(w: QWeight, h_X, h_dY, h_Y, h_dX, h_dS, d_X, d_dY, d_Y, d_dX
         h_dS.data_ptr(), d_X.data_ptr(), d_dY.data_ptr(), d_Y.data_ptr(), d_dX.data_ptr(),
         d_dS.data_ptr(), d_m.data_ptr(), d_v.data_ptr(), lr, beta1, beta2, eps, weight_decay, step,
         wp, wb, _stream()), "peqa_train_step_host")
+
+
+def qlinear_bwd_ds_static(w: QWeight, X: torch.Tensor, dY: torch.Tensor, dS: torch.Tensor):
+    """dS through the library's built-in scratch array; the caller supplies only inputs and
+    the output tensor, and nothing is allocated on the way."""
+    _dev(X, torch.bfloat16, "X")
+    _dev(dY, torch.bfloat16, "dY")
+    _dev(dS, torch.float32, "dS")
+    cs = w.c_struct()
+    _check(lib().peqa_qlinear_bwd_ds_static(ctypes.byref(cs), X.data_ptr(), dY.data_ptr(),
+                                            dY.shape[0], dS.data_ptr(), _stream()),
+           "peqa_qlinear_bwd_ds_static")
+    return dS
+
+
+def bwd_ds_static_capacity_bytes() -> int:
+    return int(lib().peqa_bwd_ds_static_capacity_bytes())
 
 
 def check_status() -> None:
