@@ -258,6 +258,56 @@ def run_cuda(args):
     value = world * flop_step / (ms_step * 1e-3) / 1e12
 
     # ---- end to end through the host-buffer entry point (pinned host memory both ways)
+    e2e = None
+    if not args.only_step:
+        e2e = bench_e2e(args, binding, torch, qws, Xs, dYs, Y, dX, dS, m, v, ws, lr, dist, dev,
+                        world, flop_step, T, N, K, G)
+
+    # ---- roofline of the dominant kernel (the slowest of the three contractions)
+    gemm = {k: stage_ms[k] for k in (1, 2, 3)}
+    dom = max(gemm, key=gemm.get)
+    ach = 2.0 * T * N * K / (gemm[dom] * 1e-3) / 1e12
+    long_region = ms_total > 1000.0
+    peak = peaks["bf16_tflops_sustained"] if long_region else peaks["bf16_tflops"]
+    roofline = {"bound": "tensor", "kernel": stage_names[dom], "achieved": ach, "peak": peak,
+                "unit": "TFLOP/s", "frac": ach / peak, "traffic": None,
+                "peak_source": f"{peak_src} bf16 {'sustained' if long_region else 'burst'}",
+                "frac_of_nominal_2250": ach / 2250.0,
+                "per_kernel_tflops": {stage_names[k]: 2.0 * T * N * K / (gemm[k] * 1e-3) / 1e12
+                                      for k in (1, 2, 3)}}
+
+    # ---- secondary metric: M=1 decode of the LLaMA-65B 3-bit per-channel shapes, cold in L2
+    decode = None
+    if rank == 0 and not args.only_step:
+        decode = bench_decode(binding, dev, peaks)
+
+    out = {
+        "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"{WORKLOAD}: LLaMA-7B attention projection N=K=4096, 3-bit, group 128, "
+                               f"T=2048 tokens; step = quantize+pack, fwd, dX, dS, AdamW, decode(M=1)",
+                   "l2": f"{N_SETS} rotating input sets (~{N_SETS * 135} MB) exceed the 126 MB L2; no flush kernel",
+                   "parallelism": "replicas only" if world > 1 else "single GPU",
+                   "flop_per_step": flop_step},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
+        "stage_ms": dict(zip(stage_names, stage_ms)),
+        "roofline": roofline, "decode": decode,
+    }
+    if rank == 0 and world == 1 and not args.only_step:
+        dt, fl, what = oracle_sample(spec, sets[0])
+        import oracle
+        out["cpu_baseline"] = {"value": fl / dt / 1e12, "unit": "TFLOP/s", "cores": oracle.num_threads(),
+                               "kind": "oracle", "sample": what, "seconds": dt}
+    if rank == 0:
+        print(json.dumps(out), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def bench_e2e(args, binding, torch, qws, Xs, dYs, Y, dX, dS, m, v, ws, lr, dist, dev, world,
+              flop_step, T, N, K, G):
+    """Same metric through peqa_train_step_host: pinned host buffers in and out every step."""
     hX = torch.empty((T, K), dtype=torch.bfloat16).pin_memory()
     hdY = torch.empty((T, N), dtype=torch.bfloat16).pin_memory()
     hX.copy_(Xs[0].cpu())
@@ -281,52 +331,11 @@ def run_cuda(args):
     e1.record()
     torch.cuda.synchronize()
     e2e_ms = aggregate_max(e0.elapsed_time(e1) / e2e_steps, dist, dev)
-    e2e = {"value": world * flop_step / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
-           "h2d_bytes_per_step": int(hX.numel() * 2 + hdY.numel() * 2),
-           "d2h_bytes_per_step": int(hY.numel() * 2 + hdX.numel() * 2 + hdS.numel() * 4),
-           "ms_per_step": e2e_ms,
-           "what": "peqa_train_step_host: H2D X,dY; fwd, dX, dS, AdamW; D2H Y,dX,dS"}
-
-    # ---- roofline of the dominant kernel (the slowest of the three contractions)
-    gemm = {k: stage_ms[k] for k in (1, 2, 3)}
-    dom = max(gemm, key=gemm.get)
-    ach = 2.0 * T * N * K / (gemm[dom] * 1e-3) / 1e12
-    long_region = ms_total > 1000.0
-    peak = peaks["bf16_tflops_sustained"] if long_region else peaks["bf16_tflops"]
-    roofline = {"bound": "tensor", "kernel": stage_names[dom], "achieved": ach, "peak": peak,
-                "unit": "TFLOP/s", "frac": ach / peak, "traffic": None,
-                "peak_source": f"{peak_src} bf16 {'sustained' if long_region else 'burst'}",
-                "frac_of_nominal_2250": ach / 2250.0,
-                "per_kernel_tflops": {stage_names[k]: 2.0 * T * N * K / (gemm[k] * 1e-3) / 1e12
-                                      for k in (1, 2, 3)}}
-
-    # ---- secondary metric: M=1 decode of the LLaMA-65B 3-bit per-channel shapes, cold in L2
-    decode = None
-    if rank == 0:
-        decode = bench_decode(binding, dev, peaks)
-
-    out = {
-        "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
-        "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": f"{WORKLOAD}: LLaMA-7B attention projection N=K=4096, 3-bit, group 128, "
-                               f"T=2048 tokens; step = quantize+pack, fwd, dX, dS, AdamW, decode(M=1)",
-                   "l2": f"{N_SETS} rotating input sets (~{N_SETS * 135} MB) exceed the 126 MB L2; no flush kernel",
-                   "parallelism": "replicas only" if world > 1 else "single GPU",
-                   "flop_per_step": flop_step},
-        "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
-        "stage_ms": dict(zip(stage_names, stage_ms)),
-        "roofline": roofline, "decode": decode,
-    }
-    if rank == 0 and world == 1:
-        dt, fl, what = oracle_sample(spec, sets[0])
-        import oracle
-        out["cpu_baseline"] = {"value": fl / dt / 1e12, "unit": "TFLOP/s", "cores": oracle.num_threads(),
-                               "kind": "oracle", "sample": what, "seconds": dt}
-    if rank == 0:
-        print(json.dumps(out), flush=True)
-    if dist is not None:
-        dist.destroy_process_group()
+    return {"value": world * flop_step / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
+            "h2d_bytes_per_step": int(hX.numel() * 2 + hdY.numel() * 2),
+            "d2h_bytes_per_step": int(hY.numel() * 2 + hdX.numel() * 2 + hdS.numel() * 4),
+            "ms_per_step": e2e_ms,
+            "what": "peqa_train_step_host: H2D X,dY; fwd, dX, dS, AdamW; D2H Y,dX,dS"}
 
 
 def bench_decode(binding, dev, peaks, reps=30):
@@ -373,6 +382,9 @@ def main():
     ap.add_argument("--steps", type=int, default=500)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--only-step", action="store_true",
+                    help="time the step only: skip the e2e, decode and CPU-baseline sections "
+                         "(lean runs under a profiler)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

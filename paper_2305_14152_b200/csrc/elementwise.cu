@@ -41,10 +41,46 @@ __device__ __forceinline__ uint32_t warp_unpack(const uint32_t* src, int lane) {
   return v & ((1u << BITS) - 1u);
 }
 
-// One CTA per output row.  Pass 1: per 32-column chunk min/max.  Pass 2: per
-// group (s, z) in strict binary32 (division and rounding as single IEEE
-// operations, no FMA).  Pass 3: codes, packed with the warp OR-reduction.
-// The row is read twice; the second read is served by L2.
+// Eight consecutive lanes hold 4 codes each (one 32-column chunk).  Builds the
+// chunk's BITS packed words; lane l8 < BITS of the group returns word l8.
+template <int BITS>
+__device__ __forceinline__ uint32_t group8_pack(uint32_t piece, int lane) {
+  constexpr int NB = 4 * BITS;                 // bits per lane piece: 12 or 16
+  const int l8 = lane & 7;
+  const int base = lane & ~7;
+  const int wbit = 32 * (l8 < BITS ? l8 : 0);  // first bit of the word this lane assembles
+  const int first = wbit / NB;                 // first piece overlapping that word
+  uint32_t word = 0u;
+#pragma unroll
+  for (int k = 0; k < (BITS == 3 ? 4 : 2); ++k) {
+    const int src = first + k;
+    const uint32_t pc = __shfl_sync(0xffffffffu, piece, base + (src & 7));
+    const int sh = src * NB - wbit;            // position of that piece relative to the word
+    if (src < 8) {
+      if (sh >= 0) { if (sh < 32) word |= pc << sh; }
+      else word |= pc >> (-sh);
+    }
+  }
+  return word;
+}
+
+// rint(fl(w / s)) with fl() the correctly rounded binary32 quotient.  The product
+// w * (1/s) is within a few ulps of that quotient, so both round to the same
+// integer unless the product sits within a few ulps of a half-integer; only then
+// (or when the product is huge or not finite) is the IEEE division carried out.
+__device__ __forceinline__ float rint_of_quotient(float w, float s, float rs) {
+  const float t = __fmul_rn(w, rs);
+  float k = rintf(t);
+  const float dist = fabsf(__fsub_rn(fabsf(__fsub_rn(t, k)), 0.5f));
+  if (!(fabsf(t) <= 4.0e6f) || dist <= __fmul_rn(fabsf(t), 2.0e-6f)) k = rintf(__fdiv_rn(w, s));
+  return k;
+}
+
+// One CTA per output row; a thread works on float4 vectors so that all loads of
+// a pass are in flight together.  Pass 1: min/max per 32-column chunk (8 lanes).
+// Pass 2: per group (s, z) in strict binary32 (division and rounding as single
+// IEEE operations, no FMA).  Pass 3: codes (second read of the row, served by
+// L2), packed by exchanging 4-code pieces inside each 8-lane group.
 template <int BITS>
 __global__ void __launch_bounds__(kQuantThreads)
 quantize_rtn_kernel(const float* __restrict__ W, int K, int g,
@@ -58,20 +94,35 @@ quantize_rtn_kernel(const float* __restrict__ W, int K, int g,
   const int row = blockIdx.x;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int chunks = K >> 5;
+  const int nvec = K >> 2;
   const int G = K / g;
   const int cpg = g >> 5;  // chunks per group
-  const float* w = W + (size_t)row * K;
+  const float4* w4 = reinterpret_cast<const float4*>(W + (size_t)row * K);
   const float qmax = (float)((1 << BITS) - 1);
+  constexpr int UNROLL = 4;
 
-  for (int c = warp; c < chunks; c += kQuantWarps) {
-    float v = w[c * 32 + lane];
-    float mn = v, mx = v;
+  // Every thread runs the same number of iterations (the shuffles below name the
+  // whole warp); vectors past the end of the row are predicated off.
+  for (int vb = 0; vb < nvec; vb += kQuantThreads * UNROLL) {
+    const int v0 = vb + threadIdx.x;
+    float4 x[UNROLL];
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
-      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    for (int u = 0; u < UNROLL; ++u) {
+      const int v = v0 + u * kQuantThreads;
+      x[u] = v < nvec ? __ldg(w4 + v) : make_float4(0.f, 0.f, 0.f, 0.f);
     }
-    if (lane == 0) { cmin[c] = mn; cmax[c] = mx; }
+#pragma unroll
+    for (int u = 0; u < UNROLL; ++u) {
+      const int v = v0 + u * kQuantThreads;   // nvec is a multiple of 8: a group of 8 lanes is all-in or all-out
+      float mn = fminf(fminf(x[u].x, x[u].y), fminf(x[u].z, x[u].w));
+      float mx = fmaxf(fmaxf(x[u].x, x[u].y), fmaxf(x[u].z, x[u].w));
+#pragma unroll
+      for (int o = 4; o > 0; o >>= 1) {
+        mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+      }
+      if ((lane & 7) == 0 && v < nvec) { cmin[v >> 3] = mn; cmax[v >> 3] = mx; }
+    }
   }
   __syncthreads();
 
@@ -100,12 +151,33 @@ quantize_rtn_kernel(const float* __restrict__ W, int K, int g,
   __syncthreads();
 
   uint32_t* qrow = qweight + (size_t)row * chunks * BITS;
-  for (int c = warp; c < chunks; c += kQuantWarps) {
-    const int gi = c / cpg;
-    const float s = gscale[gi], z = gzero[gi];
-    float q = __fadd_rn(rintf(__fdiv_rn(w[c * 32 + lane], s)), z);
-    q = fminf(fmaxf(q, 0.0f), qmax);
-    warp_pack_store<BITS>((uint32_t)q, lane, qrow + c * BITS);
+  for (int vb = 0; vb < nvec; vb += kQuantThreads * UNROLL) {
+    const int v0 = vb + threadIdx.x;
+    float4 x[UNROLL];
+#pragma unroll
+    for (int u = 0; u < UNROLL; ++u) {
+      const int v = v0 + u * kQuantThreads;
+      x[u] = v < nvec ? __ldg(w4 + v) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+#pragma unroll
+    for (int u = 0; u < UNROLL; ++u) {
+      const int v = v0 + u * kQuantThreads;
+      const bool in = v < nvec;
+      const int chunk = in ? (v >> 3) : 0;
+      const int gi = chunk / cpg;
+      const float s = gscale[gi], z = gzero[gi];
+      const float rs = __frcp_rn(s);
+      const float xs[4] = {x[u].x, x[u].y, x[u].z, x[u].w};
+      uint32_t piece = 0u;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        float q = __fadd_rn(rint_of_quotient(xs[e], s, rs), z);
+        q = fminf(fmaxf(q, 0.0f), qmax);
+        piece |= (uint32_t)q << (BITS * e);
+      }
+      const uint32_t word = group8_pack<BITS>(piece, lane);
+      if (in && (lane & 7) < BITS) qrow[chunk * BITS + (lane & 7)] = word;
+    }
   }
 }
 

@@ -108,16 +108,9 @@ struct Unit {
   float s;
 };
 
-template <int BITS, bool TRANS>
-__device__ __forceinline__ Unit<BITS> load_unit(const QGemmParams& p, int r0, int c0, int dq) {
-  int i, col0;
-  if (!TRANS) {
-    i = r0 + (dq & 127);
-    col0 = c0 + 32 * (dq >> 7);
-  } else {
-    i = c0 + (dq & 63);
-    col0 = r0 + 32 * (dq >> 6);
-  }
+// Weight row i, columns [col0, col0 + 32).
+template <int BITS>
+__device__ __forceinline__ Unit<BITS> load_unit(const QGemmParams& p, int i, int col0) {
   Unit<BITS> u;
   if (i < p.N && col0 < p.K) {
     const uint32_t* src = p.qw + (size_t)i * p.wpr + (col0 >> 5) * BITS;
@@ -140,6 +133,21 @@ __device__ __forceinline__ Unit<BITS> load_unit(const QGemmParams& p, int r0, in
   return u;
 }
 
+// Dequantise one unit and store its 64 bytes (four 16-byte chunks starting at
+// chunk0) into a 128-byte tile row; the chunk index is XORed with (row & 7)
+// as the 128-byte swizzle requires.
+template <int BITS, bool FOLD>
+__device__ __forceinline__ void store_unit(const Unit<BITS>& u, uint8_t* row_ptr, int chunk0,
+                                           int swz) {
+  uint32_t o[16];
+  dq::unit32_natural<BITS, FOLD>(u.w, u.z, u.s, o);
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    *reinterpret_cast<uint4*>(row_ptr + (((chunk0 + q) ^ swz) << 4)) =
+        make_uint4(o[4 * q], o[4 * q + 1], o[4 * q + 2], o[4 * q + 3]);
+  }
+}
+
 template <int BITS, bool TRANS, bool FOLD>
 __global__ void __launch_bounds__(kQgemmThreads, 1)
 qgemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const QGemmParams p) {
@@ -151,7 +159,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const QGemmParams p) 
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
-      mbar_init(smem_u32(&bars->full_a[s]), kDequantThreads);
+      mbar_init(smem_u32(&bars->full_a[s]), TRANS ? kDequantThreads : kDequantThreads / 2);
       mbar_init(smem_u32(&bars->full_b[s]), 1);
       mbar_init(smem_u32(&bars->empty[s]), 1);
     }
@@ -260,58 +268,87 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const QGemmParams p) 
     }
   } else if (warp >= 8) {
     // ------------------------------------------------------- weight dequant
-    const int dq = threadIdx.x - 256;
-    // Destination of this thread's 32 columns (64 bytes = four 16-byte chunks)
-    // inside the 128-byte-swizzled tile: 16-byte chunk index XOR (row & 7).
-    int row_off, chunk0, swz;
-    if (!TRANS) {
-      const int row = dq & 127;
-      row_off = row * 128;
-      chunk0 = (dq >> 7) * 4;
-      swz = row & 7;
-    } else {
-      const int crow = dq & 63;
-      const int quarter = dq >> 6;
-      row_off = (quarter >> 1) * (64 * 128) + crow * 128;
-      chunk0 = (quarter & 1) * 4;
-      swz = crow & 7;
-    }
+    // Lane mapping: 8 weight rows x 4 units of 32 columns per warp instruction,
+    // so the four lanes of a row read one contiguous 48/64-byte run of packed
+    // words and share their (s, z) address.
+    const int dw = warp - 8;
+    const int row8 = lane & 7;
+    const int u4 = lane >> 3;
     const int my_tiles = (total_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
-    const uint32_t total_it = (uint32_t)my_tiles * (uint32_t)p.k_blocks;
-    // Flattened (tile, k-block) walk with a two-deep register prefetch of the
-    // packed words so that global latency hides behind the conversions.
-    auto coords = [&](uint32_t it, int& r0, int& c0) {
-      const int tile = blockIdx.x + (int)(it / (uint32_t)p.k_blocks) * gridDim.x;
-      r0 = (tile % p.r_tiles) * BM;
-      c0 = (int)(it % (uint32_t)p.k_blocks) * BK;
-    };
-    Unit<BITS> u0, u1;
-    {
-      int r0, c0;
-      if (total_it > 0) { coords(0, r0, c0); u0 = load_unit<BITS, TRANS>(p, r0, c0, dq); }
-      if (total_it > 1) { coords(1, r0, c0); u1 = load_unit<BITS, TRANS>(p, r0, c0, dq); }
-    }
-    for (uint32_t it = 0; it < total_it; ++it) {
-      const Unit<BITS> cur = u0;
-      u0 = u1;
-      if (it + 2 < total_it) {
-        int r0, c0;
-        coords(it + 2, r0, c0);
-        u1 = load_unit<BITS, TRANS>(p, r0, c0, dq);
+    if constexpr (TRANS) {
+      // dX: a stage is 64 weight rows (contraction) x 128 columns = 4 units per row;
+      // every thread owns one unit of every stage.
+      const int crow = dw * 8 + row8;
+      const int row_off = (u4 >> 1) * (64 * 128) + crow * 128;
+      const int chunk0 = (u4 & 1) * 4;
+      const int swz = crow & 7;
+      const uint32_t total_it = (uint32_t)my_tiles * (uint32_t)p.k_blocks;
+      auto load_it = [&](uint32_t it) {
+        const int tile = blockIdx.x + (int)(it / (uint32_t)p.k_blocks) * gridDim.x;
+        const int r0 = (tile % p.r_tiles) * BM;
+        const int c0 = (int)(it % (uint32_t)p.k_blocks) * BK;
+        return load_unit<BITS>(p, c0 + crow, r0 + 32 * u4);
+      };
+      Unit<BITS> u0, u1;
+      if (total_it > 0) u0 = load_it(0);
+      if (total_it > 1) u1 = load_it(1);
+      for (uint32_t it = 0; it < total_it; ++it) {
+        const Unit<BITS> cur = u0;
+        u0 = u1;
+        if (it + 2 < total_it) u1 = load_it(it + 2);
+        const int s = it % STAGES;
+        const uint32_t ph = (it / STAGES) & 1u;
+        if (!mbar_wait(smem_u32(&bars->empty[s]), ph ^ 1u, abort_flag)) break;
+        store_unit<BITS, FOLD>(cur, sm.a[s] + row_off, chunk0, swz);
+        fence_proxy_async_smem();
+        mbar_arrive(smem_u32(&bars->full_a[s]));
       }
-      const int s = it % STAGES;
-      const uint32_t ph = (it / STAGES) & 1u;
-      uint32_t o[16];
-      dq::unit32_natural<BITS, FOLD>(cur.w, cur.z, cur.s, o);
-      if (!mbar_wait(smem_u32(&bars->empty[s]), ph ^ 1u, abort_flag)) break;
-      uint8_t* dst = sm.a[s] + row_off;
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        *reinterpret_cast<uint4*>(dst + (((chunk0 + q) ^ swz) << 4)) =
-            make_uint4(o[4 * q], o[4 * q + 1], o[4 * q + 2], o[4 * q + 3]);
+    } else {
+      // forward: a stage is 128 weight rows x 64 columns = 2 units per row, so the
+      // threads walk pairs of stages (128 columns): units 0,1 belong to the even
+      // k-block of the pair, units 2,3 to the odd one, and each thread owns two
+      // rows (r, r + 8) of one k-block.
+      const int half = u4 >> 1;
+      const int rowA = dw * 16 + row8;
+      const int chunk0 = (u4 & 1) * 4;
+      const int swz = row8;               // (rowA & 7) == ((rowA + 8) & 7) == row8
+      const int pairs = (p.k_blocks + 1) / 2;
+      const uint32_t total_pairs = (uint32_t)my_tiles * (uint32_t)pairs;
+      auto locate = [&](uint32_t q, int& r0, int& kb, uint32_t& it) {
+        const uint32_t tl = q / (uint32_t)pairs;
+        const int tile = blockIdx.x + (int)tl * gridDim.x;
+        r0 = (tile % p.r_tiles) * BM;
+        kb = 2 * (int)(q % (uint32_t)pairs) + half;
+        it = tl * (uint32_t)p.k_blocks + (uint32_t)kb;
+        return kb < p.k_blocks;
+      };
+      auto load_pair = [&](uint32_t q, Unit<BITS>& a, Unit<BITS>& b) {
+        int r0, kb;
+        uint32_t it;
+        if (locate(q, r0, kb, it)) {
+          const int col0 = kb * BK + 32 * (u4 & 1);
+          a = load_unit<BITS>(p, r0 + rowA, col0);
+          b = load_unit<BITS>(p, r0 + rowA + 8, col0);
+        }
+      };
+      Unit<BITS> a0, b0, a1, b1;
+      if (total_pairs > 0) load_pair(0, a0, b0);
+      for (uint32_t q = 0; q < total_pairs; ++q) {
+        if (q + 1 < total_pairs) load_pair(q + 1, a1, b1);
+        int r0, kb;
+        uint32_t it;
+        if (locate(q, r0, kb, it)) {
+          const int s = it % STAGES;
+          const uint32_t ph = (it / STAGES) & 1u;
+          if (!mbar_wait(smem_u32(&bars->empty[s]), ph ^ 1u, abort_flag)) break;
+          store_unit<BITS, FOLD>(a0, sm.a[s] + rowA * 128, chunk0, swz);
+          store_unit<BITS, FOLD>(b0, sm.a[s] + (rowA + 8) * 128, chunk0, swz);
+          fence_proxy_async_smem();
+          mbar_arrive(smem_u32(&bars->full_a[s]));
+        }
+        a0 = a1;
+        b0 = b1;
       }
-      fence_proxy_async_smem();
-      mbar_arrive(smem_u32(&bars->full_a[s]));
     }
   }
 
@@ -341,25 +378,45 @@ struct DsParams {
   int* status;
 };
 
+// A CTA pair (cta_group::2) owns a 256 x 256 tile of dW: CTA `rank` holds rows
+// [i0 + 128*rank, +128) of dY^T as its A operand and accumulator, and loads the
+// 128 columns [j0 + 128*rank, +128) of X as its half of the shared B operand.
+// The leader CTA (rank 0) issues every MMA; both CTAs' TMA loads credit the
+// leader's "full" barrier and tcgen05.commit releases the stage in both CTAs.
+constexpr int DS_STAGES = 6;
+constexpr int DS_STAGE_BYTES = 2 * (BM * BK * 2);                      // A 16 KiB + B half 16 KiB
+constexpr int DS_SMEM_BYTES = DS_STAGES * DS_STAGE_BYTES + 1024 + 512;
+
+struct DsBarriers {
+  uint64_t full[DS_STAGES];     // leader: bytes of both CTAs landed
+  uint64_t empty[DS_STAGES];    // each CTA: MMAs that read the stage completed
+  uint64_t acc_full[2];         // each CTA: accumulator ready
+  uint64_t acc_empty[2];        // leader: both CTAs' epilogues drained the accumulator
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
 template <int BITS>
 __global__ void __launch_bounds__(kDsThreads, 1)
 ds_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_constant__ CUtensorMap tmap_x,
           const DsParams p) {
   extern __shared__ uint8_t smem_raw[];
-  SmemView sm = carve_smem(smem_raw);
-  Barriers* bars = sm.bars;
+  uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
+                                             ~static_cast<uintptr_t>(1023));
+  DsBarriers* bars = reinterpret_cast<DsBarriers*>(base + DS_STAGES * DS_STAGE_BYTES);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  const bool leader = rank == 0;
   volatile int* abort_flag = &bars->abort_flag;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < STAGES; ++s) {
-      mbar_init(smem_u32(&bars->full_a[s]), 1);   // unused here
-      mbar_init(smem_u32(&bars->full_b[s]), 1);
+    for (int s = 0; s < DS_STAGES; ++s) {
+      mbar_init(smem_u32(&bars->full[s]), 1);
       mbar_init(smem_u32(&bars->empty[s]), 1);
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(smem_u32(&bars->acc_full[b]), 1);
-      mbar_init(smem_u32(&bars->acc_empty[b]), 256);
+      mbar_init(smem_u32(&bars->acc_empty[b]), 16);   // 8 epilogue warps in each of the 2 CTAs
     }
     bars->abort_flag = 0;
     fence_mbar_init();
@@ -367,66 +424,70 @@ ds_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_constant__ C
     prefetch_tmap(&tmap_x);
   }
   if (warp == 2) {
-    tmem_alloc(smem_u32(&bars->tmem_base), TMEM_COLS);
-    tmem_relinquish();
+    tmem_alloc_pair(smem_u32(&bars->tmem_base), TMEM_COLS);
+    tmem_relinquish_pair();
   }
   tc_fence_before();
   __syncthreads();
+  cluster_sync_all();          // barriers of both CTAs initialised before any remote arrive
   tc_fence_after();
   const uint32_t tmem_base = bars->tmem_base;
-  const int total_tiles = p.i_tiles * p.j_tiles;
+  const int total_tiles = p.i_tiles * p.j_tiles;   // pair tiles (256 x 256)
+  const int pair = blockIdx.x >> 1;
+  const int n_pairs = gridDim.x >> 1;
 
   if (warp == 0) {
     if (lane == 0) {
       uint32_t it = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
-        const int i0 = (tile % p.i_tiles) * BM;
-        const int j0 = (tile / p.i_tiles) * BN;
+      for (int tile = pair; ok && tile < total_tiles; tile += n_pairs) {
+        const int i0 = (tile % p.i_tiles) * (2 * BM) + (int)rank * BM;
+        const int j0 = (tile / p.i_tiles) * BN + (int)rank * (BN / 2);
         for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
-          const int s = it % STAGES;
-          const uint32_t ph = (it / STAGES) & 1u;
-          if (!mbar_wait(smem_u32(&bars->empty[s]), ph ^ 1u, abort_flag)) { ok = false; break; }
-          const uint32_t bar = smem_u32(&bars->full_b[s]);
-          mbar_arrive_expect_tx(bar, STAGE_BYTES);
+          const int s = it % DS_STAGES;
+          const uint32_t ph = (it / DS_STAGES) & 1u;
+          if (!mbar_wait_cluster(smem_u32(&bars->empty[s]), ph ^ 1u, abort_flag)) { ok = false; break; }
+          const uint32_t bar = mapa_shared(smem_u32(&bars->full[s]), 0);
+          if (leader) mbar_arrive_expect_tx(smem_u32(&bars->full[s]), 2 * DS_STAGE_BYTES);
+          uint8_t* st = base + s * DS_STAGE_BYTES;
           // Each box is 64 contiguous features x 64 tokens = one 8 KiB MN-major chunk.
 #pragma unroll
-          for (int m = 0; m < BM / 64; ++m)
-            tma_load_2d(smem_u32(sm.a[s]) + m * 8192, &tmap_dy, bar, i0 + 64 * m, kb * BK);
+          for (int m = 0; m < 2; ++m)
+            tma_load_2d_pair(smem_u32(st) + m * 8192, &tmap_dy, bar, i0 + 64 * m, kb * BK);
 #pragma unroll
-          for (int m = 0; m < BN / 64; ++m)
-            tma_load_2d(smem_u32(sm.b[s]) + m * 8192, &tmap_x, bar, j0 + 64 * m, kb * BK);
+          for (int m = 0; m < 2; ++m)
+            tma_load_2d_pair(smem_u32(st) + 16384 + m * 8192, &tmap_x, bar, j0 + 64 * m, kb * BK);
         }
       }
     }
   } else if (warp == 1) {
-    if (lane == 0) {
-      constexpr uint32_t idesc = idesc_bf16_f32(BM, BN, 1, 1);
+    if (leader && lane == 0) {
+      constexpr uint32_t idesc = idesc_bf16_f32(2 * BM, BN, 1, 1);
       uint32_t it = 0;
       int local = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++local) {
+      for (int tile = pair; ok && tile < total_tiles; tile += n_pairs, ++local) {
         const int buf = local & 1;
         const uint32_t acc_ph = (local >> 1) & 1u;
-        if (!mbar_wait(smem_u32(&bars->acc_empty[buf]), acc_ph ^ 1u, abort_flag)) { ok = false; break; }
+        if (!mbar_wait_cluster(smem_u32(&bars->acc_empty[buf]), acc_ph ^ 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + buf * BN;
         for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
-          const int s = it % STAGES;
-          const uint32_t ph = (it / STAGES) & 1u;
-          if (!mbar_wait(smem_u32(&bars->full_b[s]), ph, abort_flag)) { ok = false; break; }
+          const int s = it % DS_STAGES;
+          const uint32_t ph = (it / DS_STAGES) & 1u;
+          if (!mbar_wait_cluster(smem_u32(&bars->full[s]), ph, abort_flag)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t a_addr = smem_u32(sm.a[s]);
-          const uint32_t b_addr = smem_u32(sm.b[s]);
+          const uint32_t a_addr = smem_u32(base + s * DS_STAGE_BYTES);
+          const uint32_t b_addr = a_addr + 16384;
 #pragma unroll
           for (int k = 0; k < BK / UMMA_K; ++k) {
             const uint64_t adesc = smem_desc_sw128(a_addr + k * (UMMA_K * 128), 8192, 1024);
             const uint64_t bdesc = smem_desc_sw128(b_addr + k * (UMMA_K * 128), 8192, 1024);
-            mma_bf16_ss(d_tmem, adesc, bdesc, idesc, (kb | k) != 0 ? 1u : 0u);
+            mma_bf16_ss_pair(d_tmem, adesc, bdesc, idesc, (kb | k) != 0 ? 1u : 0u);
           }
-          mma_commit(smem_u32(&bars->empty[s]));
+          mma_commit_pair(smem_u32(&bars->empty[s]), 3);
         }
-        if (ok) mma_commit(smem_u32(&bars->acc_full[buf]));
+        if (ok) mma_commit_pair(smem_u32(&bars->acc_full[buf]), 3);
       }
     }
   } else if (warp >= 4) {
@@ -435,14 +496,16 @@ ds_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_constant__ C
     const int half = (warp - 4) >> 2;
     const int npieces = p.K / p.piece;
     const int chunks_per_piece = p.piece >> 5;
+    const uint32_t acc_empty_leader0 = mapa_shared(smem_u32(&bars->acc_empty[0]), 0);
+    const uint32_t acc_empty_leader1 = mapa_shared(smem_u32(&bars->acc_empty[1]), 0);
     int local = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++local) {
-      const int i0 = (tile % p.i_tiles) * BM;
+    for (int tile = pair; ok && tile < total_tiles; tile += n_pairs, ++local) {
+      const int i0 = (tile % p.i_tiles) * (2 * BM) + (int)rank * BM;
       const int j0 = (tile / p.i_tiles) * BN;
       const int buf = local & 1;
       const uint32_t acc_ph = (local >> 1) & 1u;
-      if (!mbar_wait(smem_u32(&bars->acc_full[buf]), acc_ph, abort_flag)) { ok = false; break; }
+      if (!mbar_wait_cluster(smem_u32(&bars->acc_full[buf]), acc_ph, abort_flag)) { ok = false; break; }
       tc_fence_after();
       const int i = i0 + quarter * 32 + lane;
       float acc = 0.0f;
@@ -481,16 +544,18 @@ ds_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_constant__ C
         }
       }
       tc_fence_before();
-      mbar_arrive(smem_u32(&bars->acc_empty[buf]));
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(buf ? acc_empty_leader1 : acc_empty_leader0);
     }
   }
 
   if (*abort_flag) drain_after_abort();
   tc_fence_before();
   __syncthreads();
+  cluster_sync_all();   // no CTA leaves while its peer may still signal its barriers
   if (warp == 2) {
     tc_fence_after();
-    tmem_dealloc(tmem_base, TMEM_COLS);
+    tmem_dealloc_pair(tmem_base, TMEM_COLS);
   }
   if (threadIdx.x == 0 && bars->abort_flag) {
     atomicExch(p.status, (int)PEQA_ERR_DEVICE_TIMEOUT);
@@ -646,7 +711,7 @@ int launch_ds(const peqa_qweight_t* w, int g, const void* X, const void* dY, int
   p.piece = ds_piece(g);
   const bool direct = (p.piece == g);
   p.out = direct ? dS : static_cast<float*>(workspace);
-  p.i_tiles = (p.N + BM - 1) / BM;
+  p.i_tiles = (p.N + 2 * BM - 1) / (2 * BM);   // 256-row pair tiles
   p.j_tiles = (p.K + BN - 1) / BN;
   p.k_blocks = (T + BK - 1) / BK;
   PEQA_TRY(status_word(&p.status));
@@ -656,15 +721,27 @@ int launch_ds(const peqa_qweight_t* w, int g, const void* X, const void* dY, int
   int sms = 0;
   PEQA_TRY(sm_count(&sms));
   const int tiles = p.i_tiles * p.j_tiles;
-  const int grid = tiles < sms ? tiles : sms;
+  const int max_pairs = sms / 2;
+  const int pairs = tiles < max_pairs ? tiles : max_pairs;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2 * pairs, 1, 1);
+  cfg.blockDim = dim3(kDsThreads, 1, 1);
+  cfg.dynamicSmemBytes = DS_SMEM_BYTES;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
   if (w->bits == 4) {
-    PEQA_TRY(set_smem(ds_kernel<4>));
-    ds_kernel<4><<<grid, kDsThreads, SMEM_BYTES, st>>>(tmap_dy, tmap_x, p);
+    PEQA_CUDA(cudaFuncSetAttribute(ds_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, DS_SMEM_BYTES));
+    PEQA_CUDA(cudaLaunchKernelEx(&cfg, ds_kernel<4>, tmap_dy, tmap_x, p));
   } else {
-    PEQA_TRY(set_smem(ds_kernel<3>));
-    ds_kernel<3><<<grid, kDsThreads, SMEM_BYTES, st>>>(tmap_dy, tmap_x, p);
+    PEQA_CUDA(cudaFuncSetAttribute(ds_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, DS_SMEM_BYTES));
+    PEQA_CUDA(cudaLaunchKernelEx(&cfg, ds_kernel<3>, tmap_dy, tmap_x, p));
   }
-  PEQA_CUDA(cudaGetLastError());
   if (!direct) {
     const long long n_out = (long long)p.N * p.G;
     const int ppg = g / p.piece;
