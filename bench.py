@@ -41,6 +41,24 @@ def load_peaks():
         return dict(FALLBACK_PEAKS), "fallback"
 
 
+def measured_traffic(kernel_name):
+    """DRAM bytes per launch from the committed ncu capture, or None when the kernel sources
+    have changed since the counters were taken."""
+    import hashlib
+    try:
+        with open(os.path.join(ROOT, "profiles", "dram_traffic_c2.json")) as f:
+            doc = json.load(f)
+        h = hashlib.sha256()
+        for name in ("gemm_sm100.cu", "dequant.cuh", "sm100_ptx.cuh", "decode.cu", "elementwise.cu"):
+            with open(os.path.join(ROOT, "paper_2305_14152_b200", "csrc", name), "rb") as f:
+                h.update(f.read())
+        if h.hexdigest() != doc["kernel_sources_sha256"] or doc.get("workload") != WORKLOAD:
+            return None
+        return doc["kernels"][kernel_name]["traffic_bytes"]
+    except Exception:
+        return None
+
+
 def draw_sets(n_sets):
     """Set 0 is the canonical workload draw; further sets continue the same seeded stream."""
     from paper_2305_14152_b200 import synth
@@ -270,7 +288,8 @@ def run_cuda(args):
     long_region = ms_total > 1000.0
     peak = peaks["bf16_tflops_sustained"] if long_region else peaks["bf16_tflops"]
     roofline = {"bound": "tensor", "kernel": stage_names[dom], "achieved": ach, "peak": peak,
-                "unit": "TFLOP/s", "frac": ach / peak, "traffic": None,
+                "unit": "TFLOP/s", "frac": ach / peak, "traffic": measured_traffic(stage_names[dom]),
+                "traffic_unit": "DRAM bytes per launch (ncu)",
                 "peak_source": f"{peak_src} bf16 {'sustained' if long_region else 'burst'}",
                 "frac_of_nominal_2250": ach / 2250.0,
                 "per_kernel_tflops": {stage_names[k]: 2.0 * T * N * K / (gemm[k] * 1e-3) / 1e12
