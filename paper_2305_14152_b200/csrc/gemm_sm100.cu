@@ -45,7 +45,8 @@ constexpr int UMMA_K = 16;   // contraction elements per tcgen05.mma
 constexpr int STAGES = 4;
 constexpr int A_BYTES = BM * BK * 2;   // 16 KiB
 constexpr int B_BYTES = BN * BK * 2;   // 32 KiB
-constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int PK_BYTES = 4096;         // packed codes of one stage (qgemm)
+constexpr int STAGE_BYTES = A_BYTES + B_BYTES + PK_BYTES;
 constexpr int TMEM_COLS = 512;         // two fp32 accumulators of 256 columns
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/;
 
@@ -56,6 +57,7 @@ constexpr int kDsThreads = 384;        // warps: 0 TMA, 1 MMA, 2 TMEM alloc, 4-1
 struct Barriers {
   uint64_t full_a[STAGES];   // dequantised weight tile written (qgemm only)
   uint64_t full_b[STAGES];   // TMA bytes landed
+  uint64_t full_pk[STAGES];  // packed codes landed (qgemm with TMA-staged codes)
   uint64_t empty[STAGES];    // MMAs that read the stage have completed
   uint64_t acc_full[2];      // accumulator ready for the epilogue
   uint64_t acc_empty[2];     // accumulator drained by the epilogue
@@ -66,6 +68,7 @@ struct Barriers {
 struct SmemView {
   uint8_t* a[STAGES];
   uint8_t* b[STAGES];
+  uint8_t* pk[STAGES];
   Barriers* bars;
 };
 
@@ -77,6 +80,7 @@ __device__ __forceinline__ SmemView carve_smem(uint8_t* raw) {
   for (int s = 0; s < STAGES; ++s) {
     v.a[s] = base + s * STAGE_BYTES;
     v.b[s] = base + s * STAGE_BYTES + A_BYTES;
+    v.pk[s] = base + s * STAGE_BYTES + A_BYTES + B_BYTES;
   }
   v.bars = reinterpret_cast<Barriers*>(base + STAGES * STAGE_BYTES);
   return v;
@@ -94,6 +98,7 @@ struct QGemmParams {
   const float* scales;
   __nv_bfloat16* out;   // [T, R]
   int N, K, G, g, T;
+  int g_shift;          // log2(g) when g is a power of two, else -1
   int wpr;              // packed words per weight row
   int R, C;             // output features, contraction length
   int r_tiles, t_tiles, k_blocks;
@@ -108,25 +113,33 @@ struct Unit {
   float s;
 };
 
-// Weight row i, columns [col0, col0 + 32).
-template <int BITS>
+__device__ __forceinline__ int group_of(const QGemmParams& p, int col) {
+  if (p.G == 1) return 0;
+  return p.g_shift >= 0 ? (col >> p.g_shift) : (col / p.g);
+}
+
+// Weight row i, columns [col0, col0 + 32): zero-point and scale, plus the packed
+// words when WORDS is set (otherwise the caller takes them from shared memory).
+template <int BITS, bool WORDS = true>
 __device__ __forceinline__ Unit<BITS> load_unit(const QGemmParams& p, int i, int col0) {
   Unit<BITS> u;
+#pragma unroll
+  for (int q = 0; q < BITS; ++q) u.w[q] = 0u;
   if (i < p.N && col0 < p.K) {
-    const uint32_t* src = p.qw + (size_t)i * p.wpr + (col0 >> 5) * BITS;
-    if constexpr (BITS == 4) {
-      const uint4 v = __ldg(reinterpret_cast<const uint4*>(src));
-      u.w[0] = v.x; u.w[1] = v.y; u.w[2] = v.z; u.w[3] = v.w;
-    } else {
-      u.w[0] = __ldg(src); u.w[1] = __ldg(src + 1); u.w[2] = __ldg(src + 2);
+    if (WORDS) {
+      const uint32_t* src = p.qw + (size_t)i * p.wpr + (col0 >> 5) * BITS;
+      if constexpr (BITS == 4) {
+        const uint4 v = __ldg(reinterpret_cast<const uint4*>(src));
+        u.w[0] = v.x; u.w[1] = v.y; u.w[2] = v.z; u.w[3] = v.w;
+      } else {
+        u.w[0] = __ldg(src); u.w[1] = __ldg(src + 1); u.w[2] = __ldg(src + 2);
+      }
     }
-    const size_t gidx = (size_t)i * p.G + col0 / p.g;
+    const size_t gidx = (size_t)i * p.G + group_of(p, col0);
     u.z = __ldg(p.zeros + gidx);
     u.s = __ldg(p.scales + gidx);
   } else {
     // Outside the matrix: codes equal to the zero-point dequantise to exactly 0.
-#pragma unroll
-    for (int q = 0; q < BITS; ++q) u.w[q] = 0u;
     u.z = 0u;
     u.s = 0.0f;
   }
@@ -148,9 +161,13 @@ __device__ __forceinline__ void store_unit(const Unit<BITS>& u, uint8_t* row_ptr
   }
 }
 
-template <int BITS, bool TRANS, bool FOLD>
+// PKTMA: the packed codes of a stage arrive by TMA in shared memory (needs a
+// 16-byte row pitch of the packed matrix); otherwise the dequant threads read
+// them from global memory themselves.
+template <int BITS, bool TRANS, bool FOLD, bool PKTMA>
 __global__ void __launch_bounds__(kQgemmThreads, 1)
-qgemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const QGemmParams p) {
+qgemm_kernel(const __grid_constant__ CUtensorMap tmap_act,
+             const __grid_constant__ CUtensorMap tmap_pk, const QGemmParams p) {
   extern __shared__ uint8_t smem_raw[];
   SmemView sm = carve_smem(smem_raw);
   Barriers* bars = sm.bars;
@@ -161,6 +178,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const QGemmParams p) 
     for (int s = 0; s < STAGES; ++s) {
       mbar_init(smem_u32(&bars->full_a[s]), TRANS ? kDequantThreads : kDequantThreads / 2);
       mbar_init(smem_u32(&bars->full_b[s]), 1);
+      mbar_init(smem_u32(&bars->full_pk[s]), 1);
       mbar_init(smem_u32(&bars->empty[s]), 1);
     }
     for (int b = 0; b < 2; ++b) {
@@ -170,6 +188,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const QGemmParams p) 
     bars->abort_flag = 0;
     fence_mbar_init();
     prefetch_tmap(&tmap_act);
+    if (PKTMA) prefetch_tmap(&tmap_pk);
   }
   if (warp == 2) {
     tmem_alloc(smem_u32(&bars->tmem_base), TMEM_COLS);
@@ -189,10 +208,25 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const QGemmParams p) 
       bool ok = true;
       for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
         const int t0 = (tile / p.r_tiles) * BN;
+        const int w0 = (tile % p.r_tiles) * BM;   // first weight row (forward) / column (dX) of the tile
         for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
           const int s = it % STAGES;
           const uint32_t ph = (it / STAGES) & 1u;
           if (!mbar_wait(smem_u32(&bars->empty[s]), ph ^ 1u, abort_flag)) { ok = false; break; }
+          if (PKTMA) {
+            // forward: 128 rows x 8 words holding the stage's 64 columns (3-bit: on odd
+            // k-blocks the 6 words start 2 words into the box, which keeps the box start
+            // 16-byte aligned); dX: 64 rows x the tile's 128 columns.
+            const uint32_t pbar = smem_u32(&bars->full_pk[s]);
+            if (!TRANS) {
+              mbar_arrive_expect_tx(pbar, 128 * 32);
+              tma_load_2d(smem_u32(sm.pk[s]), &tmap_pk, pbar,
+                          BITS == 3 ? 6 * kb - 2 * (kb & 1) : 8 * kb, w0);
+            } else {
+              mbar_arrive_expect_tx(pbar, 64 * 16 * BITS);
+              tma_load_2d(smem_u32(sm.pk[s]), &tmap_pk, pbar, (w0 >> 5) * BITS, kb * BK);
+            }
+          }
           const uint32_t bar = smem_u32(&bars->full_b[s]);
           mbar_arrive_expect_tx(bar, B_BYTES);
           tma_load_2d(smem_u32(sm.b[s]), &tmap_act, bar, kb * BK, t0);
@@ -283,25 +317,40 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const QGemmParams p) 
       const int chunk0 = (u4 & 1) * 4;
       const int swz = crow & 7;
       const uint32_t total_it = (uint32_t)my_tiles * (uint32_t)p.k_blocks;
-      auto load_it = [&](uint32_t it) {
-        const int tile = blockIdx.x + (int)(it / (uint32_t)p.k_blocks) * gridDim.x;
-        const int r0 = (tile % p.r_tiles) * BM;
-        const int c0 = (int)(it % (uint32_t)p.k_blocks) * BK;
-        return load_unit<BITS>(p, c0 + crow, r0 + 32 * u4);
+      // (tile, k-block) of the unit being prefetched, advanced without divisions
+      int pf_tile = blockIdx.x, pf_kb = 0;
+      int pf_r0 = (pf_tile % p.r_tiles) * BM;
+      auto load_next = [&]() {
+        Unit<BITS> u = load_unit<BITS, !PKTMA>(p, pf_kb * BK + crow, pf_r0 + 32 * u4);
+        if (++pf_kb == p.k_blocks) {
+          pf_kb = 0;
+          pf_tile += gridDim.x;
+          pf_r0 = (pf_tile % p.r_tiles) * BM;
+        }
+        return u;
       };
       Unit<BITS> u0, u1;
-      if (total_it > 0) u0 = load_it(0);
-      if (total_it > 1) u1 = load_it(1);
+      if (total_it > 0) u0 = load_next();
+      if (total_it > 1) u1 = load_next();
+      int s = 0;
+      uint32_t ph = 0;
       for (uint32_t it = 0; it < total_it; ++it) {
-        const Unit<BITS> cur = u0;
+        Unit<BITS> cur = u0;
         u0 = u1;
-        if (it + 2 < total_it) u1 = load_it(it + 2);
-        const int s = it % STAGES;
-        const uint32_t ph = (it / STAGES) & 1u;
-        if (!mbar_wait(smem_u32(&bars->empty[s]), ph ^ 1u, abort_flag)) break;
+        if (it + 2 < total_it) u1 = load_next();
+        if (PKTMA) {
+          // the codes landing implies that the producer saw this stage released
+          if (!mbar_wait(smem_u32(&bars->full_pk[s]), ph, abort_flag)) break;
+          const uint32_t* src = reinterpret_cast<const uint32_t*>(sm.pk[s]) + crow * (4 * BITS) + u4 * BITS;
+#pragma unroll
+          for (int q = 0; q < BITS; ++q) cur.w[q] = src[q];
+        } else {
+          if (!mbar_wait(smem_u32(&bars->empty[s]), ph ^ 1u, abort_flag)) break;
+        }
         store_unit<BITS, FOLD>(cur, sm.a[s] + row_off, chunk0, swz);
         fence_proxy_async_smem();
         mbar_arrive(smem_u32(&bars->full_a[s]));
+        if (++s == STAGES) { s = 0; ph ^= 1u; }
       }
     } else {
       // forward: a stage is 128 weight rows x 64 columns = 2 units per row, so the
@@ -314,33 +363,45 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const QGemmParams p) 
       const int swz = row8;               // (rowA & 7) == ((rowA + 8) & 7) == row8
       const int pairs = (p.k_blocks + 1) / 2;
       const uint32_t total_pairs = (uint32_t)my_tiles * (uint32_t)pairs;
-      auto locate = [&](uint32_t q, int& r0, int& kb, uint32_t& it) {
-        const uint32_t tl = q / (uint32_t)pairs;
-        const int tile = blockIdx.x + (int)tl * gridDim.x;
-        r0 = (tile % p.r_tiles) * BM;
-        kb = 2 * (int)(q % (uint32_t)pairs) + half;
-        it = tl * (uint32_t)p.k_blocks + (uint32_t)kb;
-        return kb < p.k_blocks;
-      };
-      auto load_pair = [&](uint32_t q, Unit<BITS>& a, Unit<BITS>& b) {
-        int r0, kb;
-        uint32_t it;
-        if (locate(q, r0, kb, it)) {
+      // prefetch cursor (one pair of k-blocks ahead), advanced without divisions
+      int pf_tile = blockIdx.x, pf_pair = 0;
+      int pf_r0 = (pf_tile % p.r_tiles) * BM;
+      auto load_next = [&](Unit<BITS>& a, Unit<BITS>& b) {
+        const int kb = 2 * pf_pair + half;
+        if (kb < p.k_blocks) {
           const int col0 = kb * BK + 32 * (u4 & 1);
-          a = load_unit<BITS>(p, r0 + rowA, col0);
-          b = load_unit<BITS>(p, r0 + rowA + 8, col0);
+          a = load_unit<BITS, !PKTMA>(p, pf_r0 + rowA, col0);
+          b = load_unit<BITS, !PKTMA>(p, pf_r0 + rowA + 8, col0);
+        }
+        if (++pf_pair == pairs) {
+          pf_pair = 0;
+          pf_tile += gridDim.x;
+          pf_r0 = (pf_tile % p.r_tiles) * BM;
         }
       };
       Unit<BITS> a0, b0, a1, b1;
-      if (total_pairs > 0) load_pair(0, a0, b0);
+      if (total_pairs > 0) load_next(a0, b0);
+      int cur_pair = 0;
+      uint32_t it_base = 0;               // stage counter of k-block 0 of the current tile
       for (uint32_t q = 0; q < total_pairs; ++q) {
-        if (q + 1 < total_pairs) load_pair(q + 1, a1, b1);
-        int r0, kb;
-        uint32_t it;
-        if (locate(q, r0, kb, it)) {
+        if (q + 1 < total_pairs) load_next(a1, b1);
+        const int kb = 2 * cur_pair + half;
+        if (kb < p.k_blocks) {
+          const uint32_t it = it_base + (uint32_t)kb;
           const int s = it % STAGES;
           const uint32_t ph = (it / STAGES) & 1u;
-          if (!mbar_wait(smem_u32(&bars->empty[s]), ph ^ 1u, abort_flag)) break;
+          if (PKTMA) {
+            if (!mbar_wait(smem_u32(&bars->full_pk[s]), ph, abort_flag)) break;
+            const int woff = (BITS == 3 ? 2 * (kb & 1) : 0) + (u4 & 1) * BITS;
+            const uint32_t* src = reinterpret_cast<const uint32_t*>(sm.pk[s]) + woff;
+#pragma unroll
+            for (int e = 0; e < BITS; ++e) {
+              a0.w[e] = src[rowA * 8 + e];
+              b0.w[e] = src[(rowA + 8) * 8 + e];
+            }
+          } else {
+            if (!mbar_wait(smem_u32(&bars->empty[s]), ph ^ 1u, abort_flag)) break;
+          }
           store_unit<BITS, FOLD>(a0, sm.a[s] + rowA * 128, chunk0, swz);
           store_unit<BITS, FOLD>(b0, sm.a[s] + (rowA + 8) * 128, chunk0, swz);
           fence_proxy_async_smem();
@@ -348,6 +409,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const QGemmParams p) 
         }
         a0 = a1;
         b0 = b1;
+        if (++cur_pair == pairs) { cur_pair = 0; it_base += (uint32_t)p.k_blocks; }
       }
     }
   }
@@ -628,13 +690,21 @@ int set_smem(Kern k) {
   return PEQA_OK;
 }
 
-template <int BITS, bool TRANS, bool FOLD>
-int launch_qgemm_t(const CUtensorMap& tmap, const QGemmParams& p, int grid, cudaStream_t st) {
-  auto kern = qgemm_kernel<BITS, TRANS, FOLD>;
+template <int BITS, bool TRANS, bool FOLD, bool PKTMA>
+int launch_qgemm_k(const CUtensorMap& tmap, const CUtensorMap& tmap_pk, const QGemmParams& p,
+                   int grid, cudaStream_t st) {
+  auto kern = qgemm_kernel<BITS, TRANS, FOLD, PKTMA>;
   PEQA_TRY(set_smem(kern));
-  kern<<<grid, kQgemmThreads, SMEM_BYTES, st>>>(tmap, p);
+  kern<<<grid, kQgemmThreads, SMEM_BYTES, st>>>(tmap, tmap_pk, p);
   PEQA_CUDA(cudaGetLastError());
   return PEQA_OK;
+}
+
+template <int BITS, bool TRANS, bool FOLD>
+int launch_qgemm_t(const CUtensorMap& tmap, const CUtensorMap& tmap_pk, bool pktma,
+                   const QGemmParams& p, int grid, cudaStream_t st) {
+  return pktma ? launch_qgemm_k<BITS, TRANS, FOLD, true>(tmap, tmap_pk, p, grid, st)
+               : launch_qgemm_k<BITS, TRANS, FOLD, false>(tmap, tmap_pk, p, grid, st);
 }
 
 int launch_qgemm(const peqa_qweight_t* w, int g, const void* act, int T, void* out, bool trans,
@@ -648,6 +718,9 @@ int launch_qgemm(const peqa_qweight_t* w, int g, const void* act, int T, void* o
   p.K = w->in_features;
   p.g = g;
   p.G = p.K / g;
+  p.g_shift = -1;
+  for (int b = 5; b < 31; ++b)
+    if ((1 << b) == g) p.g_shift = b;
   p.T = T;
   p.wpr = p.K * w->bits / 32;
   p.R = trans ? p.K : p.N;
@@ -663,14 +736,29 @@ int launch_qgemm(const peqa_qweight_t* w, int g, const void* act, int T, void* o
   const int tiles = p.r_tiles * p.t_tiles;
   const int grid = tiles < sms ? tiles : sms;
   const bool fold = trans || p.G > 1;
-  if (w->bits == 4) {
-    if (trans) return launch_qgemm_t<4, true, true>(tmap, p, grid, st);
-    return fold ? launch_qgemm_t<4, false, true>(tmap, p, grid, st)
-                : launch_qgemm_t<4, false, false>(tmap, p, grid, st);
+  // Packed codes by TMA need a 16-byte row pitch: always true for 4-bit, K % 128 == 0 for 3-bit.
+  const bool pktma = ((size_t)p.wpr * 4) % 16 == 0;
+  CUtensorMap tmap_pk = tmap;
+  if (pktma) {
+    EncodeTiledFn enc = nullptr;
+    PEQA_TRY(get_encode_fn(&enc));
+    cuuint64_t dims[2] = {(cuuint64_t)p.wpr, (cuuint64_t)p.N};
+    cuuint64_t strides[1] = {(cuuint64_t)p.wpr * 4};
+    cuuint32_t box[2] = {trans ? (cuuint32_t)(4 * w->bits) : 8u, trans ? 64u : 128u};
+    cuuint32_t estr[2] = {1, 1};
+    if (enc(&tmap_pk, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<uint32_t*>(w->qweight), dims,
+            strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return cuda_fail(cudaErrorInvalidValue);
   }
-  if (trans) return launch_qgemm_t<3, true, true>(tmap, p, grid, st);
-  return fold ? launch_qgemm_t<3, false, true>(tmap, p, grid, st)
-              : launch_qgemm_t<3, false, false>(tmap, p, grid, st);
+  if (w->bits == 4) {
+    if (trans) return launch_qgemm_t<4, true, true>(tmap, tmap_pk, pktma, p, grid, st);
+    return fold ? launch_qgemm_t<4, false, true>(tmap, tmap_pk, pktma, p, grid, st)
+                : launch_qgemm_t<4, false, false>(tmap, tmap_pk, pktma, p, grid, st);
+  }
+  if (trans) return launch_qgemm_t<3, true, true>(tmap, tmap_pk, pktma, p, grid, st);
+  return fold ? launch_qgemm_t<3, false, true>(tmap, tmap_pk, pktma, p, grid, st)
+              : launch_qgemm_t<3, false, false>(tmap, tmap_pk, pktma, p, grid, st);
 }
 
 int gcd_int(int a, int b) { return b == 0 ? a : gcd_int(b, a % b); }

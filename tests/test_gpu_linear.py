@@ -42,6 +42,15 @@ def test_ragged_multi_tile(bits, g):
     _run_all(d, bits, g)
 
 
+@pytest.mark.parametrize("bits,g", [(4, 0), (3, 0), (3, 64), (4, 32), (3, 192)])
+def test_in_features_not_a_multiple_of_128(bits, g):
+    # K = 192 and 576 are multiples of 64 only: 3-bit rows then have no 16-byte pitch and the
+    # kernels read the packed codes directly instead of through TMA
+    for K in (192, 576):
+        d = synth.custom(200 + bits + g + K, 264, K, 150, bits, g, outliers=True, sigma_dy=1e-2)
+        _run_all(d, bits, g)
+
+
 @pytest.mark.parametrize("T", [1, 7, 64, 257, 513])
 def test_token_counts(T):
     d = synth.custom(T, 256, 512, T, 3, 128, sigma_dy=1e-2)
