@@ -46,9 +46,10 @@ constexpr int STAGES = 4;
 constexpr int A_BYTES = BM * BK * 2;   // 16 KiB
 constexpr int B_BYTES = BN * BK * 2;   // 32 KiB
 constexpr int PK_BYTES = 4096;         // packed codes of one stage (qgemm)
-constexpr int STAGE_BYTES = A_BYTES + B_BYTES + PK_BYTES;
+constexpr int PK_SLOTS = 8;            // their own, deeper ring: the codes run ahead of the operands
+constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int TMEM_COLS = 512;         // two fp32 accumulators of 256 columns
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + PK_SLOTS * PK_BYTES + 1024 /*align*/ + 512 /*barriers*/;
 
 constexpr int kQgemmThreads = 512;     // warps: 0 TMA, 1 MMA, 2 TMEM alloc, 4-7 epilogue, 8-15 dequant
 constexpr int kDequantThreads = 256;
@@ -57,7 +58,8 @@ constexpr int kDsThreads = 384;        // warps: 0 TMA, 1 MMA, 2 TMEM alloc, 4-1
 struct Barriers {
   uint64_t full_a[STAGES];   // dequantised weight tile written (qgemm only)
   uint64_t full_b[STAGES];   // TMA bytes landed
-  uint64_t full_pk[STAGES];  // packed codes landed (qgemm with TMA-staged codes)
+  uint64_t full_pk[PK_SLOTS];   // packed codes landed (qgemm with TMA-staged codes)
+  uint64_t empty_pk[PK_SLOTS];  // all dequant warps have read the slot
   uint64_t empty[STAGES];    // MMAs that read the stage have completed
   uint64_t acc_full[2];      // accumulator ready for the epilogue
   uint64_t acc_empty[2];     // accumulator drained by the epilogue
@@ -68,7 +70,7 @@ struct Barriers {
 struct SmemView {
   uint8_t* a[STAGES];
   uint8_t* b[STAGES];
-  uint8_t* pk[STAGES];
+  uint8_t* pk[PK_SLOTS];
   Barriers* bars;
 };
 
@@ -80,9 +82,10 @@ __device__ __forceinline__ SmemView carve_smem(uint8_t* raw) {
   for (int s = 0; s < STAGES; ++s) {
     v.a[s] = base + s * STAGE_BYTES;
     v.b[s] = base + s * STAGE_BYTES + A_BYTES;
-    v.pk[s] = base + s * STAGE_BYTES + A_BYTES + B_BYTES;
   }
-  v.bars = reinterpret_cast<Barriers*>(base + STAGES * STAGE_BYTES);
+#pragma unroll
+  for (int q = 0; q < PK_SLOTS; ++q) v.pk[q] = base + STAGES * STAGE_BYTES + q * PK_BYTES;
+  v.bars = reinterpret_cast<Barriers*>(base + STAGES * STAGE_BYTES + PK_SLOTS * PK_BYTES);
   return v;
 }
 
@@ -178,8 +181,11 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmap_act,
     for (int s = 0; s < STAGES; ++s) {
       mbar_init(smem_u32(&bars->full_a[s]), TRANS ? kDequantThreads : kDequantThreads / 2);
       mbar_init(smem_u32(&bars->full_b[s]), 1);
-      mbar_init(smem_u32(&bars->full_pk[s]), 1);
       mbar_init(smem_u32(&bars->empty[s]), 1);
+    }
+    for (int q = 0; q < PK_SLOTS; ++q) {
+      mbar_init(smem_u32(&bars->full_pk[q]), 1);
+      mbar_init(smem_u32(&bars->empty_pk[q]), kDequantThreads / 32);
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(smem_u32(&bars->acc_full[b]), 1);
@@ -208,28 +214,39 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmap_act,
       bool ok = true;
       for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
         const int t0 = (tile / p.r_tiles) * BN;
-        const int w0 = (tile % p.r_tiles) * BM;   // first weight row (forward) / column (dX) of the tile
         for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
           const int s = it % STAGES;
           const uint32_t ph = (it / STAGES) & 1u;
           if (!mbar_wait(smem_u32(&bars->empty[s]), ph ^ 1u, abort_flag)) { ok = false; break; }
-          if (PKTMA) {
-            // forward: 128 rows x 8 words holding the stage's 64 columns (3-bit: on odd
-            // k-blocks the 6 words start 2 words into the box, which keeps the box start
-            // 16-byte aligned); dX: 64 rows x the tile's 128 columns.
-            const uint32_t pbar = smem_u32(&bars->full_pk[s]);
-            if (!TRANS) {
-              mbar_arrive_expect_tx(pbar, 128 * 32);
-              tma_load_2d(smem_u32(sm.pk[s]), &tmap_pk, pbar,
-                          BITS == 3 ? 6 * kb - 2 * (kb & 1) : 8 * kb, w0);
-            } else {
-              mbar_arrive_expect_tx(pbar, 64 * 16 * BITS);
-              tma_load_2d(smem_u32(sm.pk[s]), &tmap_pk, pbar, (w0 >> 5) * BITS, kb * BK);
-            }
-          }
           const uint32_t bar = smem_u32(&bars->full_b[s]);
           mbar_arrive_expect_tx(bar, B_BYTES);
           tma_load_2d(smem_u32(sm.b[s]), &tmap_act, bar, kb * BK, t0);
+        }
+      }
+    }
+  } else if (warp == 3) {
+    // ------------------------------------------ packed-code TMA producer (one lane)
+    // forward: a box is 128 rows x 8 words holding the stage's 64 columns (3-bit: on odd
+    // k-blocks the 6 words start 2 words into the box, which keeps the box start
+    // 16-byte aligned); dX: 64 rows x the tile's 128 columns.
+    if (PKTMA && lane == 0) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+        const int w0 = (tile % p.r_tiles) * BM;   // first weight row (forward) / column (dX)
+        for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
+          const int q = it % PK_SLOTS;
+          const uint32_t ph = (it / PK_SLOTS) & 1u;
+          if (!mbar_wait(smem_u32(&bars->empty_pk[q]), ph ^ 1u, abort_flag)) { ok = false; break; }
+          const uint32_t pbar = smem_u32(&bars->full_pk[q]);
+          if (!TRANS) {
+            mbar_arrive_expect_tx(pbar, 128 * 32);
+            tma_load_2d(smem_u32(sm.pk[q]), &tmap_pk, pbar,
+                        BITS == 3 ? 6 * kb - 2 * (kb & 1) : 8 * kb, w0);
+          } else {
+            mbar_arrive_expect_tx(pbar, 64 * 16 * BITS);
+            tma_load_2d(smem_u32(sm.pk[q]), &tmap_pk, pbar, (w0 >> 5) * BITS, kb * BK);
+          }
         }
       }
     }
@@ -339,17 +356,21 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmap_act,
         u0 = u1;
         if (it + 2 < total_it) u1 = load_next();
         if (PKTMA) {
-          // the codes landing implies that the producer saw this stage released
-          if (!mbar_wait(smem_u32(&bars->full_pk[s]), ph, abort_flag)) break;
-          const uint32_t* src = reinterpret_cast<const uint32_t*>(sm.pk[s]) + crow * (4 * BITS) + u4 * BITS;
+          const int pq = it % PK_SLOTS;
+          if (!mbar_wait(smem_u32(&bars->full_pk[pq]), (it / PK_SLOTS) & 1u, abort_flag)) break;
+          const uint32_t* src = reinterpret_cast<const uint32_t*>(sm.pk[pq]) + crow * (4 * BITS) + u4 * BITS;
 #pragma unroll
           for (int q = 0; q < BITS; ++q) cur.w[q] = src[q];
-        } else {
-          if (!mbar_wait(smem_u32(&bars->empty[s]), ph ^ 1u, abort_flag)) break;
         }
+        if (!mbar_wait(smem_u32(&bars->empty[s]), ph ^ 1u, abort_flag)) break;
         store_unit<BITS, FOLD>(cur, sm.a[s] + row_off, chunk0, swz);
         fence_proxy_async_smem();
         mbar_arrive(smem_u32(&bars->full_a[s]));
+        if (PKTMA) {
+          // every lane has consumed its codes by now: hand the slot back
+          __syncwarp();
+          if (lane == 0) mbar_arrive(smem_u32(&bars->empty_pk[it % PK_SLOTS]));
+        }
         if (++s == STAGES) { s = 0; ph ^= 1u; }
       }
     } else {
@@ -391,21 +412,28 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmap_act,
           const int s = it % STAGES;
           const uint32_t ph = (it / STAGES) & 1u;
           if (PKTMA) {
-            if (!mbar_wait(smem_u32(&bars->full_pk[s]), ph, abort_flag)) break;
+            const int pq = it % PK_SLOTS;
+            if (!mbar_wait(smem_u32(&bars->full_pk[pq]), (it / PK_SLOTS) & 1u, abort_flag)) break;
             const int woff = (BITS == 3 ? 2 * (kb & 1) : 0) + (u4 & 1) * BITS;
-            const uint32_t* src = reinterpret_cast<const uint32_t*>(sm.pk[s]) + woff;
+            const uint32_t* src = reinterpret_cast<const uint32_t*>(sm.pk[pq]) + woff;
 #pragma unroll
             for (int e = 0; e < BITS; ++e) {
               a0.w[e] = src[rowA * 8 + e];
               b0.w[e] = src[(rowA + 8) * 8 + e];
             }
-          } else {
-            if (!mbar_wait(smem_u32(&bars->empty[s]), ph ^ 1u, abort_flag)) break;
           }
+          if (!mbar_wait(smem_u32(&bars->empty[s]), ph ^ 1u, abort_flag)) break;
           store_unit<BITS, FOLD>(a0, sm.a[s] + rowA * 128, chunk0, swz);
           store_unit<BITS, FOLD>(b0, sm.a[s] + (rowA + 8) * 128, chunk0, swz);
           fence_proxy_async_smem();
           mbar_arrive(smem_u32(&bars->full_a[s]));
+        }
+        if (PKTMA) {
+          // lanes 0-15 served the even k-block's slot, lanes 16-31 the odd one; once the
+          // whole warp has consumed its codes, one lane of each half hands its slot back
+          __syncwarp();
+          if ((lane & 15) == 0 && kb < p.k_blocks)
+            mbar_arrive(smem_u32(&bars->empty_pk[(it_base + (uint32_t)kb) % PK_SLOTS]));
         }
         a0 = a1;
         b0 = b1;
