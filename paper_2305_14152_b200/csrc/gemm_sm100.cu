@@ -179,13 +179,13 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmap_act,
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
-      mbar_init(smem_u32(&bars->full_a[s]), TRANS ? kDequantThreads : kDequantThreads / 2);
+      mbar_init(smem_u32(&bars->full_a[s]), kDequantThreads / 2);   // one group of four dequant warps
       mbar_init(smem_u32(&bars->full_b[s]), 1);
       mbar_init(smem_u32(&bars->empty[s]), 1);
     }
     for (int q = 0; q < PK_SLOTS; ++q) {
       mbar_init(smem_u32(&bars->full_pk[q]), 1);
-      mbar_init(smem_u32(&bars->empty_pk[q]), kDequantThreads / 32);
+      mbar_init(smem_u32(&bars->empty_pk[q]), kDequantThreads / 64);    // the four warps of one group
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(smem_u32(&bars->acc_full[b]), 1);
@@ -319,126 +319,90 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmap_act,
     }
   } else if (warp >= 8) {
     // ------------------------------------------------------- weight dequant
-    // Lane mapping: 8 weight rows x 4 units of 32 columns per warp instruction,
-    // so the four lanes of a row read one contiguous 48/64-byte run of packed
-    // words and share their (s, z) address.
+    // Two groups of four warps alternate stages, so that one group's wait -> read ->
+    // convert -> store -> signal chain overlaps the other group's; a thread converts
+    // two units (2 x 32 columns) of its group's stage.
     const int dw = warp - 8;
-    const int row8 = lane & 7;
-    const int u4 = lane >> 3;
+    const int grp = dw >> 2;
+    const int gw = dw & 3;
     const int my_tiles = (total_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
-    if constexpr (TRANS) {
-      // dX: a stage is 64 weight rows (contraction) x 128 columns = 4 units per row;
-      // every thread owns one unit of every stage.
-      const int crow = dw * 8 + row8;
-      const int row_off = (u4 >> 1) * (64 * 128) + crow * 128;
-      const int chunk0 = (u4 & 1) * 4;
-      const int swz = crow & 7;
-      const uint32_t total_it = (uint32_t)my_tiles * (uint32_t)p.k_blocks;
-      // (tile, k-block) of the unit being prefetched, advanced without divisions
-      int pf_tile = blockIdx.x, pf_kb = 0;
-      int pf_r0 = (pf_tile % p.r_tiles) * BM;
-      auto load_next = [&]() {
-        Unit<BITS> u = load_unit<BITS, !PKTMA>(p, pf_kb * BK + crow, pf_r0 + 32 * u4);
-        if (++pf_kb == p.k_blocks) {
-          pf_kb = 0;
-          pf_tile += gridDim.x;
-          pf_r0 = (pf_tile % p.r_tiles) * BM;
-        }
-        return u;
-      };
-      Unit<BITS> u0, u1;
-      if (total_it > 0) u0 = load_next();
-      if (total_it > 1) u1 = load_next();
-      int s = 0;
-      uint32_t ph = 0;
-      for (uint32_t it = 0; it < total_it; ++it) {
-        Unit<BITS> cur = u0;
-        u0 = u1;
-        if (it + 2 < total_it) u1 = load_next();
-        if (PKTMA) {
-          const int pq = it % PK_SLOTS;
-          if (!mbar_wait(smem_u32(&bars->full_pk[pq]), (it / PK_SLOTS) & 1u, abort_flag)) break;
-          const uint32_t* src = reinterpret_cast<const uint32_t*>(sm.pk[pq]) + crow * (4 * BITS) + u4 * BITS;
-#pragma unroll
-          for (int q = 0; q < BITS; ++q) cur.w[q] = src[q];
-        }
-        if (!mbar_wait(smem_u32(&bars->empty[s]), ph ^ 1u, abort_flag)) break;
-        store_unit<BITS, FOLD>(cur, sm.a[s] + row_off, chunk0, swz);
-        fence_proxy_async_smem();
-        mbar_arrive(smem_u32(&bars->full_a[s]));
-        if (PKTMA) {
-          // every lane has consumed its codes by now: hand the slot back
-          __syncwarp();
-          if (lane == 0) mbar_arrive(smem_u32(&bars->empty_pk[it % PK_SLOTS]));
-        }
-        if (++s == STAGES) { s = 0; ph ^= 1u; }
-      }
+    const uint32_t total_it = (uint32_t)my_tiles * (uint32_t)p.k_blocks;
+    // forward: thread = weight row (gw*32 + lane) of the 128-row tile, units = the two
+    //          32-column halves of the 64-column stage;
+    // dX:      stage = 64 weight rows x 128 columns; lanes = 8 rows x 4 units, the
+    //          thread's second unit is the same columns 32 rows further down.
+    int rowl[2], chunk0[2], row_off[2];
+    if constexpr (!TRANS) {
+      const int row = gw * 32 + lane;
+      rowl[0] = rowl[1] = row;
+      chunk0[0] = 0; chunk0[1] = 4;
+      row_off[0] = row_off[1] = row * 128;
     } else {
-      // forward: a stage is 128 weight rows x 64 columns = 2 units per row, so the
-      // threads walk pairs of stages (128 columns): units 0,1 belong to the even
-      // k-block of the pair, units 2,3 to the odd one, and each thread owns two
-      // rows (r, r + 8) of one k-block.
-      const int half = u4 >> 1;
-      const int rowA = dw * 16 + row8;
-      const int chunk0 = (u4 & 1) * 4;
-      const int swz = row8;               // (rowA & 7) == ((rowA + 8) & 7) == row8
-      const int pairs = (p.k_blocks + 1) / 2;
-      const uint32_t total_pairs = (uint32_t)my_tiles * (uint32_t)pairs;
-      // prefetch cursor (one pair of k-blocks ahead), advanced without divisions
-      int pf_tile = blockIdx.x, pf_pair = 0;
-      int pf_r0 = (pf_tile % p.r_tiles) * BM;
-      auto load_next = [&](Unit<BITS>& a, Unit<BITS>& b) {
-        const int kb = 2 * pf_pair + half;
-        if (kb < p.k_blocks) {
-          const int col0 = kb * BK + 32 * (u4 & 1);
-          a = load_unit<BITS, !PKTMA>(p, pf_r0 + rowA, col0);
-          b = load_unit<BITS, !PKTMA>(p, pf_r0 + rowA + 8, col0);
-        }
-        if (++pf_pair == pairs) {
-          pf_pair = 0;
-          pf_tile += gridDim.x;
-          pf_r0 = (pf_tile % p.r_tiles) * BM;
-        }
-      };
-      Unit<BITS> a0, b0, a1, b1;
-      if (total_pairs > 0) load_next(a0, b0);
-      int cur_pair = 0;
-      uint32_t it_base = 0;               // stage counter of k-block 0 of the current tile
-      for (uint32_t q = 0; q < total_pairs; ++q) {
-        if (q + 1 < total_pairs) load_next(a1, b1);
-        const int kb = 2 * cur_pair + half;
-        if (kb < p.k_blocks) {
-          const uint32_t it = it_base + (uint32_t)kb;
-          const int s = it % STAGES;
-          const uint32_t ph = (it / STAGES) & 1u;
-          if (PKTMA) {
-            const int pq = it % PK_SLOTS;
-            if (!mbar_wait(smem_u32(&bars->full_pk[pq]), (it / PK_SLOTS) & 1u, abort_flag)) break;
-            const int woff = (BITS == 3 ? 2 * (kb & 1) : 0) + (u4 & 1) * BITS;
-            const uint32_t* src = reinterpret_cast<const uint32_t*>(sm.pk[pq]) + woff;
-#pragma unroll
-            for (int e = 0; e < BITS; ++e) {
-              a0.w[e] = src[rowA * 8 + e];
-              b0.w[e] = src[(rowA + 8) * 8 + e];
-            }
-          }
-          if (!mbar_wait(smem_u32(&bars->empty[s]), ph ^ 1u, abort_flag)) break;
-          store_unit<BITS, FOLD>(a0, sm.a[s] + rowA * 128, chunk0, swz);
-          store_unit<BITS, FOLD>(b0, sm.a[s] + (rowA + 8) * 128, chunk0, swz);
-          fence_proxy_async_smem();
-          mbar_arrive(smem_u32(&bars->full_a[s]));
-        }
-        if (PKTMA) {
-          // lanes 0-15 served the even k-block's slot, lanes 16-31 the odd one; once the
-          // whole warp has consumed its codes, one lane of each half hands its slot back
-          __syncwarp();
-          if ((lane & 15) == 0 && kb < p.k_blocks)
-            mbar_arrive(smem_u32(&bars->empty_pk[(it_base + (uint32_t)kb) % PK_SLOTS]));
-        }
-        a0 = a1;
-        b0 = b1;
-        if (++cur_pair == pairs) { cur_pair = 0; it_base += (uint32_t)p.k_blocks; }
+      const int row8 = lane & 7, u4 = lane >> 3;
+      rowl[0] = gw * 8 + row8;
+      rowl[1] = rowl[0] + 32;
+      chunk0[0] = chunk0[1] = (u4 & 1) * 4;
+      row_off[0] = (u4 >> 1) * (64 * 128) + rowl[0] * 128;
+      row_off[1] = (u4 >> 1) * (64 * 128) + rowl[1] * 128;
+    }
+    const int swz = rowl[0] & 7;            // rowl[1] differs by a multiple of 8
+    const int u4 = lane >> 3;
+    // cursor of the stage being prefetched (this group's next stage), no divisions
+    int pf_tile = blockIdx.x, pf_kb = grp;
+    while (pf_kb >= p.k_blocks) { pf_kb -= p.k_blocks; pf_tile += gridDim.x; }
+    int pf_w0 = (pf_tile % p.r_tiles) * BM;
+    auto load_next = [&](Unit<BITS>& a, Unit<BITS>& b) {
+      if constexpr (!TRANS) {
+        a = load_unit<BITS, !PKTMA>(p, pf_w0 + rowl[0], pf_kb * BK);
+        b = load_unit<BITS, !PKTMA>(p, pf_w0 + rowl[1], pf_kb * BK + 32);
+      } else {
+        a = load_unit<BITS, !PKTMA>(p, pf_kb * BK + rowl[0], pf_w0 + 32 * u4);
+        b = load_unit<BITS, !PKTMA>(p, pf_kb * BK + rowl[1], pf_w0 + 32 * u4);
       }
+      pf_kb += 2;
+      while (pf_kb >= p.k_blocks) {
+        pf_kb -= p.k_blocks;
+        pf_tile += gridDim.x;
+        pf_w0 = (pf_tile % p.r_tiles) * BM;
+      }
+    };
+    Unit<BITS> a0, b0, a1, b1;
+    int cur_kb = pf_kb;                      // k-block of the stage about to be processed
+    if ((uint32_t)grp < total_it) load_next(a0, b0);
+    for (uint32_t it = grp; it < total_it; it += 2) {
+      const int next_kb = pf_kb;
+      if (it + 2 < total_it) load_next(a1, b1);
+      const int s = it % STAGES;
+      const uint32_t ph = (it / STAGES) & 1u;
+      if (PKTMA) {
+        const int pq = it % PK_SLOTS;
+        if (!mbar_wait(smem_u32(&bars->full_pk[pq]), (it / PK_SLOTS) & 1u, abort_flag)) break;
+        const uint32_t* src = reinterpret_cast<const uint32_t*>(sm.pk[pq]);
+        if constexpr (!TRANS) {
+          const uint32_t* r = src + rowl[0] * 8 + (BITS == 3 ? 2 * (cur_kb & 1) : 0);
+#pragma unroll
+          for (int e = 0; e < BITS; ++e) { a0.w[e] = r[e]; b0.w[e] = r[BITS + e]; }
+        } else {
+#pragma unroll
+          for (int e = 0; e < BITS; ++e) {
+            a0.w[e] = src[rowl[0] * (4 * BITS) + u4 * BITS + e];
+            b0.w[e] = src[rowl[1] * (4 * BITS) + u4 * BITS + e];
+          }
+        }
+      }
+      if (!mbar_wait(smem_u32(&bars->empty[s]), ph ^ 1u, abort_flag)) break;
+      store_unit<BITS, FOLD>(a0, sm.a[s] + row_off[0], chunk0[0], swz);
+      store_unit<BITS, FOLD>(b0, sm.a[s] + row_off[1], chunk0[1], swz);
+      fence_proxy_async_smem();
+      mbar_arrive(smem_u32(&bars->full_a[s]));
+      if (PKTMA) {
+        // every lane has consumed its codes by now: hand the slot back
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&bars->empty_pk[it % PK_SLOTS]));
+      }
+      a0 = a1;
+      b0 = b1;
+      cur_kb = next_kb;
     }
   }
 
