@@ -53,6 +53,7 @@ constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + PK_SLOTS * PK_BYTES + 1024 /*a
 
 constexpr int kQgemmThreads = 512;     // warps: 0 TMA, 1 MMA, 2 TMEM alloc, 4-7 epilogue, 8-15 dequant
 constexpr int kDequantThreads = 256;
+constexpr int DQ_GROUPS = 4;           // dequant warp groups that take the stages round-robin
 constexpr int kDsThreads = 384;        // warps: 0 TMA, 1 MMA, 2 TMEM alloc, 4-11 epilogue
 
 struct Barriers {
@@ -179,13 +180,13 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmap_act,
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
-      mbar_init(smem_u32(&bars->full_a[s]), kDequantThreads / 2);   // one group of four dequant warps
+      mbar_init(smem_u32(&bars->full_a[s]), kDequantThreads / DQ_GROUPS);   // the threads of one dequant group
       mbar_init(smem_u32(&bars->full_b[s]), 1);
       mbar_init(smem_u32(&bars->empty[s]), 1);
     }
     for (int q = 0; q < PK_SLOTS; ++q) {
       mbar_init(smem_u32(&bars->full_pk[q]), 1);
-      mbar_init(smem_u32(&bars->empty_pk[q]), kDequantThreads / 64);    // the four warps of one group
+      mbar_init(smem_u32(&bars->empty_pk[q]), (kDequantThreads / 32) / DQ_GROUPS);   // the warps of one group
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(smem_u32(&bars->acc_full[b]), 1);
@@ -319,89 +320,97 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmap_act,
     }
   } else if (warp >= 8) {
     // ------------------------------------------------------- weight dequant
-    // Two groups of four warps alternate stages, so that one group's wait -> read ->
-    // convert -> store -> signal chain overlaps the other group's; a thread converts
-    // two units (2 x 32 columns) of its group's stage.
+    // DQ_GROUPS groups of warps take the stages round-robin, so that one group's
+    // wait -> read -> convert -> store -> signal chain overlaps the other groups';
+    // a thread converts UPT units (32 columns each) of its group's stage, all of
+    // them into registers before it waits for the stage buffer to be released.
+    constexpr int UPT = DQ_GROUPS;                      // 256 units per stage / threads per group
+    constexpr int GW = (kDequantThreads / 32) / DQ_GROUPS;   // warps per group
     const int dw = warp - 8;
-    const int grp = dw >> 2;
-    const int gw = dw & 3;
+    const int grp = dw / GW;
+    const int gw = dw % GW;
     const int my_tiles = (total_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
     const uint32_t total_it = (uint32_t)my_tiles * (uint32_t)p.k_blocks;
-    // forward: thread = weight row (gw*32 + lane) of the 128-row tile, units = the two
-    //          32-column halves of the 64-column stage;
-    // dX:      stage = 64 weight rows x 128 columns; lanes = 8 rows x 4 units, the
-    //          thread's second unit is the same columns 32 rows further down.
-    int rowl[2], chunk0[2], row_off[2];
-    if constexpr (!TRANS) {
-      const int row = gw * 32 + lane;
-      rowl[0] = rowl[1] = row;
-      chunk0[0] = 0; chunk0[1] = 4;
-      row_off[0] = row_off[1] = row * 128;
-    } else {
-      const int row8 = lane & 7, u4 = lane >> 3;
-      rowl[0] = gw * 8 + row8;
-      rowl[1] = rowl[0] + 32;
-      chunk0[0] = chunk0[1] = (u4 & 1) * 4;
-      row_off[0] = (u4 >> 1) * (64 * 128) + rowl[0] * 128;
-      row_off[1] = (u4 >> 1) * (64 * 128) + rowl[1] * 128;
-    }
-    const int swz = rowl[0] & 7;            // rowl[1] differs by a multiple of 8
+    // forward: stage = 128 weight rows x 2 units; lanes = 32 consecutive rows; the
+    //          thread's units are (row, 0), (row, 1), (row + 32*GW, 0), ...
+    // dX:      stage = 64 weight rows x 4 units; lanes = 8 rows x 4 units; further
+    //          units of the thread are the same columns 8*GW rows further down.
     const int u4 = lane >> 3;
+    int rowl[UPT], col_off[UPT], chunk0[UPT], row_off[UPT];
+#pragma unroll
+    for (int k = 0; k < UPT; ++k) {
+      if constexpr (!TRANS) {
+        rowl[k] = gw * 32 + lane + (k >> 1) * (32 * GW);
+        col_off[k] = 32 * (k & 1);
+        chunk0[k] = 4 * (k & 1);
+        row_off[k] = rowl[k] * 128;
+      } else {
+        rowl[k] = gw * 8 + (lane & 7) + k * (8 * GW);
+        col_off[k] = 32 * u4;
+        chunk0[k] = (u4 & 1) * 4;
+        row_off[k] = (u4 >> 1) * (64 * 128) + rowl[k] * 128;
+      }
+    }
+    const int swz = rowl[0] & 7;            // all rows of a thread agree modulo 8
     // cursor of the stage being prefetched (this group's next stage), no divisions
     int pf_tile = blockIdx.x, pf_kb = grp;
     while (pf_kb >= p.k_blocks) { pf_kb -= p.k_blocks; pf_tile += gridDim.x; }
     int pf_w0 = (pf_tile % p.r_tiles) * BM;
-    auto load_next = [&](Unit<BITS>& a, Unit<BITS>& b) {
-      if constexpr (!TRANS) {
-        a = load_unit<BITS, !PKTMA>(p, pf_w0 + rowl[0], pf_kb * BK);
-        b = load_unit<BITS, !PKTMA>(p, pf_w0 + rowl[1], pf_kb * BK + 32);
-      } else {
-        a = load_unit<BITS, !PKTMA>(p, pf_kb * BK + rowl[0], pf_w0 + 32 * u4);
-        b = load_unit<BITS, !PKTMA>(p, pf_kb * BK + rowl[1], pf_w0 + 32 * u4);
+    auto load_next = [&](Unit<BITS> (&u)[UPT]) {
+#pragma unroll
+      for (int k = 0; k < UPT; ++k) {
+        if constexpr (!TRANS) u[k] = load_unit<BITS, !PKTMA>(p, pf_w0 + rowl[k], pf_kb * BK + col_off[k]);
+        else u[k] = load_unit<BITS, !PKTMA>(p, pf_kb * BK + rowl[k], pf_w0 + col_off[k]);
       }
-      pf_kb += 2;
+      pf_kb += DQ_GROUPS;
       while (pf_kb >= p.k_blocks) {
         pf_kb -= p.k_blocks;
         pf_tile += gridDim.x;
         pf_w0 = (pf_tile % p.r_tiles) * BM;
       }
     };
-    Unit<BITS> a0, b0, a1, b1;
+    Unit<BITS> cur[UPT], nxt[UPT];
     int cur_kb = pf_kb;                      // k-block of the stage about to be processed
-    if ((uint32_t)grp < total_it) load_next(a0, b0);
-    for (uint32_t it = grp; it < total_it; it += 2) {
+    if ((uint32_t)grp < total_it) load_next(cur);
+    for (uint32_t it = grp; it < total_it; it += DQ_GROUPS) {
       const int next_kb = pf_kb;
-      if (it + 2 < total_it) load_next(a1, b1);
+      if (it + DQ_GROUPS < total_it) load_next(nxt);
       const int s = it % STAGES;
       const uint32_t ph = (it / STAGES) & 1u;
       if (PKTMA) {
         const int pq = it % PK_SLOTS;
         if (!mbar_wait(smem_u32(&bars->full_pk[pq]), (it / PK_SLOTS) & 1u, abort_flag)) break;
         const uint32_t* src = reinterpret_cast<const uint32_t*>(sm.pk[pq]);
-        if constexpr (!TRANS) {
-          const uint32_t* r = src + rowl[0] * 8 + (BITS == 3 ? 2 * (cur_kb & 1) : 0);
 #pragma unroll
-          for (int e = 0; e < BITS; ++e) { a0.w[e] = r[e]; b0.w[e] = r[BITS + e]; }
-        } else {
+        for (int k = 0; k < UPT; ++k) {
+          const uint32_t* r;
+          if constexpr (!TRANS) r = src + rowl[k] * 8 + (BITS == 3 ? 2 * (cur_kb & 1) : 0) + (k & 1) * BITS;
+          else r = src + rowl[k] * (4 * BITS) + u4 * BITS;
 #pragma unroll
-          for (int e = 0; e < BITS; ++e) {
-            a0.w[e] = src[rowl[0] * (4 * BITS) + u4 * BITS + e];
-            b0.w[e] = src[rowl[1] * (4 * BITS) + u4 * BITS + e];
-          }
+          for (int e = 0; e < BITS; ++e) cur[k].w[e] = r[e];
         }
       }
-      if (!mbar_wait(smem_u32(&bars->empty[s]), ph ^ 1u, abort_flag)) break;
-      store_unit<BITS, FOLD>(a0, sm.a[s] + row_off[0], chunk0[0], swz);
-      store_unit<BITS, FOLD>(b0, sm.a[s] + row_off[1], chunk0[1], swz);
-      fence_proxy_async_smem();
-      mbar_arrive(smem_u32(&bars->full_a[s]));
+      uint32_t o[UPT][16];
+#pragma unroll
+      for (int k = 0; k < UPT; ++k) dq::unit32_natural<BITS, FOLD>(cur[k].w, cur[k].z, cur[k].s, o[k]);
       if (PKTMA) {
         // every lane has consumed its codes by now: hand the slot back
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&bars->empty_pk[it % PK_SLOTS]));
       }
-      a0 = a1;
-      b0 = b1;
+      if (!mbar_wait(smem_u32(&bars->empty[s]), ph ^ 1u, abort_flag)) break;
+#pragma unroll
+      for (int k = 0; k < UPT; ++k) {
+        uint8_t* row_ptr = sm.a[s] + row_off[k];
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+          *reinterpret_cast<uint4*>(row_ptr + (((chunk0[k] + q) ^ swz) << 4)) =
+              make_uint4(o[k][4 * q], o[k][4 * q + 1], o[k][4 * q + 2], o[k][4 * q + 3]);
+      }
+      fence_proxy_async_smem();
+      mbar_arrive(smem_u32(&bars->full_a[s]));
+#pragma unroll
+      for (int k = 0; k < UPT; ++k) cur[k] = nxt[k];
       cur_kb = next_kb;
     }
   }
