@@ -381,13 +381,34 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmap_act,
         const int pq = it % PK_SLOTS;
         if (!mbar_wait(smem_u32(&bars->full_pk[pq]), (it / PK_SLOTS) & 1u, abort_flag)) break;
         const uint32_t* src = reinterpret_cast<const uint32_t*>(sm.pk[pq]);
+        if constexpr (!TRANS) {
+          // a row of the slot is 32 bytes: read it whole with two 16-byte loads (consecutive
+          // lanes are consecutive rows, so narrower loads would pile onto four banks) and
+          // pick this stage's words: 4-bit uses all eight, 3-bit six starting at word 0 or 2
 #pragma unroll
-        for (int k = 0; k < UPT; ++k) {
-          const uint32_t* r;
-          if constexpr (!TRANS) r = src + rowl[k] * 8 + (BITS == 3 ? 2 * (cur_kb & 1) : 0) + (k & 1) * BITS;
-          else r = src + rowl[k] * (4 * BITS) + u4 * BITS;
+          for (int k = 0; k < UPT; k += 2) {
+            const uint4 lo = *reinterpret_cast<const uint4*>(src + rowl[k] * 8);
+            const uint4 hi = *reinterpret_cast<const uint4*>(src + rowl[k] * 8 + 4);
+            const uint32_t w8[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
+            if constexpr (BITS == 4) {
 #pragma unroll
-          for (int e = 0; e < BITS; ++e) cur[k].w[e] = r[e];
+              for (int e = 0; e < 4; ++e) { cur[k].w[e] = w8[e]; cur[k + 1].w[e] = w8[4 + e]; }
+            } else {
+              const bool odd = (cur_kb & 1) != 0;
+#pragma unroll
+              for (int e = 0; e < 3; ++e) {
+                cur[k].w[e] = odd ? w8[2 + e] : w8[e];
+                cur[k + 1].w[e] = odd ? w8[5 + e] : w8[3 + e];
+              }
+            }
+          }
+        } else {
+#pragma unroll
+          for (int k = 0; k < UPT; ++k) {
+            const uint32_t* r = src + rowl[k] * (4 * BITS) + u4 * BITS;
+#pragma unroll
+            for (int e = 0; e < BITS; ++e) cur[k].w[e] = r[e];
+          }
         }
       }
       uint32_t o[UPT][16];
