@@ -792,6 +792,7 @@ int ds_piece(int g) { return gcd_int(g, 128); }
 }  // namespace
 
 int launch_fwd(const peqa_qweight_t* w, int g, const void* X, int T, void* Y, cudaStream_t st) {
+  if (fwd_pair_supported(w)) return launch_fwd_pair(w, g, X, T, Y, st);
   return launch_qgemm(w, g, X, T, Y, false, st);
 }
 
