@@ -43,7 +43,7 @@ constexpr int P_ACC_COL = 0;
 constexpr int P_A_COL = 256;
 constexpr int P_SMEM_BYTES = PSTAGES * (PB_BYTES + PQ_BYTES) + 1024 + 512;
 constexpr int P_GROUPS = 4;        // dequant groups (four warps each)
-constexpr int kPairThreads = 768;  // warps: 0 act TMA, 1 MMA, 2 TMEM alloc, 3 code TMA, 4-7 epilogue, 8-23 dequant
+constexpr int kPairThreads = 896;  // warps: 0 act TMA, 1 MMA, 2 TMEM alloc, 3 code TMA, 4-7 and 24-27 epilogue, 8-23 dequant
 
 struct PairBarriers {
   uint64_t full_a[PSTAGES];     // leader: weight stage written to tensor memory by both CTAs
@@ -95,7 +95,7 @@ qfwd_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
       mbar_init(smem_u32(&bars->pk_empty[s]), 4);         // 4 warps of the owning group
     }
     mbar_init(smem_u32(&bars->acc_full), 1);
-    mbar_init(smem_u32(&bars->acc_empty), 8);             // 4 epilogue warps in each CTA
+    mbar_init(smem_u32(&bars->acc_empty), 16);            // 8 epilogue warps in each CTA
     bars->abort_flag = 0;
     fence_mbar_init();
     prefetch_tmap(&tmap_x);
@@ -182,9 +182,12 @@ qfwd_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         if (ok) mma_commit_pair(smem_u32(&bars->acc_full), 3);
       }
     }
-  } else if (warp >= 4 && warp < 8) {
+  } else if ((warp >= 4 && warp < 8) || warp >= 24) {
     // ------------------------------------------ epilogue (lane = output channel)
-    const int ew = warp - 4;
+    // Two warps per TMEM lane quarter: warps 4-7 take tokens [0,128) of the tile,
+    // warps 24-27 tokens [128,256).
+    const int ew = warp & 3;
+    const int thalf = warp >= 24 ? 1 : 0;
     const uint32_t acc_empty_leader = mapa_shared(smem_u32(&bars->acc_empty), 0);
     int local = 0;
     bool ok = true;
@@ -197,7 +200,7 @@ qfwd_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
       float scale = 1.0f;
       if (!FOLD && r < p.N) scale = __ldg(p.scales + r);
 #pragma unroll 1
-      for (int cc = 0; cc < PN / 32; ++cc) {
+      for (int cc = thalf * (PN / 64); cc < (thalf + 1) * (PN / 64); ++cc) {
         const int tc0 = t0 + cc * 32;
         if (tc0 >= p.T) break;
         uint32_t v[32];
@@ -215,7 +218,7 @@ qfwd_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(acc_empty_leader);
     }
-  } else if (warp >= 8) {
+  } else if (warp >= 8 && warp < 24) {
     // ------------------------------------------ weight dequant -> tensor memory
     // Group g (four warps) serves the stages with it % 4 == g.  Warp (w % 4) owns TMEM
     // lanes 32*(w % 4)..+31, so a thread is one output channel; it converts the 64

@@ -166,7 +166,16 @@ __device__ __forceinline__ uint32_t mapa_shared(uint32_t addr, uint32_t rank) {
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
   return r;
 }
+// Arrive on a barrier that may live in the peer CTA (address from mapa_shared).
+// What these arrives publish is tensor-memory state, which tcgen05.fence orders,
+// so the default (CTA-scope release) form is used: a cluster-scope release on
+// every arrive costs well over a thousand cycles.
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// Same, with cluster-scope release: for arrives that publish shared-memory data
+// to a consumer in the peer CTA.
+__device__ __forceinline__ void mbar_arrive_cluster_release(uint32_t cluster_addr) {
   asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr)
                : "memory");
 }
