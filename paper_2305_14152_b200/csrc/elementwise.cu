@@ -41,29 +41,6 @@ __device__ __forceinline__ uint32_t warp_unpack(const uint32_t* src, int lane) {
   return v & ((1u << BITS) - 1u);
 }
 
-// Eight consecutive lanes hold 4 codes each (one 32-column chunk).  Builds the
-// chunk's BITS packed words; lane l8 < BITS of the group returns word l8.
-template <int BITS>
-__device__ __forceinline__ uint32_t group8_pack(uint32_t piece, int lane) {
-  constexpr int NB = 4 * BITS;                 // bits per lane piece: 12 or 16
-  const int l8 = lane & 7;
-  const int base = lane & ~7;
-  const int wbit = 32 * (l8 < BITS ? l8 : 0);  // first bit of the word this lane assembles
-  const int first = wbit / NB;                 // first piece overlapping that word
-  uint32_t word = 0u;
-#pragma unroll
-  for (int k = 0; k < (BITS == 3 ? 4 : 2); ++k) {
-    const int src = first + k;
-    const uint32_t pc = __shfl_sync(0xffffffffu, piece, base + (src & 7));
-    const int sh = src * NB - wbit;            // position of that piece relative to the word
-    if (src < 8) {
-      if (sh >= 0) { if (sh < 32) word |= pc << sh; }
-      else word |= pc >> (-sh);
-    }
-  }
-  return word;
-}
-
 // rint(fl(w / s)) with fl() the correctly rounded binary32 quotient.  The product
 // w * (1/s) is within a few ulps of that quotient, so both round to the same
 // integer unless the product sits within a few ulps of a half-integer; only then
@@ -76,14 +53,16 @@ __device__ __forceinline__ float rint_of_quotient(float w, float s, float rs) {
   return k;
 }
 
-// One CTA per output row; a thread works on float4 vectors so that all loads of
-// a pass are in flight together.  Pass 1: min/max per 32-column chunk (8 lanes).
-// Pass 2: per group (s, z) in strict binary32 (division and rounding as single
-// IEEE operations, no FMA).  Pass 3: codes (second read of the row, served by
-// L2), packed by exchanging 4-code pieces inside each 8-lane group.
+// One CTA per output row; a thread works on runs of 8 consecutive columns, so
+// a 32-column chunk is 4 adjacent lanes.  Pass 1: min/max per chunk.  Pass 2:
+// per group (s, z) in strict binary32 (division and rounding as single IEEE
+// operations, no FMA).  Pass 3: codes (second read of the row, served by L1/L2)
+// and packing: eight 4-bit codes are exactly one word; eight 3-bit codes are 24
+// bits, and lanes 0..2 of a 4-lane chunk assemble the three words from their
+// own and their right neighbour's piece.
 template <int BITS>
 __global__ void __launch_bounds__(kQuantThreads)
-quantize_rtn_kernel(const float* __restrict__ W, int K, int g,
+quantize_rtn_kernel(const float* __restrict__ W, int K, int g, int cpg_shift,
                     uint32_t* __restrict__ qweight, uint8_t* __restrict__ zeros,
                     float* __restrict__ scales) {
   __shared__ float cmin[kMaxChunks];
@@ -94,89 +73,95 @@ quantize_rtn_kernel(const float* __restrict__ W, int K, int g,
   const int row = blockIdx.x;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int chunks = K >> 5;
-  const int nvec = K >> 2;
+  const int nv8 = K >> 3;
   const int G = K / g;
   const int cpg = g >> 5;  // chunks per group
   const float4* w4 = reinterpret_cast<const float4*>(W + (size_t)row * K);
   const float qmax = (float)((1 << BITS) - 1);
-  constexpr int UNROLL = 4;
 
-  // Every thread runs the same number of iterations (the shuffles below name the
-  // whole warp); vectors past the end of the row are predicated off.
-  for (int vb = 0; vb < nvec; vb += kQuantThreads * UNROLL) {
-    const int v0 = vb + threadIdx.x;
-    float4 x[UNROLL];
+  // Every thread runs the same number of iterations (the shuffles name the whole
+  // warp); runs past the end of the row are predicated off.  nv8 is a multiple of 4,
+  // so the 4 lanes of a chunk are all in or all out.
+  for (int vb = 0; vb < nv8; vb += kQuantThreads) {
+    const int v = vb + threadIdx.x;
+    const bool in = v < nv8;
+    float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
+    if (in) { a = __ldg(w4 + 2 * v); b = __ldg(w4 + 2 * v + 1); }
+    float mn = fminf(fminf(fminf(a.x, a.y), fminf(a.z, a.w)), fminf(fminf(b.x, b.y), fminf(b.z, b.w)));
+    float mx = fmaxf(fmaxf(fmaxf(a.x, a.y), fmaxf(a.z, a.w)), fmaxf(fmaxf(b.x, b.y), fmaxf(b.z, b.w)));
 #pragma unroll
-    for (int u = 0; u < UNROLL; ++u) {
-      const int v = v0 + u * kQuantThreads;
-      x[u] = v < nvec ? __ldg(w4 + v) : make_float4(0.f, 0.f, 0.f, 0.f);
-    }
-#pragma unroll
-    for (int u = 0; u < UNROLL; ++u) {
-      const int v = v0 + u * kQuantThreads;   // nvec is a multiple of 8: a group of 8 lanes is all-in or all-out
-      float mn = fminf(fminf(x[u].x, x[u].y), fminf(x[u].z, x[u].w));
-      float mx = fmaxf(fmaxf(x[u].x, x[u].y), fmaxf(x[u].z, x[u].w));
-#pragma unroll
-      for (int o = 4; o > 0; o >>= 1) {
-        mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
-        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-      }
-      if ((lane & 7) == 0 && v < nvec) { cmin[v >> 3] = mn; cmax[v >> 3] = mx; }
-    }
-  }
-  __syncthreads();
-
-  for (int gi = warp; gi < G; gi += kQuantWarps) {
-    float mn = INFINITY, mx = -INFINITY;
-    for (int c = lane; c < cpg; c += 32) {
-      mn = fminf(mn, cmin[gi * cpg + c]);
-      mx = fmaxf(mx, cmax[gi * cpg + c]);
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
+    for (int o = 2; o > 0; o >>= 1) {
       mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
       mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
     }
-    if (lane == 0) {
-      float s = __fdiv_rn(__fsub_rn(mx, mn), qmax);
-      if (mx == mn) s = 1.0f;
-      float z = rintf(__fdiv_rn(-mn, s));
-      z = fminf(fmaxf(z, 0.0f), qmax);
-      gscale[gi] = s;
-      gzero[gi] = z;
-      scales[(size_t)row * G + gi] = s;
-      zeros[(size_t)row * G + gi] = (uint8_t)z;
+    if (in && (lane & 3) == 0) { cmin[v >> 2] = mn; cmax[v >> 2] = mx; }
+  }
+  __syncthreads();
+
+  auto finish_group = [&](int gi, float mn, float mx) {
+    float s = __fdiv_rn(__fsub_rn(mx, mn), qmax);
+    if (mx == mn) s = 1.0f;
+    float z = rintf(__fdiv_rn(-mn, s));
+    z = fminf(fmaxf(z, 0.0f), qmax);
+    gscale[gi] = s;
+    gzero[gi] = z;
+    scales[(size_t)row * G + gi] = s;
+    zeros[(size_t)row * G + gi] = (uint8_t)z;
+  };
+  if (cpg <= 32) {
+    // narrow groups: one thread per group
+    for (int gi = threadIdx.x; gi < G; gi += kQuantThreads) {
+      float mn = INFINITY, mx = -INFINITY;
+      for (int c = 0; c < cpg; ++c) {
+        mn = fminf(mn, cmin[gi * cpg + c]);
+        mx = fmaxf(mx, cmax[gi * cpg + c]);
+      }
+      finish_group(gi, mn, mx);
+    }
+  } else {
+    // wide groups (per-channel above all): one warp per group
+    for (int gi = warp; gi < G; gi += kQuantWarps) {
+      float mn = INFINITY, mx = -INFINITY;
+      for (int c = lane; c < cpg; c += 32) {
+        mn = fminf(mn, cmin[gi * cpg + c]);
+        mx = fmaxf(mx, cmax[gi * cpg + c]);
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+      }
+      if (lane == 0) finish_group(gi, mn, mx);
     }
   }
   __syncthreads();
 
   uint32_t* qrow = qweight + (size_t)row * chunks * BITS;
-  for (int vb = 0; vb < nvec; vb += kQuantThreads * UNROLL) {
-    const int v0 = vb + threadIdx.x;
-    float4 x[UNROLL];
+  for (int vb = 0; vb < nv8; vb += kQuantThreads) {
+    const int v = vb + threadIdx.x;
+    const bool in = v < nv8;
+    float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
+    if (in) { a = __ldg(w4 + 2 * v); b = __ldg(w4 + 2 * v + 1); }
+    const int chunk = in ? (v >> 2) : 0;
+    const int gi = cpg_shift >= 0 ? (chunk >> cpg_shift) : (chunk / cpg);
+    const float s = gscale[gi], z = gzero[gi];
+    const float rs = __frcp_rn(s);
+    const float xs[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+    uint32_t piece = 0u;
 #pragma unroll
-    for (int u = 0; u < UNROLL; ++u) {
-      const int v = v0 + u * kQuantThreads;
-      x[u] = v < nvec ? __ldg(w4 + v) : make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int e = 0; e < 8; ++e) {
+      float q = __fadd_rn(rint_of_quotient(xs[e], s, rs), z);
+      q = fminf(fmaxf(q, 0.0f), qmax);
+      piece |= (uint32_t)q << (BITS * e);
     }
-#pragma unroll
-    for (int u = 0; u < UNROLL; ++u) {
-      const int v = v0 + u * kQuantThreads;
-      const bool in = v < nvec;
-      const int chunk = in ? (v >> 3) : 0;
-      const int gi = chunk / cpg;
-      const float s = gscale[gi], z = gzero[gi];
-      const float rs = __frcp_rn(s);
-      const float xs[4] = {x[u].x, x[u].y, x[u].z, x[u].w};
-      uint32_t piece = 0u;
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        float q = __fadd_rn(rint_of_quotient(xs[e], s, rs), z);
-        q = fminf(fmaxf(q, 0.0f), qmax);
-        piece |= (uint32_t)q << (BITS * e);
-      }
-      const uint32_t word = group8_pack<BITS>(piece, lane);
-      if (in && (lane & 7) < BITS) qrow[chunk * BITS + (lane & 7)] = word;
+    if constexpr (BITS == 4) {
+      if (in) qrow[v] = piece;
+    } else {
+      // chunk = 96 bits = pieces p0..p3 of 24 bits: word j = (p_j >> 8j) | (p_{j+1} << (24 - 8j))
+      const uint32_t nextp = __shfl_down_sync(0xffffffffu, piece, 1);
+      const int j = lane & 3;
+      const uint32_t word = (piece >> (8 * j)) | (nextp << (24 - 8 * j));
+      if (in && j < 3) qrow[chunk * 3 + j] = word;
     }
   }
 }
@@ -245,10 +230,13 @@ extern "C" int peqa_quantize_rtn(const float* W, int N, int K, int bits, int gro
   PEQA_TRY(check_arch());
   const int g = effective_group(K, group_size);
   cudaStream_t st = as_stream(stream);
+  int cpg_shift = -1;
+  for (int b = 0; b < 26; ++b)
+    if ((32 << b) == g) cpg_shift = b;
   if (bits == 4)
-    quantize_rtn_kernel<4><<<N, kQuantThreads, 0, st>>>(W, K, g, qweight, zeros, scales);
+    quantize_rtn_kernel<4><<<N, kQuantThreads, 0, st>>>(W, K, g, cpg_shift, qweight, zeros, scales);
   else
-    quantize_rtn_kernel<3><<<N, kQuantThreads, 0, st>>>(W, K, g, qweight, zeros, scales);
+    quantize_rtn_kernel<3><<<N, kQuantThreads, 0, st>>>(W, K, g, cpg_shift, qweight, zeros, scales);
   PEQA_CUDA(cudaGetLastError());
   return PEQA_OK;
 }
