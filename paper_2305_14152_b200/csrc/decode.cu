@@ -91,16 +91,19 @@ __device__ __forceinline__ void unit_words(const RowChunk<BITS>& r, int u, uint3
 template <int BITS, int BLK, int E, bool FOLD>
 __device__ __forceinline__ void two_pairs(const uint32_t (&w)[BITS], uint32_t zc, uint32_t s2,
                                           uint32_t& p0, uint32_t& p1) {
-  p0 = dq::bf162_sub(dq::pair_raw<BITS, 8 * BLK + E>(w), zc);
-  p1 = dq::bf162_sub(dq::pair_raw<BITS, 8 * BLK + E + 1>(w), zc);
+  // Per-channel layers (!FOLD) feed the biased values (bias + q) straight to the MMA and
+  // take the (bias + z) * sum(x) term out of the result at the end: one operation less
+  // per pair in the loop that decides whether the weight stream can be kept up with.
+  p0 = dq::pair_raw<BITS, 8 * BLK + E>(w);
+  p1 = dq::pair_raw<BITS, 8 * BLK + E + 1>(w);
   if (FOLD) {
-    p0 = dq::bf162_mul(p0, s2);
-    p1 = dq::bf162_mul(p1, s2);
+    p0 = dq::bf162_mul(dq::bf162_sub(p0, zc), s2);
+    p1 = dq::bf162_mul(dq::bf162_sub(p1, zc), s2);
   }
 }
 
 template <int BITS, int NT, bool FOLD>
-__global__ void __launch_bounds__(kDecThreads)
+__global__ void __launch_bounds__(kDecThreads, (NT == 1 && BITS == 3) ? 4 : 3)
 decode_kernel(const DecodeParams p) {
   extern __shared__ __align__(16) uint8_t dec_smem[];
   // layout: [staged activations: M rows of x_pitch bytes][partials: 128 rows x (8*NT) fp32]
@@ -115,6 +118,38 @@ decode_kernel(const DecodeParams p) {
 
   uint8_t* xs = dec_smem;
   float* partial = reinterpret_cast<float*>(dec_smem + (((size_t)p.M * p.x_pitch + 15) & ~(size_t)15));
+
+  // The first weight chunks are requested before anything else: they do not depend on
+  // the activations, so their latency overlaps the staging below.
+  const int row_base = blockIdx.x * kRowsPerCta + warp * kRowsPerWarp;
+  // rows of this lane: fragment rows g and g+8 of the two 16-row blocks
+  int rows[4] = {row_base + g8, row_base + g8 + 8, row_base + 16 + g8, row_base + 24 + g8};
+
+  float acc[2][NT][4];
+#pragma unroll
+  for (int rb = 0; rb < 2; ++rb)
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) acc[rb][nt][e] = 0.0f;
+
+  float z_row[4] = {0.f, 0.f, 0.f, 0.f};   // per-channel zero-points of this lane's rows
+  if (!FOLD) {
+#pragma unroll
+    for (int r = 0; r < 4; ++r)
+      if (rows[r] < p.N) z_row[r] = (float)__ldg(p.zeros + rows[r]);
+  }
+
+  // token rows this lane reads as the MMA "B" operand (token index = lane / 4);
+  // lanes beyond M read row 0: their accumulator columns are never stored.
+  const uint8_t* xrow0 = xs + (size_t)(g8 < p.M ? g8 : 0) * p.x_pitch;
+  const uint8_t* xrow1 = xs + (size_t)(g8 + 8 < p.M ? g8 + 8 : 0) * p.x_pitch;
+
+  RowChunk<BITS> cur[4], nxt[4];
+  if (nsteps > 0) {
+#pragma unroll
+    for (int r = 0; r < 4; ++r) cur[r] = load_chunk<BITS>(p, rows[r], kbeg + c4 * 128);
+  }
 
   // ---- stage the activation slice: blocks of 8 columns stored as (0,4,1,5,2,6,3,7)
   {
@@ -135,36 +170,32 @@ decode_kernel(const DecodeParams p) {
   }
   __syncthreads();
 
-  const int row_base = blockIdx.x * kRowsPerCta + warp * kRowsPerWarp;
-  // rows of this lane: fragment rows g and g+8 of the two 16-row blocks
-  int rows[4] = {row_base + g8, row_base + g8 + 8, row_base + 16 + g8, row_base + 24 + g8};
-
-  float acc[2][NT][4];
-#pragma unroll
-  for (int rb = 0; rb < 2; ++rb)
-#pragma unroll
-    for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-      for (int e = 0; e < 4; ++e) acc[rb][nt][e] = 0.0f;
-
-  uint32_t zc_row[4] = {0u, 0u, 0u, 0u};
+  // Per-channel path: sums of the staged activations over the columns that land in the
+  // low and in the high half of the bf16 pairs (they carry different biases).  In the
+  // staged order every 32-bit word is one (low, high) pair.  Fixed summation order.
+  float* xsum = partial + kRowsPerCta * 8 * NT;   // [2][16]
   if (!FOLD) {
+    for (int m = warp; m < p.M; m += kDecWarps) {
+      const uint8_t* xr = xs + (size_t)m * p.x_pitch;
+      float lo = 0.f, hi = 0.f;
+      for (int blk = 0; blk < nsteps * 4; ++blk) {
+        const uint32_t* wds = reinterpret_cast<const uint32_t*>(xr + blk * kBlockBytes);
 #pragma unroll
-    for (int r = 0; r < 4; ++r)
-      if (rows[r] < p.N) zc_row[r] = dq::zero_const<BITS>(__ldg(p.zeros + rows[r]));
-      else zc_row[r] = dq::zero_const<BITS>(0u);
+        for (int h = 0; h < 2; ++h) {
+          const uint32_t v = wds[lane + 32 * h];
+          lo += __uint_as_float(v << 16);
+          hi += __uint_as_float(v & 0xFFFF0000u);
+        }
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        lo += __shfl_xor_sync(0xffffffffu, lo, o);
+        hi += __shfl_xor_sync(0xffffffffu, hi, o);
+      }
+      if (lane == 0) { xsum[m] = lo; xsum[16 + m] = hi; }
+    }
   }
 
-  // token rows this lane reads as the MMA "B" operand (token index = lane / 4);
-  // lanes beyond M read row 0: their accumulator columns are never stored.
-  const uint8_t* xrow0 = xs + (size_t)(g8 < p.M ? g8 : 0) * p.x_pitch;
-  const uint8_t* xrow1 = xs + (size_t)(g8 + 8 < p.M ? g8 + 8 : 0) * p.x_pitch;
-
-  RowChunk<BITS> cur[4], nxt[4];
-  if (nsteps > 0) {
-#pragma unroll
-    for (int r = 0; r < 4; ++r) cur[r] = load_chunk<BITS>(p, rows[r], kbeg + c4 * 128);
-  }
   for (int st = 0; st < nsteps; ++st) {
     const int col0 = kbeg + st * kStepCols + c4 * 128;   // first column of this lane's chunk
     if (st + 1 < nsteps) {
@@ -191,7 +222,7 @@ decode_kernel(const DecodeParams p) {
           zc[r] = dq::zero_const<BITS>(z);
           s2[r] = dq::bf162_broadcast(s);
         } else {
-          zc[r] = zc_row[r];
+          zc[r] = 0u;
           s2[r] = 0u;
         }
       }
@@ -240,16 +271,29 @@ decode_kernel(const DecodeParams p) {
 
   // ---- partial sums of this CTA: [128 rows][8*NT tokens]
   constexpr int TOK = 8 * NT;
+  if (!FOLD) __syncthreads();   // xsum of every token is written
+  constexpr float kBiasLo = BITS == 4 ? 128.0f : 8.0f;
 #pragma unroll
   for (int rb = 0; rb < 2; ++rb)
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
       const int lr = warp * kRowsPerWarp + rb * 16 + g8;
       const int tk = nt * 8 + c4 * 2;
-      partial[lr * TOK + tk] = acc[rb][nt][0];
-      partial[lr * TOK + tk + 1] = acc[rb][nt][1];
-      partial[(lr + 8) * TOK + tk] = acc[rb][nt][2];
-      partial[(lr + 8) * TOK + tk + 1] = acc[rb][nt][3];
+      float c00 = 0.f, c01 = 0.f, c10 = 0.f, c11 = 0.f;
+      if (!FOLD) {
+        // (bias + z) * sum(x) over this CTA's K slice, per row and token
+        const float lo0 = tk < p.M ? xsum[tk] : 0.f, hi0 = tk < p.M ? xsum[16 + tk] : 0.f;
+        const float lo1 = tk + 1 < p.M ? xsum[tk + 1] : 0.f, hi1 = tk + 1 < p.M ? xsum[16 + tk + 1] : 0.f;
+        const float za = z_row[2 * rb], zb = z_row[2 * rb + 1];
+        c00 = (kBiasLo + za) * lo0 + (128.0f + za) * hi0;
+        c01 = (kBiasLo + za) * lo1 + (128.0f + za) * hi1;
+        c10 = (kBiasLo + zb) * lo0 + (128.0f + zb) * hi0;
+        c11 = (kBiasLo + zb) * lo1 + (128.0f + zb) * hi1;
+      }
+      partial[lr * TOK + tk] = acc[rb][nt][0] - c00;
+      partial[lr * TOK + tk + 1] = acc[rb][nt][1] - c01;
+      partial[(lr + 8) * TOK + tk] = acc[rb][nt][2] - c10;
+      partial[(lr + 8) * TOK + tk + 1] = acc[rb][nt][3] - c11;
     }
 
   // ---- add the K-slices of the cluster in rank order and write Y
@@ -355,7 +399,8 @@ int launch_decode(const peqa_qweight_t* w, int g, const void* X, int M, void* Y,
     // pitch = nblk*288 + pad with pitch % 128 == 8: consecutive tokens land 2 banks apart
     const int pad = ((8 - (nblk * kBlockBytes) % 128) % 128 + 128) % 128;
     p.x_pitch = nblk * kBlockBytes + pad;
-    smem = (((size_t)M * p.x_pitch + 15) & ~(size_t)15) + (size_t)kRowsPerCta * 8 * NT * sizeof(float);
+    smem = (((size_t)M * p.x_pitch + 15) & ~(size_t)15) + (size_t)kRowsPerCta * 8 * NT * sizeof(float) +
+           32 * sizeof(float);   // + the [2][16] activation sums
     if (smem <= 200 * 1024 || split == kMaxSplit) break;
     split *= 2;
   }
