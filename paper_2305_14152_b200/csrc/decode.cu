@@ -20,8 +20,11 @@
 #include <cooperative_groups.h>
 #include <cuda_bf16.h>
 
+#include <cuda.h>
+
 #include "common.cuh"
 #include "dequant.cuh"
+#include "sm100_ptx.cuh"
 
 namespace cg = cooperative_groups;
 
@@ -29,8 +32,11 @@ namespace peqa {
 
 namespace {
 
-constexpr int kDecWarps = 4;
+constexpr int kDecWarps = 4;                            // compute warps
 constexpr int kDecThreads = kDecWarps * 32;
+constexpr int kDecBlock = kDecThreads + 32;             // + one warp that issues the TMA copies
+constexpr int kDecSlots = 2;                            // weight steps in flight per CTA
+constexpr int kDecBoxBytes = 128 * 64;                  // one TMA box: 128 rows x 16 words
 constexpr int kRowsPerWarp = 32;
 constexpr int kRowsPerCta = kDecWarps * kRowsPerWarp;   // 128
 constexpr int kStepCols = 512;                          // columns per warp step (4 lanes x 128)
@@ -48,6 +54,13 @@ struct DecodeParams {
   int total_steps;          // ceil(K / 512)
   int split;                // CTAs per cluster along K
   int x_pitch;              // bytes between token rows of the staged activations
+  int* status;
+};
+
+struct DecBarriers {
+  uint64_t full[kDecSlots];    // weight step landed in its slot
+  uint64_t empty[kDecSlots];   // all compute warps have read the slot
+  int abort_flag;
 };
 
 __device__ __forceinline__ void mma_16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0,
@@ -103,13 +116,20 @@ __device__ __forceinline__ void two_pairs(const uint32_t (&w)[BITS], uint32_t zc
 }
 
 template <int BITS, int NT, bool FOLD>
-__global__ void __launch_bounds__(kDecThreads, (NT == 1 && BITS == 3) ? 4 : 3)
-decode_kernel(const DecodeParams p) {
-  extern __shared__ __align__(16) uint8_t dec_smem[];
-  // layout: [staged activations: M rows of x_pitch bytes][partials: 128 rows x (8*NT) fp32]
+__global__ void __launch_bounds__(kDecBlock, BITS == 3 ? 4 : 3)
+decode_kernel(const __grid_constant__ CUtensorMap tmap_q, const DecodeParams p) {
+  extern __shared__ uint8_t dec_smem_raw[];
+  // layout: [weight slots: kDecSlots x BITS boxes of 8 KiB, 64-byte-swizzled]
+  //         [staged activations: M rows of x_pitch bytes][partials: 128 rows x (8*NT) fp32]
+  //         [activation sums 2 x 16 fp32][barriers]
+  constexpr int kStepBytes = BITS * kDecBoxBytes;     // 512 columns of 128 rows
+  uint8_t* slots = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(dec_smem_raw) + 1023) &
+                                              ~static_cast<uintptr_t>(1023));
+  uint8_t* dec_smem = slots + kDecSlots * kStepBytes;
   const int rank = blockIdx.y;   // position along K inside the cluster
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g8 = lane >> 2, c4 = lane & 3;
+  const bool is_producer = warp == kDecWarps;
 
   const int steps_lo = (int)(((long long)p.total_steps * rank) / p.split);
   const int steps_hi = (int)(((long long)p.total_steps * (rank + 1)) / p.split);
@@ -118,6 +138,30 @@ decode_kernel(const DecodeParams p) {
 
   uint8_t* xs = dec_smem;
   float* partial = reinterpret_cast<float*>(dec_smem + (((size_t)p.M * p.x_pitch + 15) & ~(size_t)15));
+  DecBarriers* bars = reinterpret_cast<DecBarriers*>(partial + kRowsPerCta * 8 * NT + 32);
+  volatile int* abort_flag = &bars->abort_flag;
+
+  // One weight step (128 rows x 512 columns) = BITS boxes of 16 words x 128 rows.
+  auto issue_step = [&](int st) {
+    const int slot = st % kDecSlots;
+    const uint32_t bar = ptx::smem_u32(&bars->full[slot]);
+    ptx::mbar_arrive_expect_tx(bar, kStepBytes);
+#pragma unroll
+    for (int b = 0; b < BITS; ++b)
+      ptx::tma_load_2d(ptx::smem_u32(slots + slot * kStepBytes + b * kDecBoxBytes), &tmap_q, bar,
+                       (steps_lo + st) * (16 * BITS) + 16 * b, blockIdx.x * kRowsPerCta);
+  };
+  if (is_producer && lane == 0) {
+    // The weight copies are requested before anything else: they do not depend on the
+    // activations, so their latency overlaps the staging below.
+    for (int q = 0; q < kDecSlots; ++q) {
+      ptx::mbar_init(ptx::smem_u32(&bars->full[q]), 1);
+      ptx::mbar_init(ptx::smem_u32(&bars->empty[q]), kDecWarps);
+    }
+    bars->abort_flag = 0;
+    ptx::fence_mbar_init();
+    for (int st = 0; st < nsteps && st < kDecSlots; ++st) issue_step(st);
+  }
 
   // The first weight chunks are requested before anything else: they do not depend on
   // the activations, so their latency overlaps the staging below.
@@ -145,16 +189,22 @@ decode_kernel(const DecodeParams p) {
   const uint8_t* xrow0 = xs + (size_t)(g8 < p.M ? g8 : 0) * p.x_pitch;
   const uint8_t* xrow1 = xs + (size_t)(g8 + 8 < p.M ? g8 + 8 : 0) * p.x_pitch;
 
-  RowChunk<BITS> cur[4], nxt[4];
-  if (nsteps > 0) {
+  RowChunk<BITS> cur[4];
+  // Where this lane's 16-byte pieces of a step sit in a slot: word w of the step's row is
+  // in box w/16, 16-byte chunk (w%16)/4, and the 64-byte swizzle XORs the chunk index with
+  // bits 1-2 of the row (equal for the lane's four rows, which differ by multiples of 8).
+  uint32_t piece_off[BITS];
 #pragma unroll
-    for (int r = 0; r < 4; ++r) cur[r] = load_chunk<BITS>(p, rows[r], kbeg + c4 * 128);
+  for (int q = 0; q < BITS; ++q) {
+    const int w = 4 * BITS * c4 + 4 * q;
+    piece_off[q] = (uint32_t)((w >> 4) * kDecBoxBytes + ((((w & 15) >> 2) ^ ((g8 >> 1) & 3)) << 4));
   }
+  const uint32_t row_off0 = (uint32_t)(warp * kRowsPerWarp + g8) * 64u;   // local rows g8, +8, +16, +24
 
   // ---- stage the activation slice: blocks of 8 columns stored as (0,4,1,5,2,6,3,7)
   {
     const int blocks8 = nsteps * (kStepCols / 8);
-    for (int idx = threadIdx.x; idx < p.M * blocks8; idx += kDecThreads) {
+    for (int idx = threadIdx.x; idx < p.M * blocks8; idx += kDecBlock) {
       const int m = idx / blocks8;
       const int b8 = idx - m * blocks8;
       const int col = kbeg + b8 * 8;
@@ -174,7 +224,7 @@ decode_kernel(const DecodeParams p) {
   // low and in the high half of the bf16 pairs (they carry different biases).  In the
   // staged order every 32-bit word is one (low, high) pair.  Fixed summation order.
   float* xsum = partial + kRowsPerCta * 8 * NT;   // [2][16]
-  if (!FOLD) {
+  if (!FOLD && !is_producer) {
     for (int m = warp; m < p.M; m += kDecWarps) {
       const uint8_t* xr = xs + (size_t)m * p.x_pitch;
       float lo = 0.f, hi = 0.f;
@@ -196,11 +246,28 @@ decode_kernel(const DecodeParams p) {
     }
   }
 
+  if (is_producer) {
+    // keep the slots full: step st goes into slot st % kDecSlots once every compute warp
+    // has finished with the step that was there
+    if (lane == 0) {
+      for (int st = kDecSlots; st < nsteps; ++st) {
+        const int slot = st % kDecSlots;
+        if (!ptx::mbar_wait(ptx::smem_u32(&bars->empty[slot]), ((st / kDecSlots) & 1u) ^ 1u, abort_flag)) break;
+        issue_step(st);
+      }
+    }
+  } else
   for (int st = 0; st < nsteps; ++st) {
     const int col0 = kbeg + st * kStepCols + c4 * 128;   // first column of this lane's chunk
-    if (st + 1 < nsteps) {
+    const int slot = st % kDecSlots;
+    if (!ptx::mbar_wait(ptx::smem_u32(&bars->full[slot]), (st / kDecSlots) & 1u, abort_flag)) break;
+    {
+      const uint8_t* sb = slots + slot * kStepBytes + row_off0;
 #pragma unroll
-      for (int r = 0; r < 4; ++r) nxt[r] = load_chunk<BITS>(p, rows[r], col0 + kStepCols);
+      for (int r = 0; r < 4; ++r)
+#pragma unroll
+        for (int q = 0; q < BITS; ++q)
+          cur[r].v[q] = *reinterpret_cast<const uint4*>(sb + r * (8 * 64) + piece_off[q]);
     }
     const int xoff = (st * 4 + c4) * kBlockBytes;
 #pragma unroll
@@ -263,16 +330,16 @@ decode_kernel(const DecodeParams p) {
         }
       }
     }
-    if (st + 1 < nsteps) {
-#pragma unroll
-      for (int r = 0; r < 4; ++r) cur[r] = nxt[r];
-    }
+    // the codes of this step are in registers and consumed: hand the slot back
+    __syncwarp();
+    if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&bars->empty[slot]));
   }
 
   // ---- partial sums of this CTA: [128 rows][8*NT tokens]
   constexpr int TOK = 8 * NT;
   if (!FOLD) __syncthreads();   // xsum of every token is written
   constexpr float kBiasLo = BITS == 4 ? 128.0f : 8.0f;
+  if (!is_producer)
 #pragma unroll
   for (int rb = 0; rb < 2; ++rb)
 #pragma unroll
@@ -301,7 +368,7 @@ decode_kernel(const DecodeParams p) {
   if (p.split > 1) {
     cg::cluster_group cluster = cg::this_cluster();
     cluster.sync();
-    for (int idx = threadIdx.x; idx < rows_per_rank * p.M; idx += kDecThreads) {
+    for (int idx = threadIdx.x; idx < rows_per_rank * p.M; idx += kDecBlock) {
       const int m = idx / rows_per_rank;
       const int lr = rank * rows_per_rank + (idx - m * rows_per_rank);
       const int row = blockIdx.x * kRowsPerCta + lr;
@@ -318,7 +385,7 @@ decode_kernel(const DecodeParams p) {
     cluster.sync();   // keep every CTA's shared memory alive until all ranks have read it
   } else {
     __syncthreads();
-    for (int idx = threadIdx.x; idx < kRowsPerCta * p.M; idx += kDecThreads) {
+    for (int idx = threadIdx.x; idx < kRowsPerCta * p.M; idx += kDecBlock) {
       const int m = idx / kRowsPerCta;
       const int lr = idx - m * kRowsPerCta;
       const int row = blockIdx.x * kRowsPerCta + lr;
@@ -329,6 +396,7 @@ decode_kernel(const DecodeParams p) {
       }
     }
   }
+  if (threadIdx.x == 0 && bars->abort_flag) atomicExch(p.status, (int)PEQA_ERR_DEVICE_TIMEOUT);
 }
 
 int sm_count_cached(int* n) {
@@ -344,12 +412,13 @@ int sm_count_cached(int* n) {
 }
 
 template <int BITS, int NT, bool FOLD>
-int launch_decode_t(const DecodeParams& p, int row_blocks, size_t smem, cudaStream_t st) {
+int launch_decode_t(const CUtensorMap& tmap_q, const DecodeParams& p, int row_blocks, size_t smem,
+                    cudaStream_t st) {
   auto kern = decode_kernel<BITS, NT, FOLD>;
   PEQA_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(row_blocks, p.split, 1);
-  cfg.blockDim = dim3(kDecThreads, 1, 1);
+  cfg.blockDim = dim3(kDecBlock, 1, 1);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
@@ -359,7 +428,7 @@ int launch_decode_t(const DecodeParams& p, int row_blocks, size_t smem, cudaStre
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  PEQA_CUDA(cudaLaunchKernelEx(&cfg, kern, p));
+  PEQA_CUDA(cudaLaunchKernelEx(&cfg, kern, tmap_q, p));
   return PEQA_OK;
 }
 
@@ -399,23 +468,49 @@ int launch_decode(const peqa_qweight_t* w, int g, const void* X, int M, void* Y,
     // pitch = nblk*288 + pad with pitch % 128 == 8: consecutive tokens land 2 banks apart
     const int pad = ((8 - (nblk * kBlockBytes) % 128) % 128 + 128) % 128;
     p.x_pitch = nblk * kBlockBytes + pad;
-    smem = (((size_t)M * p.x_pitch + 15) & ~(size_t)15) + (size_t)kRowsPerCta * 8 * NT * sizeof(float) +
-           32 * sizeof(float);   // + the [2][16] activation sums
+    smem = 1024 /*alignment*/ + (size_t)kDecSlots * w->bits * kDecBoxBytes /*weight slots*/ +
+           (((size_t)M * p.x_pitch + 15) & ~(size_t)15) + (size_t)kRowsPerCta * 8 * NT * sizeof(float) +
+           32 * sizeof(float) /*activation sums*/ + sizeof(DecBarriers) + 16;
     if (smem <= 200 * 1024 || split == kMaxSplit) break;
     split *= 2;
   }
   if (smem > 227 * 1024) return PEQA_ERR_TOO_LARGE;
+  PEQA_TRY(status_word(&p.status));
+  // packed matrix as uint32 [N, wpr]; box = 16 words x 128 rows, 64-byte swizzle
+  CUtensorMap tmap_q;
+  {
+    typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                      const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                      const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                      CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    static EncodeTiledFn enc = nullptr;
+    if (!enc) {
+      void* fn = nullptr;
+      cudaDriverEntryPointQueryResult qres;
+      PEQA_CUDA(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
+      if (!fn || qres != cudaDriverEntryPointSuccess) return cuda_fail(cudaErrorUnknown);
+      enc = reinterpret_cast<EncodeTiledFn>(fn);
+    }
+    cuuint64_t dims[2] = {(cuuint64_t)p.wpr, (cuuint64_t)p.N};
+    cuuint64_t strides[1] = {(cuuint64_t)p.wpr * 4};
+    cuuint32_t box[2] = {16, (cuuint32_t)kRowsPerCta};
+    cuuint32_t estr[2] = {1, 1};
+    if (enc(&tmap_q, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<uint32_t*>(w->qweight), dims,
+            strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return cuda_fail(cudaErrorInvalidValue);
+  }
   const bool fold = p.G > 1;
   if (w->bits == 4) {
-    if (NT == 1) return fold ? launch_decode_t<4, 1, true>(p, row_blocks, smem, st)
-                             : launch_decode_t<4, 1, false>(p, row_blocks, smem, st);
-    return fold ? launch_decode_t<4, 2, true>(p, row_blocks, smem, st)
-                : launch_decode_t<4, 2, false>(p, row_blocks, smem, st);
+    if (NT == 1) return fold ? launch_decode_t<4, 1, true>(tmap_q, p, row_blocks, smem, st)
+                             : launch_decode_t<4, 1, false>(tmap_q, p, row_blocks, smem, st);
+    return fold ? launch_decode_t<4, 2, true>(tmap_q, p, row_blocks, smem, st)
+                : launch_decode_t<4, 2, false>(tmap_q, p, row_blocks, smem, st);
   }
-  if (NT == 1) return fold ? launch_decode_t<3, 1, true>(p, row_blocks, smem, st)
-                           : launch_decode_t<3, 1, false>(p, row_blocks, smem, st);
-  return fold ? launch_decode_t<3, 2, true>(p, row_blocks, smem, st)
-              : launch_decode_t<3, 2, false>(p, row_blocks, smem, st);
+  if (NT == 1) return fold ? launch_decode_t<3, 1, true>(tmap_q, p, row_blocks, smem, st)
+                           : launch_decode_t<3, 1, false>(tmap_q, p, row_blocks, smem, st);
+  return fold ? launch_decode_t<3, 2, true>(tmap_q, p, row_blocks, smem, st)
+              : launch_decode_t<3, 2, false>(tmap_q, p, row_blocks, smem, st);
 }
 
 }  // namespace peqa
