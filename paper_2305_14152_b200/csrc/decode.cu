@@ -154,6 +154,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmap_q, const DecodeParams p) 
   if (is_producer && lane == 0) {
     // The weight copies are requested before anything else: they do not depend on the
     // activations, so their latency overlaps the staging below.
+    ptx::prefetch_tmap(&tmap_q);
     for (int q = 0; q < kDecSlots; ++q) {
       ptx::mbar_init(ptx::smem_u32(&bars->full[q]), 1);
       ptx::mbar_init(ptx::smem_u32(&bars->empty[q]), kDecWarps);
