@@ -59,6 +59,8 @@ inline cudaStream_t as_stream(void* s) { return reinterpret_cast<cudaStream_t>(s
 int launch_fwd(const peqa_qweight_t* w, int g, const void* X, int T, void* Y, cudaStream_t st);
 bool fwd_pair_supported(const peqa_qweight_t* w);
 int launch_fwd_pair(const peqa_qweight_t* w, int g, const void* X, int T, void* Y, cudaStream_t st);
+bool dx_pair_supported(const peqa_qweight_t* w);
+int launch_dx_pair(const peqa_qweight_t* w, int g, const void* dY, int T, void* dX, cudaStream_t st);
 int launch_dx(const peqa_qweight_t* w, int g, const void* dY, int T, void* dX, cudaStream_t st);
 int launch_ds(const peqa_qweight_t* w, int g, const void* X, const void* dY, int T, float* dS,
               void* workspace, size_t workspace_bytes, cudaStream_t st);

@@ -1,0 +1,413 @@
+// Backward with respect to the input, dX = dY * W_hat (chain rule on Eq. 2), on
+// CTA pairs.
+//
+// A pair of CTAs (cta_group::2) owns a tile of 256 tokens x 256 input columns j.
+// The tokens are the MMA "M" side: CTA `rank` TMA-loads its 128 tokens of dY
+// (A operand, K-major: the contraction index i is contiguous in dY) and keeps
+// their accumulator rows.  The weights are the "N" side, split between the two
+// CTAs: each dequantises the 128 columns [j0 + 128*rank, +128) of the stage's
+// 64 weight rows into its own shared memory, MN-major (a row of packed codes is
+// unpacked along j, exactly as it is stored), and the pair's tensor cores read
+// both halves.  Per 64-deep stage a CTA moves 32 KiB into shared memory and its
+// tensor core reads 48 KiB, against 48 + 48 KiB in the single-CTA kernel, and
+// the accumulator is token-major, so every epilogue thread writes contiguous
+// 64-byte runs of dX.
+//
+// Packed codes come through their own TMA ring (one box = 64 weight rows x the
+// CTA's 128 columns); four groups of four dequant warps take the stages
+// round-robin.  Two 256-column accumulators overlap the epilogue of one tile
+// with the main loop of the next.
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include "common.cuh"
+#include "dequant.cuh"
+#include "sm100_ptx.cuh"
+
+namespace peqa {
+
+namespace {
+
+using namespace ptx;
+
+constexpr int XK = 64;                       // contraction elements (weight rows i) per stage
+constexpr int XSTAGES = 6;
+constexpr int XA_BYTES = 128 * XK * 2;       // this CTA's 128 tokens of dY: 16 KiB
+constexpr int XB_BYTES = XK * 128 * 2;       // this CTA's 128 weight columns: 16 KiB
+constexpr int XSTAGE_BYTES = XA_BYTES + XB_BYTES;
+constexpr int XQ_SLOTS = 8;
+constexpr int XQ_BYTES = 4096;               // 64 rows x up to 64 B of codes
+constexpr int X_TMEM_COLS = 512;
+constexpr int X_SMEM_BYTES = XSTAGES * XSTAGE_BYTES + XQ_SLOTS * XQ_BYTES + 1024 + 512;
+constexpr int X_GROUPS = 4;
+constexpr int kDxThreads = 896;  // warps: 0 act TMA, 1 MMA, 2 TMEM alloc, 3 code TMA, 4-11 epilogue, 12-27 dequant
+
+struct DxBarriers {
+  uint64_t full_act[XSTAGES];   // leader: dY bytes of both CTAs landed
+  uint64_t full_w[XSTAGES];     // leader: weight halves of both CTAs written
+  uint64_t empty[XSTAGES];      // each CTA: MMAs that read the stage completed
+  uint64_t pk_full[XQ_SLOTS];   // each CTA: packed codes landed
+  uint64_t pk_empty[XQ_SLOTS];  // each CTA: the owning group has read the slot
+  uint64_t acc_full[2];         // each CTA: accumulator ready
+  uint64_t acc_empty[2];        // leader: both CTAs' epilogues drained the accumulator
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+struct DxParams {
+  const uint8_t* zeros;
+  const float* scales;
+  __nv_bfloat16* out;   // dX [T, K]
+  int N, K, G, g, g_shift, T;
+  int j_tiles, t_tiles, k_blocks;   // 256-column tiles, 256-token tiles, 64-row stages over N
+  int* status;
+};
+
+__device__ __forceinline__ int dx_group_of(const DxParams& p, int col) {
+  if (p.G == 1) return 0;
+  return p.g_shift >= 0 ? (col >> p.g_shift) : (col / p.g);
+}
+
+template <int BITS>
+__global__ void __launch_bounds__(kDxThreads, 1)
+qdx_pair_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_constant__ CUtensorMap tmap_q,
+                const DxParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
+                                             ~static_cast<uintptr_t>(1023));
+  uint8_t* sm_q = base + XSTAGES * XSTAGE_BYTES;
+  DxBarriers* bars = reinterpret_cast<DxBarriers*>(sm_q + XQ_SLOTS * XQ_BYTES);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  const bool leader = rank == 0;
+  volatile int* abort_flag = &bars->abort_flag;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < XSTAGES; ++s) {
+      mbar_init(smem_u32(&bars->full_act[s]), 1);
+      mbar_init(smem_u32(&bars->full_w[s]), 8);           // 4 warps of one group in each CTA
+      mbar_init(smem_u32(&bars->empty[s]), 1);
+    }
+    for (int q = 0; q < XQ_SLOTS; ++q) {
+      mbar_init(smem_u32(&bars->pk_full[q]), 1);
+      mbar_init(smem_u32(&bars->pk_empty[q]), 4);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(smem_u32(&bars->acc_full[b]), 1);
+      mbar_init(smem_u32(&bars->acc_empty[b]), 16);       // 8 epilogue warps in each CTA
+    }
+    bars->abort_flag = 0;
+    fence_mbar_init();
+    prefetch_tmap(&tmap_dy);
+    prefetch_tmap(&tmap_q);
+  }
+  if (warp == 2) {
+    tmem_alloc_pair(smem_u32(&bars->tmem_base), X_TMEM_COLS);
+    tmem_relinquish_pair();
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();
+  tc_fence_after();
+  const uint32_t tmem_base = bars->tmem_base;
+  const int total_tiles = p.j_tiles * p.t_tiles;
+  const int pair = blockIdx.x >> 1;
+  const int n_pairs = gridDim.x >> 1;
+  const int my_tiles = (total_tiles - pair + n_pairs - 1) / n_pairs;
+
+  if (warp == 0) {
+    // ------------------------------------------ dY TMA (one lane)
+    if (lane == 0) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (int tile = pair; ok && tile < total_tiles; tile += n_pairs) {
+        const int t0 = (tile / p.j_tiles) * 256 + (int)rank * 128;
+        for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
+          const int s = it % XSTAGES;
+          const uint32_t ph = (it / XSTAGES) & 1u;
+          if (!mbar_wait_cluster(smem_u32(&bars->empty[s]), ph ^ 1u, abort_flag)) { ok = false; break; }
+          if (leader) mbar_arrive_expect_tx(smem_u32(&bars->full_act[s]), 2 * XA_BYTES);
+          tma_load_2d_pair(smem_u32(base + s * XSTAGE_BYTES), &tmap_dy,
+                           mapa_shared(smem_u32(&bars->full_act[s]), 0), kb * XK, t0);
+        }
+      }
+    }
+  } else if (warp == 3) {
+    // ------------------------------------------ packed-code TMA (one lane)
+    if (lane == 0) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (int tile = pair; ok && tile < total_tiles; tile += n_pairs) {
+        const int w0 = (tile % p.j_tiles) * 256 + (int)rank * 128;   // first column of this CTA
+        for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
+          const int q = it % XQ_SLOTS;
+          const uint32_t ph = (it / XQ_SLOTS) & 1u;
+          if (!mbar_wait(smem_u32(&bars->pk_empty[q]), ph ^ 1u, abort_flag)) { ok = false; break; }
+          const uint32_t bar = smem_u32(&bars->pk_full[q]);
+          mbar_arrive_expect_tx(bar, 64 * 16 * BITS);
+          tma_load_2d(smem_u32(sm_q + q * XQ_BYTES), &tmap_q, bar, (w0 >> 5) * BITS, kb * XK);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------ MMA issuer (leader CTA, one lane)
+    if (leader && lane == 0) {
+      constexpr uint32_t idesc = idesc_bf16_f32(256, 256, 0, 1);
+      uint32_t it = 0;
+      int local = 0;
+      bool ok = true;
+      for (int tile = pair; ok && tile < total_tiles; tile += n_pairs, ++local) {
+        const int buf = local & 1;
+        const uint32_t acc_ph = (local >> 1) & 1u;
+        if (!mbar_wait_cluster(smem_u32(&bars->acc_empty[buf]), acc_ph ^ 1u, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + buf * 256;
+        for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
+          const int s = it % XSTAGES;
+          const uint32_t ph = (it / XSTAGES) & 1u;
+          if (!mbar_wait_cluster(smem_u32(&bars->full_w[s]), ph, abort_flag) ||
+              !mbar_wait_cluster(smem_u32(&bars->full_act[s]), ph, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t a_addr = smem_u32(base + s * XSTAGE_BYTES);
+          const uint32_t b_addr = a_addr + XA_BYTES;
+#pragma unroll
+          for (int k = 0; k < XK / 16; ++k) {
+            const uint64_t adesc = smem_desc_sw128(a_addr + k * 32, 16, 1024);
+            const uint64_t bdesc = smem_desc_sw128(b_addr + k * (16 * 128), 64 * 128, 1024);
+            mma_bf16_ss_pair(d_tmem, adesc, bdesc, idesc, (kb | k) != 0 ? 1u : 0u);
+          }
+          mma_commit_pair(smem_u32(&bars->empty[s]), 3);
+        }
+        if (ok) mma_commit_pair(smem_u32(&bars->acc_full[buf]), 3);
+      }
+    }
+  } else if (warp >= 4 && warp < 12) {
+    // ------------------------------------------ epilogue: thread = token, 128 columns
+    const int quarter = warp & 3;
+    const int half = (warp - 4) >> 2;
+    const uint32_t acc_empty_leader0 = mapa_shared(smem_u32(&bars->acc_empty[0]), 0);
+    int local = 0;
+    bool ok = true;
+    for (int tile = pair; ok && tile < total_tiles; tile += n_pairs, ++local) {
+      const int j0 = (tile % p.j_tiles) * 256;
+      const int t = (tile / p.j_tiles) * 256 + (int)rank * 128 + quarter * 32 + lane;
+      const int buf = local & 1;
+      const uint32_t acc_ph = (local >> 1) & 1u;
+      if (!mbar_wait_cluster(smem_u32(&bars->acc_full[buf]), acc_ph, abort_flag)) { ok = false; break; }
+      tc_fence_after();
+#pragma unroll 1
+      for (int cc = 0; cc < 4; ++cc) {
+        const int c0 = j0 + half * 128 + cc * 32;
+        if (c0 >= p.K) break;
+        uint32_t v[32];
+        tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * 256 + half * 128 + cc * 32, v);
+        tmem_ld_wait();
+        if (t < p.T) {
+          __nv_bfloat16* dst = p.out + (size_t)t * p.K + c0;
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            uint4 o;
+            __nv_bfloat162 h;
+            h = __floats2bfloat162_rn(__uint_as_float(v[8 * q + 0]), __uint_as_float(v[8 * q + 1])); o.x = *reinterpret_cast<uint32_t*>(&h);
+            h = __floats2bfloat162_rn(__uint_as_float(v[8 * q + 2]), __uint_as_float(v[8 * q + 3])); o.y = *reinterpret_cast<uint32_t*>(&h);
+            h = __floats2bfloat162_rn(__uint_as_float(v[8 * q + 4]), __uint_as_float(v[8 * q + 5])); o.z = *reinterpret_cast<uint32_t*>(&h);
+            h = __floats2bfloat162_rn(__uint_as_float(v[8 * q + 6]), __uint_as_float(v[8 * q + 7])); o.w = *reinterpret_cast<uint32_t*>(&h);
+            *reinterpret_cast<uint4*>(dst + 8 * q) = o;   // K is a multiple of 32: the 32 columns are all valid
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(acc_empty_leader0 + buf * 8);
+    }
+  } else if (warp >= 12) {
+    // ------------------------------------------ weight dequant (this CTA's 128 columns)
+    // Group g (four warps) serves the stages with it % 4 == g.  A stage is 64 weight rows x
+    // 4 units of 32 columns; lanes = 8 rows x 4 units, a thread converts (row, u) and
+    // (row + 32, u) and writes them MN-major: chunk (u / 2) of 64 columns, 128 bytes per row.
+    const int grp = (warp - 12) >> 2;
+    const int gw = (warp - 12) & 3;
+    const int row8 = lane & 7, u4 = lane >> 3;
+    const int row_a = gw * 8 + row8, row_b = row_a + 32;
+    const int chunk0 = (u4 & 1) * 4;
+    const int swz = row_a & 7;
+    const uint32_t off_a = (uint32_t)((u4 >> 1) * (64 * 128) + row_a * 128);
+    const uint32_t off_b = (uint32_t)((u4 >> 1) * (64 * 128) + row_b * 128);
+    const uint32_t full_w_leader0 = mapa_shared(smem_u32(&bars->full_w[0]), 0);
+    const uint32_t total_it = (uint32_t)my_tiles * (uint32_t)p.k_blocks;
+    int pf_tile = pair, pf_kb = grp;
+    while (pf_kb >= p.k_blocks) { pf_kb -= p.k_blocks; pf_tile += n_pairs; }
+    int pf_col = (pf_tile % p.j_tiles) * 256 + (int)rank * 128 + 32 * u4;
+    auto load_zs = [&](uint32_t (&z)[2], float (&sc)[2]) {
+#pragma unroll
+      for (int k = 0; k < 2; ++k) {
+        const int i = pf_kb * XK + (k ? row_b : row_a);
+        z[k] = 0u;
+        sc[k] = 0.0f;
+        if (i < p.N && pf_col < p.K) {
+          const size_t gi = (size_t)i * p.G + dx_group_of(p, pf_col);
+          z[k] = __ldg(p.zeros + gi);
+          sc[k] = __ldg(p.scales + gi);
+        }
+      }
+      pf_kb += X_GROUPS;
+      while (pf_kb >= p.k_blocks) {
+        pf_kb -= p.k_blocks;
+        pf_tile += n_pairs;
+        pf_col = (pf_tile % p.j_tiles) * 256 + (int)rank * 128 + 32 * u4;
+      }
+    };
+    uint32_t z[2], zn[2];
+    float sc[2], scn[2];
+    if ((uint32_t)grp < total_it) load_zs(z, sc);
+    for (uint32_t it = grp; it < total_it; it += X_GROUPS) {
+      if (it + X_GROUPS < total_it) load_zs(zn, scn);
+      const int s = it % XSTAGES;
+      const int q = it % XQ_SLOTS;
+      if (!mbar_wait(smem_u32(&bars->pk_full[q]), (it / XQ_SLOTS) & 1u, abort_flag)) break;
+      uint32_t wa[BITS], wb[BITS];
+      {
+        const uint32_t* src = reinterpret_cast<const uint32_t*>(sm_q + q * XQ_BYTES) + u4 * BITS;
+#pragma unroll
+        for (int e = 0; e < BITS; ++e) {
+          wa[e] = src[row_a * (4 * BITS) + e];
+          wb[e] = src[row_b * (4 * BITS) + e];
+        }
+      }
+      uint32_t oa[16], ob[16];
+      dq::unit32_natural<BITS, true>(wa, z[0], sc[0], oa);
+      dq::unit32_natural<BITS, true>(wb, z[1], sc[1], ob);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&bars->pk_empty[q]));   // codes consumed: slot free
+      if (!mbar_wait_cluster(smem_u32(&bars->empty[s]), ((it / XSTAGES) & 1u) ^ 1u, abort_flag)) break;
+      uint8_t* wbuf = base + s * XSTAGE_BYTES + XA_BYTES;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        *reinterpret_cast<uint4*>(wbuf + off_a + (((chunk0 + c) ^ swz) << 4)) =
+            make_uint4(oa[4 * c], oa[4 * c + 1], oa[4 * c + 2], oa[4 * c + 3]);
+        *reinterpret_cast<uint4*>(wbuf + off_b + (((chunk0 + c) ^ swz) << 4)) =
+            make_uint4(ob[4 * c], ob[4 * c + 1], ob[4 * c + 2], ob[4 * c + 3]);
+      }
+      // make the tile visible to the tensor cores of both CTAs, then tell the leader
+      fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster_release(full_w_leader0 + s * 8);
+      z[0] = zn[0]; z[1] = zn[1];
+      sc[0] = scn[0]; sc[1] = scn[1];
+    }
+  }
+
+  if (*abort_flag) {
+    // let copies and MMAs already in flight finish before memory is released
+    for (int i = 0; i < 64; ++i) __nanosleep(1000);
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();
+  if (warp == 2) {
+    tc_fence_after();
+    tmem_dealloc_pair(tmem_base, X_TMEM_COLS);
+  }
+  if (threadIdx.x == 0 && bars->abort_flag) {
+    atomicExch(p.status, (int)PEQA_ERR_DEVICE_TIMEOUT);
+    p.status[1] = (int)blockIdx.x;
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+int dx_encode_fn(EncodeTiledFn* out) {
+  static EncodeTiledFn cached = nullptr;
+  if (!cached) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    PEQA_CUDA(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
+    if (!fn || qres != cudaDriverEntryPointSuccess) return cuda_fail(cudaErrorUnknown);
+    cached = reinterpret_cast<EncodeTiledFn>(fn);
+  }
+  *out = cached;
+  return PEQA_OK;
+}
+
+template <int BITS>
+int launch_dx_pair_t(const CUtensorMap& ta, const CUtensorMap& tq, const DxParams& p, int pairs,
+                     cudaStream_t st) {
+  auto kern = qdx_pair_kernel<BITS>;
+  PEQA_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, X_SMEM_BYTES));
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2 * pairs, 1, 1);
+  cfg.blockDim = dim3(kDxThreads, 1, 1);
+  cfg.dynamicSmemBytes = X_SMEM_BYTES;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  PEQA_CUDA(cudaLaunchKernelEx(&cfg, kern, ta, tq, p));
+  return PEQA_OK;
+}
+
+}  // namespace
+
+// Same shape rule as the forward pair kernel: the code boxes need a 16-byte row pitch.
+bool dx_pair_supported(const peqa_qweight_t* w) {
+  return ((size_t)w->in_features * w->bits / 8) % 16 == 0;
+}
+
+int launch_dx_pair(const peqa_qweight_t* w, int g, const void* dY, int T, void* dX, cudaStream_t st) {
+  DxParams p;
+  p.zeros = w->zeros;
+  p.scales = w->scales;
+  p.out = static_cast<__nv_bfloat16*>(dX);
+  p.N = w->out_features;
+  p.K = w->in_features;
+  p.g = g;
+  p.G = p.K / g;
+  p.g_shift = -1;
+  for (int b = 5; b < 31; ++b)
+    if ((1 << b) == g) p.g_shift = b;
+  p.T = T;
+  p.j_tiles = (p.K + 255) / 256;
+  p.t_tiles = (T + 255) / 256;
+  p.k_blocks = (p.N + XK - 1) / XK;
+  PEQA_TRY(status_word(&p.status));
+  EncodeTiledFn enc = nullptr;
+  PEQA_TRY(dx_encode_fn(&enc));
+  CUtensorMap ta, tq;
+  {
+    cuuint64_t dims[2] = {(cuuint64_t)p.N, (cuuint64_t)T};
+    cuuint64_t strides[1] = {(cuuint64_t)p.N * 2};
+    cuuint32_t box[2] = {64, 128};
+    cuuint32_t estr[2] = {1, 1};
+    if (enc(&ta, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(dY), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return cuda_fail(cudaErrorInvalidValue);
+  }
+  {
+    const int wpr = p.K * w->bits / 32;
+    cuuint64_t dims[2] = {(cuuint64_t)wpr, (cuuint64_t)p.N};
+    cuuint64_t strides[1] = {(cuuint64_t)wpr * 4};
+    cuuint32_t box[2] = {(cuuint32_t)(4 * w->bits), 64};
+    cuuint32_t estr[2] = {1, 1};
+    if (enc(&tq, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<uint32_t*>(w->qweight), dims, strides,
+            box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return cuda_fail(cudaErrorInvalidValue);
+  }
+  int sms = 0, dev = 0;
+  PEQA_CUDA(cudaGetDevice(&dev));
+  PEQA_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+  const int tiles = p.j_tiles * p.t_tiles;
+  const int max_pairs = sms / 2;
+  const int pairs = tiles < max_pairs ? tiles : max_pairs;
+  return w->bits == 4 ? launch_dx_pair_t<4>(ta, tq, p, pairs, st) : launch_dx_pair_t<3>(ta, tq, p, pairs, st);
+}
+
+}  // namespace peqa

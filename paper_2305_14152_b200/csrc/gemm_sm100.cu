@@ -797,6 +797,7 @@ int launch_fwd(const peqa_qweight_t* w, int g, const void* X, int T, void* Y, cu
 }
 
 int launch_dx(const peqa_qweight_t* w, int g, const void* dY, int T, void* dX, cudaStream_t st) {
+  if (dx_pair_supported(w)) return launch_dx_pair(w, g, dY, T, dX, st);
   return launch_qgemm(w, g, dY, T, dX, true, st);
 }
 
