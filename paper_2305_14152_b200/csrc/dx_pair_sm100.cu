@@ -1,22 +1,24 @@
 // Backward with respect to the input, dX = dY * W_hat (chain rule on Eq. 2), on
 // CTA pairs.
 //
-// A pair of CTAs (cta_group::2) owns a tile of 256 tokens x 256 input columns j.
-// The tokens are the MMA "M" side: CTA `rank` TMA-loads its 128 tokens of dY
-// (A operand, K-major: the contraction index i is contiguous in dY) and keeps
-// their accumulator rows.  The weights are the "N" side, split between the two
-// CTAs: each dequantises the 128 columns [j0 + 128*rank, +128) of the stage's
-// 64 weight rows into its own shared memory, MN-major (a row of packed codes is
-// unpacked along j, exactly as it is stored), and the pair's tensor cores read
-// both halves.  Per 64-deep stage a CTA moves 32 KiB into shared memory and its
-// tensor core reads 48 KiB, against 48 + 48 KiB in the single-CTA kernel, and
-// the accumulator is token-major, so every epilogue thread writes contiguous
-// 64-byte runs of dX.
+// A pair of CTAs (cta_group::2) owns a tile of 512 tokens x 256 input columns j,
+// held as two 256 x 256 accumulators that fill tensor memory.  The tokens are
+// the MMA "M" side: CTA `rank` TMA-loads two blocks of 128 tokens of dY per
+// stage (A operands, K-major: the contraction index i is contiguous in dY) and
+// keeps their accumulator rows.  The weights are the "N" side, split between the
+// two CTAs: each dequantises the 128 columns [j0 + 128*rank, +128) of the
+// stage's 64 weight rows into its own shared memory, MN-major (a row of packed
+// codes is unpacked along j, exactly as it is stored), and both token blocks
+// multiply the same weight stage.  A weight element is therefore rebuilt once
+// per 512 tokens, which brings the conversion work per stage (8192 elements per
+// CTA) under the time the tensor cores need for it (two 256x256x64 products);
+// and the accumulator is token-major, so an epilogue thread writes contiguous
+// runs of dX.
 //
 // Packed codes come through their own TMA ring (one box = 64 weight rows x the
 // CTA's 128 columns); four groups of four dequant warps take the stages
-// round-robin.  Two 256-column accumulators overlap the epilogue of one tile
-// with the main loop of the next.
+// round-robin.  A tile whose second token block lies wholly beyond T runs with
+// one block.
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -31,8 +33,9 @@ namespace {
 using namespace ptx;
 
 constexpr int XK = 64;                       // contraction elements (weight rows i) per stage
-constexpr int XSTAGES = 6;
-constexpr int XA_BYTES = 128 * XK * 2;       // this CTA's 128 tokens of dY: 16 KiB
+constexpr int XSTAGES = 4;
+constexpr int XBLK_BYTES = 128 * XK * 2;     // one block of 128 tokens of dY: 16 KiB
+constexpr int XA_BYTES = 2 * XBLK_BYTES;     // this CTA's two token blocks
 constexpr int XB_BYTES = XK * 128 * 2;       // this CTA's 128 weight columns: 16 KiB
 constexpr int XSTAGE_BYTES = XA_BYTES + XB_BYTES;
 constexpr int XQ_SLOTS = 8;
@@ -48,8 +51,8 @@ struct DxBarriers {
   uint64_t empty[XSTAGES];      // each CTA: MMAs that read the stage completed
   uint64_t pk_full[XQ_SLOTS];   // each CTA: packed codes landed
   uint64_t pk_empty[XQ_SLOTS];  // each CTA: the owning group has read the slot
-  uint64_t acc_full[2];         // each CTA: accumulator ready
-  uint64_t acc_empty[2];        // leader: both CTAs' epilogues drained the accumulator
+  uint64_t acc_full;            // each CTA: both accumulators ready
+  uint64_t acc_empty;           // leader: both CTAs' epilogues drained them
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -59,7 +62,7 @@ struct DxParams {
   const float* scales;
   __nv_bfloat16* out;   // dX [T, K]
   int N, K, G, g, g_shift, T;
-  int j_tiles, t_tiles, k_blocks;   // 256-column tiles, 256-token tiles, 64-row stages over N
+  int j_tiles, t_tiles, k_blocks;   // 256-column tiles, 512-token tiles, 64-row stages over N
   int* status;
 };
 
@@ -92,10 +95,8 @@ qdx_pair_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_consta
       mbar_init(smem_u32(&bars->pk_full[q]), 1);
       mbar_init(smem_u32(&bars->pk_empty[q]), 4);
     }
-    for (int b = 0; b < 2; ++b) {
-      mbar_init(smem_u32(&bars->acc_full[b]), 1);
-      mbar_init(smem_u32(&bars->acc_empty[b]), 16);       // 8 epilogue warps in each CTA
-    }
+    mbar_init(smem_u32(&bars->acc_full), 1);
+    mbar_init(smem_u32(&bars->acc_empty), 16);            // 8 epilogue warps in each CTA
     bars->abort_flag = 0;
     fence_mbar_init();
     prefetch_tmap(&tmap_dy);
@@ -121,14 +122,18 @@ qdx_pair_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_consta
       uint32_t it = 0;
       bool ok = true;
       for (int tile = pair; ok && tile < total_tiles; tile += n_pairs) {
-        const int t0 = (tile / p.j_tiles) * 256 + (int)rank * 128;
+        const int tt0 = (tile / p.j_tiles) * 512;
+        const int blocks = tt0 + 256 < p.T ? 2 : 1;
+        const int t0 = tt0 + (int)rank * 128;
         for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
           const int s = it % XSTAGES;
           const uint32_t ph = (it / XSTAGES) & 1u;
           if (!mbar_wait_cluster(smem_u32(&bars->empty[s]), ph ^ 1u, abort_flag)) { ok = false; break; }
-          if (leader) mbar_arrive_expect_tx(smem_u32(&bars->full_act[s]), 2 * XA_BYTES);
-          tma_load_2d_pair(smem_u32(base + s * XSTAGE_BYTES), &tmap_dy,
-                           mapa_shared(smem_u32(&bars->full_act[s]), 0), kb * XK, t0);
+          if (leader) mbar_arrive_expect_tx(smem_u32(&bars->full_act[s]), 2 * blocks * XBLK_BYTES);
+          const uint32_t bar = mapa_shared(smem_u32(&bars->full_act[s]), 0);
+          tma_load_2d_pair(smem_u32(base + s * XSTAGE_BYTES), &tmap_dy, bar, kb * XK, t0);
+          if (blocks == 2)
+            tma_load_2d_pair(smem_u32(base + s * XSTAGE_BYTES + XBLK_BYTES), &tmap_dy, bar, kb * XK, t0 + 256);
         }
       }
     }
@@ -157,11 +162,9 @@ qdx_pair_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_consta
       int local = 0;
       bool ok = true;
       for (int tile = pair; ok && tile < total_tiles; tile += n_pairs, ++local) {
-        const int buf = local & 1;
-        const uint32_t acc_ph = (local >> 1) & 1u;
-        if (!mbar_wait_cluster(smem_u32(&bars->acc_empty[buf]), acc_ph ^ 1u, abort_flag)) { ok = false; break; }
+        const int blocks = (tile / p.j_tiles) * 512 + 256 < p.T ? 2 : 1;
+        if (!mbar_wait_cluster(smem_u32(&bars->acc_empty), (uint32_t)(local & 1) ^ 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + buf * 256;
         for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
           const int s = it % XSTAGES;
           const uint32_t ph = (it / XSTAGES) & 1u;
@@ -170,37 +173,39 @@ qdx_pair_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_consta
           tc_fence_after();
           const uint32_t a_addr = smem_u32(base + s * XSTAGE_BYTES);
           const uint32_t b_addr = a_addr + XA_BYTES;
+          for (int m = 0; m < blocks; ++m) {
 #pragma unroll
-          for (int k = 0; k < XK / 16; ++k) {
-            const uint64_t adesc = smem_desc_sw128(a_addr + k * 32, 16, 1024);
-            const uint64_t bdesc = smem_desc_sw128(b_addr + k * (16 * 128), 64 * 128, 1024);
-            mma_bf16_ss_pair(d_tmem, adesc, bdesc, idesc, (kb | k) != 0 ? 1u : 0u);
+            for (int k = 0; k < XK / 16; ++k) {
+              const uint64_t adesc = smem_desc_sw128(a_addr + m * XBLK_BYTES + k * 32, 16, 1024);
+              const uint64_t bdesc = smem_desc_sw128(b_addr + k * (16 * 128), 64 * 128, 1024);
+              mma_bf16_ss_pair(tmem_base + m * 256, adesc, bdesc, idesc, (kb | k) != 0 ? 1u : 0u);
+            }
           }
           mma_commit_pair(smem_u32(&bars->empty[s]), 3);
         }
-        if (ok) mma_commit_pair(smem_u32(&bars->acc_full[buf]), 3);
+        if (ok) mma_commit_pair(smem_u32(&bars->acc_full), 3);
       }
     }
   } else if (warp >= 4 && warp < 12) {
-    // ------------------------------------------ epilogue: thread = token, 128 columns
+    // ------------------------------------------ epilogue: thread = token, 256 columns
     const int quarter = warp & 3;
-    const int half = (warp - 4) >> 2;
-    const uint32_t acc_empty_leader0 = mapa_shared(smem_u32(&bars->acc_empty[0]), 0);
+    const int m = (warp - 4) >> 2;                 // token block = accumulator
+    const uint32_t acc_empty_leader = mapa_shared(smem_u32(&bars->acc_empty), 0);
     int local = 0;
     bool ok = true;
     for (int tile = pair; ok && tile < total_tiles; tile += n_pairs, ++local) {
       const int j0 = (tile % p.j_tiles) * 256;
-      const int t = (tile / p.j_tiles) * 256 + (int)rank * 128 + quarter * 32 + lane;
-      const int buf = local & 1;
-      const uint32_t acc_ph = (local >> 1) & 1u;
-      if (!mbar_wait_cluster(smem_u32(&bars->acc_full[buf]), acc_ph, abort_flag)) { ok = false; break; }
+      const int tt0 = (tile / p.j_tiles) * 512;
+      const int blocks = tt0 + 256 < p.T ? 2 : 1;
+      const int t = tt0 + m * 256 + (int)rank * 128 + quarter * 32 + lane;
+      if (!mbar_wait_cluster(smem_u32(&bars->acc_full), (uint32_t)(local & 1), abort_flag)) { ok = false; break; }
       tc_fence_after();
 #pragma unroll 1
-      for (int cc = 0; cc < 4; ++cc) {
-        const int c0 = j0 + half * 128 + cc * 32;
-        if (c0 >= p.K) break;
+      for (int cc = 0; cc < 8; ++cc) {
+        const int c0 = j0 + cc * 32;
+        if (c0 >= p.K || m >= blocks) break;
         uint32_t v[32];
-        tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * 256 + half * 128 + cc * 32, v);
+        tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + m * 256 + cc * 32, v);
         tmem_ld_wait();
         if (t < p.T) {
           __nv_bfloat16* dst = p.out + (size_t)t * p.K + c0;
@@ -218,7 +223,7 @@ qdx_pair_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_consta
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive_cluster(acc_empty_leader0 + buf * 8);
+      if (lane == 0) mbar_arrive_cluster(acc_empty_leader);
     }
   } else if (warp >= 12) {
     // ------------------------------------------ weight dequant (this CTA's 128 columns)
@@ -374,7 +379,7 @@ int launch_dx_pair(const peqa_qweight_t* w, int g, const void* dY, int T, void* 
     if ((1 << b) == g) p.g_shift = b;
   p.T = T;
   p.j_tiles = (p.K + 255) / 256;
-  p.t_tiles = (T + 255) / 256;
+  p.t_tiles = (T + 511) / 512;
   p.k_blocks = (p.N + XK - 1) / XK;
   PEQA_TRY(status_word(&p.status));
   EncodeTiledFn enc = nullptr;
