@@ -1,24 +1,27 @@
-// Forward of the PEQA layer, Y = X * W_hat^T (Eq. 2), on CTA pairs with the
-// dequantised weight operand in tensor memory.
+// Forward of the PEQA layer, Y = X * W_hat^T (Eq. 2), on CTA pairs.
 //
-// A pair of CTAs (cta_group::2) owns a tile of 256 output channels x 256 tokens.
-// CTA `rank` owns channels [r0 + 128*rank, +128): it rebuilds their (Q - z)
-// [* bf16(s)] as bf16 and writes them with tcgen05.st into tensor memory, where
-// tcgen05.mma reads them as its A operand (lane = channel, one 32-bit column =
-// two consecutive contraction elements).  The activation tile is the B operand:
-// each CTA TMA-loads 128 of the 256 tokens into its own shared memory and the
-// pair's MMAs read both halves.  Only the activations go through shared memory
-// at MMA rate: 16 KiB in and 32 KiB out per 64-deep stage, against the 96 KiB a
-// single-CTA kernel with both operands in shared memory moves -- and it is that
-// shared-memory traffic which bounds the single-CTA kernel.
+// A pair of CTAs (cta_group::2) owns a tile of 512 tokens x 256 output channels,
+// held as two 256 x 256 accumulators that fill tensor memory.  The tokens are
+// the MMA "M" side: CTA `rank` TMA-loads two blocks of 128 tokens of X per
+// 64-deep stage (A operands, K-major).  The weights are the "N" side, split
+// between the two CTAs: each rebuilds (Q - z) [* bf16(s)] of its 128 channels
+// [n0 + 128*rank, +128) as bf16 in its own shared memory, K-major with the
+// 128-byte swizzle the tensor core expects, and both token blocks multiply the
+// same weight stage.  A weight element is therefore rebuilt once per 512
+// tokens, which brings the conversion work per stage (8192 elements per CTA)
+// under the time the tensor cores need for it (two 256x256x64 products), and
+// the accumulator is token-major, so an epilogue thread writes contiguous runs
+// of Y.
 //
 // Packed codes reach the dequant warps through their own TMA ring (one box =
-// 128 channels x 64 columns of codes), so the global reads are bulk copies.
-// Four groups of four dequant warps take the stages round-robin, so that one
-// group's wait -> read -> convert -> store -> signal chain overlaps the others'.
+// 128 channels x 64 columns of codes).  Four groups of four dequant warps take
+// the stages round-robin, so that one group's wait -> read -> convert -> store
+// -> signal chain overlaps the others'.  A tile whose second token block lies
+// wholly beyond T runs with one block.
 //
-// Tensor memory (512 columns): [0,256) fp32 accumulator (256 tokens),
-// [256,512) eight weight stages of 32 columns (64 contraction elements).
+// With one scale per channel (G == 1) the weights stay the exact integers
+// Q - z and the fp32 scale multiplies the accumulator columns in the epilogue;
+// with grouped scales the product (Q - z) * bf16(s) is formed before the MMA.
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -32,27 +35,27 @@ namespace {
 
 using namespace ptx;
 
-constexpr int PM = 128;            // output channels per CTA (TMEM lanes)
-constexpr int PN = 256;            // tokens per pair tile (MMA N)
-constexpr int PK = 64;             // contraction elements per stage
-constexpr int PSTAGES = 8;
-constexpr int PB_BYTES = (PN / 2) * PK * 2;          // activation half tile: 16 KiB
-constexpr int PQ_BYTES = PM * 32;                    // packed codes of one stage: 128 rows x 8 words
+constexpr int PK = 64;                       // contraction elements per stage
+constexpr int PSTAGES = 4;
+constexpr int PBLK_BYTES = 128 * PK * 2;     // one block of 128 tokens of X: 16 KiB
+constexpr int PA_BYTES = 2 * PBLK_BYTES;     // this CTA's two token blocks
+constexpr int PB_BYTES = 128 * PK * 2;       // this CTA's 128 channels: 16 KiB
+constexpr int PSTAGE_BYTES = PA_BYTES + PB_BYTES;
+constexpr int PQ_SLOTS = 8;
+constexpr int PQ_BYTES = 128 * 32;           // packed codes of one stage: 128 rows x 8 words
 constexpr int P_TMEM_COLS = 512;
-constexpr int P_ACC_COL = 0;
-constexpr int P_A_COL = 256;
-constexpr int P_SMEM_BYTES = PSTAGES * (PB_BYTES + PQ_BYTES) + 1024 + 512;
+constexpr int P_SMEM_BYTES = PSTAGES * PSTAGE_BYTES + PQ_SLOTS * PQ_BYTES + 1024 + 512;
 constexpr int P_GROUPS = 4;        // dequant groups (four warps each)
-constexpr int kPairThreads = 896;  // warps: 0 act TMA, 1 MMA, 2 TMEM alloc, 3 code TMA, 4-7 and 24-27 epilogue, 8-23 dequant
+constexpr int kPairThreads = 896;  // warps: 0 act TMA, 1 MMA, 2 TMEM alloc, 3 code TMA, 4-11 epilogue, 12-27 dequant
 
 struct PairBarriers {
-  uint64_t full_a[PSTAGES];     // leader: weight stage written to tensor memory by both CTAs
-  uint64_t full_b[PSTAGES];     // leader: activation bytes of both CTAs landed
+  uint64_t full_act[PSTAGES];   // leader: X bytes of both CTAs landed
+  uint64_t full_w[PSTAGES];     // leader: weight halves of both CTAs written
   uint64_t empty[PSTAGES];      // each CTA: MMAs that read the stage completed
-  uint64_t pk_full[PSTAGES];    // each CTA: packed codes landed
-  uint64_t pk_empty[PSTAGES];   // each CTA: the group that owns the slot has read it
-  uint64_t acc_full;            // each CTA: accumulator ready
-  uint64_t acc_empty;           // leader: both CTAs' epilogues drained the accumulator
+  uint64_t pk_full[PQ_SLOTS];   // each CTA: packed codes landed
+  uint64_t pk_empty[PQ_SLOTS];  // each CTA: the group that owns the slot has read it
+  uint64_t acc_full;            // each CTA: both accumulators ready
+  uint64_t acc_empty;           // leader: both CTAs' epilogues drained them
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -62,7 +65,7 @@ struct PairParams {
   const float* scales;
   __nv_bfloat16* out;   // Y [T, N]
   int N, K, G, g, g_shift, T;
-  int r_tiles, t_tiles, k_blocks;   // 256-channel tiles, 256-token tiles, 64-deep stages
+  int n_tiles, t_tiles, k_blocks;   // 256-channel tiles, 512-token tiles, 64-deep stages
   int* status;
 };
 
@@ -78,9 +81,8 @@ qfwd_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
   extern __shared__ uint8_t smem_raw[];
   uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                              ~static_cast<uintptr_t>(1023));
-  uint8_t* sm_b = base;                                   // PSTAGES x 16 KiB, 128B-swizzled
-  uint8_t* sm_q = base + PSTAGES * PB_BYTES;              // PSTAGES x 4 KiB, plain 32-byte rows
-  PairBarriers* bars = reinterpret_cast<PairBarriers*>(sm_q + PSTAGES * PQ_BYTES);
+  uint8_t* sm_q = base + PSTAGES * PSTAGE_BYTES;          // PQ_SLOTS x 4 KiB, plain 32-byte rows
+  PairBarriers* bars = reinterpret_cast<PairBarriers*>(sm_q + PQ_SLOTS * PQ_BYTES);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();
   const bool leader = rank == 0;
@@ -88,11 +90,13 @@ qfwd_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < PSTAGES; ++s) {
-      mbar_init(smem_u32(&bars->full_a[s]), 8);           // 4 warps of one group in each CTA
-      mbar_init(smem_u32(&bars->full_b[s]), 1);
+      mbar_init(smem_u32(&bars->full_act[s]), 1);
+      mbar_init(smem_u32(&bars->full_w[s]), 8);           // 4 warps of one group in each CTA
       mbar_init(smem_u32(&bars->empty[s]), 1);
-      mbar_init(smem_u32(&bars->pk_full[s]), 1);
-      mbar_init(smem_u32(&bars->pk_empty[s]), 4);         // 4 warps of the owning group
+    }
+    for (int q = 0; q < PQ_SLOTS; ++q) {
+      mbar_init(smem_u32(&bars->pk_full[q]), 1);
+      mbar_init(smem_u32(&bars->pk_empty[q]), 4);         // 4 warps of the owning group
     }
     mbar_init(smem_u32(&bars->acc_full), 1);
     mbar_init(smem_u32(&bars->acc_empty), 16);            // 8 epilogue warps in each CTA
@@ -110,7 +114,7 @@ qfwd_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
   cluster_sync_all();
   tc_fence_after();
   const uint32_t tmem_base = bars->tmem_base;
-  const int total_tiles = p.r_tiles * p.t_tiles;
+  const int total_tiles = p.n_tiles * p.t_tiles;
   const int pair = blockIdx.x >> 1;
   const int n_pairs = gridDim.x >> 1;
   const int my_tiles = (total_tiles - pair + n_pairs - 1) / n_pairs;
@@ -121,14 +125,18 @@ qfwd_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
       uint32_t it = 0;
       bool ok = true;
       for (int tile = pair; ok && tile < total_tiles; tile += n_pairs) {
-        const int t0 = (tile / p.r_tiles) * PN + (int)rank * (PN / 2);
+        const int tt0 = (tile / p.n_tiles) * 512;
+        const int blocks = tt0 + 256 < p.T ? 2 : 1;
+        const int t0 = tt0 + (int)rank * 128;
         for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
           const int s = it % PSTAGES;
           const uint32_t ph = (it / PSTAGES) & 1u;
           if (!mbar_wait_cluster(smem_u32(&bars->empty[s]), ph ^ 1u, abort_flag)) { ok = false; break; }
-          if (leader) mbar_arrive_expect_tx(smem_u32(&bars->full_b[s]), 2 * PB_BYTES);
-          tma_load_2d_pair(smem_u32(sm_b + s * PB_BYTES), &tmap_x,
-                           mapa_shared(smem_u32(&bars->full_b[s]), 0), kb * PK, t0);
+          if (leader) mbar_arrive_expect_tx(smem_u32(&bars->full_act[s]), 2 * blocks * PBLK_BYTES);
+          const uint32_t bar = mapa_shared(smem_u32(&bars->full_act[s]), 0);
+          tma_load_2d_pair(smem_u32(base + s * PSTAGE_BYTES), &tmap_x, bar, kb * PK, t0);
+          if (blocks == 2)
+            tma_load_2d_pair(smem_u32(base + s * PSTAGE_BYTES + PBLK_BYTES), &tmap_x, bar, kb * PK, t0 + 256);
         }
       }
     }
@@ -141,10 +149,10 @@ qfwd_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
       uint32_t it = 0;
       bool ok = true;
       for (int tile = pair; ok && tile < total_tiles; tile += n_pairs) {
-        const int r0 = (tile % p.r_tiles) * (2 * PM) + (int)rank * PM;
+        const int r0 = (tile % p.n_tiles) * 256 + (int)rank * 128;
         for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
-          const int q = it % PSTAGES;
-          const uint32_t ph = (it / PSTAGES) & 1u;
+          const int q = it % PQ_SLOTS;
+          const uint32_t ph = (it / PQ_SLOTS) & 1u;
           if (!mbar_wait(smem_u32(&bars->pk_empty[q]), ph ^ 1u, abort_flag)) { ok = false; break; }
           const uint32_t bar = smem_u32(&bars->pk_full[q]);
           mbar_arrive_expect_tx(bar, PQ_BYTES);
@@ -156,61 +164,82 @@ qfwd_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
   } else if (warp == 1) {
     // ------------------------------------------ MMA issuer (leader CTA, one lane)
     if (leader && lane == 0) {
-      constexpr uint32_t idesc = idesc_bf16_f32(2 * PM, PN, 0, 0);
+      constexpr uint32_t idesc = idesc_bf16_f32(256, 256, 0, 0);
       uint32_t it = 0;
       int local = 0;
       bool ok = true;
       for (int tile = pair; ok && tile < total_tiles; tile += n_pairs, ++local) {
+        const int blocks = (tile / p.n_tiles) * 512 + 256 < p.T ? 2 : 1;
         if (!mbar_wait_cluster(smem_u32(&bars->acc_empty), (uint32_t)(local & 1) ^ 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + P_ACC_COL;
         for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
           const int s = it % PSTAGES;
           const uint32_t ph = (it / PSTAGES) & 1u;
-          if (!mbar_wait_cluster(smem_u32(&bars->full_a[s]), ph, abort_flag) ||
-              !mbar_wait_cluster(smem_u32(&bars->full_b[s]), ph, abort_flag)) { ok = false; break; }
+          if (!mbar_wait_cluster(smem_u32(&bars->full_w[s]), ph, abort_flag) ||
+              !mbar_wait_cluster(smem_u32(&bars->full_act[s]), ph, abort_flag)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t b_addr = smem_u32(sm_b + s * PB_BYTES);
-          const uint32_t a_tmem = tmem_base + P_A_COL + s * (PK / 2);
+          const uint32_t a_addr = smem_u32(base + s * PSTAGE_BYTES);
+          const uint32_t b_addr = a_addr + PA_BYTES;
+          for (int m = 0; m < blocks; ++m) {
 #pragma unroll
-          for (int k = 0; k < PK / 16; ++k) {
-            const uint64_t bdesc = smem_desc_sw128(b_addr + k * 32, 16, 1024);
-            mma_bf16_ts_pair(d_tmem, a_tmem + k * 8, bdesc, idesc, (kb | k) != 0 ? 1u : 0u);
+            for (int k = 0; k < PK / 16; ++k) {
+              const uint64_t adesc = smem_desc_sw128(a_addr + m * PBLK_BYTES + k * 32, 16, 1024);
+              const uint64_t bdesc = smem_desc_sw128(b_addr + k * 32, 16, 1024);
+              mma_bf16_ss_pair(tmem_base + m * 256, adesc, bdesc, idesc, (kb | k) != 0 ? 1u : 0u);
+            }
           }
           mma_commit_pair(smem_u32(&bars->empty[s]), 3);
         }
         if (ok) mma_commit_pair(smem_u32(&bars->acc_full), 3);
       }
     }
-  } else if ((warp >= 4 && warp < 8) || warp >= 24) {
-    // ------------------------------------------ epilogue (lane = output channel)
-    // Two warps per TMEM lane quarter: warps 4-7 take tokens [0,128) of the tile,
-    // warps 24-27 tokens [128,256).
-    const int ew = warp & 3;
-    const int thalf = warp >= 24 ? 1 : 0;
+  } else if (warp >= 4 && warp < 12) {
+    // ------------------------------------------ epilogue: thread = token, 256 channels
+    const int quarter = warp & 3;
+    const int m = (warp - 4) >> 2;                 // token block = accumulator
     const uint32_t acc_empty_leader = mapa_shared(smem_u32(&bars->acc_empty), 0);
+    const bool vec_ok = (p.N & 7) == 0;
     int local = 0;
     bool ok = true;
     for (int tile = pair; ok && tile < total_tiles; tile += n_pairs, ++local) {
-      const int r0 = (tile % p.r_tiles) * (2 * PM) + (int)rank * PM;
-      const int t0 = (tile / p.r_tiles) * PN;
+      const int n0 = (tile % p.n_tiles) * 256;
+      const int tt0 = (tile / p.n_tiles) * 512;
+      const int blocks = tt0 + 256 < p.T ? 2 : 1;
+      const int t = tt0 + m * 256 + (int)rank * 128 + quarter * 32 + lane;
       if (!mbar_wait_cluster(smem_u32(&bars->acc_full), (uint32_t)(local & 1), abort_flag)) { ok = false; break; }
       tc_fence_after();
-      const int r = r0 + ew * 32 + lane;
-      float scale = 1.0f;
-      if (!FOLD && r < p.N) scale = __ldg(p.scales + r);
 #pragma unroll 1
-      for (int cc = thalf * (PN / 64); cc < (thalf + 1) * (PN / 64); ++cc) {
-        const int tc0 = t0 + cc * 32;
-        if (tc0 >= p.T) break;
+      for (int cc = 0; cc < 8; ++cc) {
+        const int c0 = n0 + cc * 32;
+        if (c0 >= p.N || m >= blocks) break;
         uint32_t v[32];
-        tmem_ld_32x32(tmem_base + ((uint32_t)(ew * 32) << 16) + P_ACC_COL + cc * 32, v);
+        tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + m * 256 + cc * 32, v);
         tmem_ld_wait();
-        if (r < p.N) {
-          __nv_bfloat16* dst = p.out + (size_t)tc0 * p.N + r;
+        if (!FOLD) {
+          // one scale per channel: every lane reads the same 32 scales (broadcast loads)
 #pragma unroll
           for (int j = 0; j < 32; ++j) {
-            if (tc0 + j < p.T) dst[(size_t)j * p.N] = __float2bfloat16_rn(__uint_as_float(v[j]) * scale);
+            const float sc = c0 + j < p.N ? __ldg(p.scales + c0 + j) : 0.0f;
+            v[j] = __float_as_uint(__uint_as_float(v[j]) * sc);
+          }
+        }
+        if (t < p.T) {
+          __nv_bfloat16* dst = p.out + (size_t)t * p.N + c0;
+          if (vec_ok && c0 + 32 <= p.N) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              uint4 o;
+              __nv_bfloat162 h;
+              h = __floats2bfloat162_rn(__uint_as_float(v[8 * q + 0]), __uint_as_float(v[8 * q + 1])); o.x = *reinterpret_cast<uint32_t*>(&h);
+              h = __floats2bfloat162_rn(__uint_as_float(v[8 * q + 2]), __uint_as_float(v[8 * q + 3])); o.y = *reinterpret_cast<uint32_t*>(&h);
+              h = __floats2bfloat162_rn(__uint_as_float(v[8 * q + 4]), __uint_as_float(v[8 * q + 5])); o.z = *reinterpret_cast<uint32_t*>(&h);
+              h = __floats2bfloat162_rn(__uint_as_float(v[8 * q + 6]), __uint_as_float(v[8 * q + 7])); o.w = *reinterpret_cast<uint32_t*>(&h);
+              *reinterpret_cast<uint4*>(dst + 8 * q) = o;
+            }
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (c0 + j < p.N) dst[j] = __float2bfloat16_rn(__uint_as_float(v[j]));
           }
         }
       }
@@ -218,28 +247,29 @@ qfwd_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(acc_empty_leader);
     }
-  } else if (warp >= 8 && warp < 24) {
-    // ------------------------------------------ weight dequant -> tensor memory
-    // Group g (four warps) serves the stages with it % 4 == g.  Warp (w % 4) owns TMEM
-    // lanes 32*(w % 4)..+31, so a thread is one output channel; it converts the 64
-    // contraction elements of the stage (two units of 32 columns) and stores them as
-    // 32 tensor-memory columns.
-    const int grp = (warp - 8) >> 2;
-    const int q4 = warp & 3;
-    const int row = q4 * 32 + lane;
-    const uint32_t full_a_leader0 = mapa_shared(smem_u32(&bars->full_a[0]), 0);
+  } else if (warp >= 12) {
+    // ------------------------------------------ weight dequant (this CTA's 128 channels)
+    // Group g (four warps) serves the stages with it % 4 == g.  A thread is one channel:
+    // it converts the 64 contraction elements of the stage (two units of 32 columns)
+    // and writes them as the channel's 128-byte row, 16-byte chunk c at position
+    // c ^ (row % 8) (the 128-byte swizzle).
+    const int grp = (warp - 12) >> 2;
+    const int row = ((warp - 12) & 3) * 32 + lane;
+    const int swz = row & 7;
+    const uint32_t full_w_leader0 = mapa_shared(smem_u32(&bars->full_w[0]), 0);
     const uint32_t total_it = (uint32_t)my_tiles * (uint32_t)p.k_blocks;
     // cursor of the stage whose (s, z) is being prefetched, walked without divisions
     int pf_tile = pair, pf_kb = grp;
     while (pf_kb >= p.k_blocks) { pf_kb -= p.k_blocks; pf_tile += n_pairs; }
-    int pf_r = (pf_tile % p.r_tiles) * (2 * PM) + (int)rank * PM + row;
+    int pf_r = (pf_tile % p.n_tiles) * 256 + (int)rank * 128 + row;
     auto load_zs = [&](uint32_t (&z)[2], float (&sc)[2]) {
 #pragma unroll
       for (int u = 0; u < 2; ++u) {
         z[u] = 0u;
         sc[u] = 0.0f;
-        if (pf_r < p.N) {
-          const size_t gi = (size_t)pf_r * p.G + pair_group_of(p, pf_kb * PK + 32 * u);
+        const int col = pf_kb * PK + 32 * u;
+        if (pf_r < p.N && col < p.K) {
+          const size_t gi = (size_t)pf_r * p.G + pair_group_of(p, col);
           z[u] = __ldg(p.zeros + gi);
           if (FOLD) sc[u] = __ldg(p.scales + gi);
         }
@@ -248,7 +278,7 @@ qfwd_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
       while (pf_kb >= p.k_blocks) {
         pf_kb -= p.k_blocks;
         pf_tile += n_pairs;
-        pf_r = (pf_tile % p.r_tiles) * (2 * PM) + (int)rank * PM + row;
+        pf_r = (pf_tile % p.n_tiles) * 256 + (int)rank * 128 + row;
       }
     };
     uint32_t z[2], zn[2];
@@ -259,11 +289,11 @@ qfwd_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
       const int next_kb = pf_kb;
       if (it + P_GROUPS < total_it) load_zs(zn, scn);
       const int s = it % PSTAGES;
-      const uint32_t ph = (it / PSTAGES) & 1u;
-      if (!mbar_wait(smem_u32(&bars->pk_full[s]), ph, abort_flag)) break;
+      const int q = it % PQ_SLOTS;
+      if (!mbar_wait(smem_u32(&bars->pk_full[q]), (it / PQ_SLOTS) & 1u, abort_flag)) break;
       uint32_t w[2][BITS];
       {
-        const uint32_t* src = reinterpret_cast<const uint32_t*>(sm_q + s * PQ_BYTES) + row * 8;
+        const uint32_t* src = reinterpret_cast<const uint32_t*>(sm_q + q * PQ_BYTES) + row * 8;
         const uint4 lo = *reinterpret_cast<const uint4*>(src);
         const uint4 hi = *reinterpret_cast<const uint4*>(src + 4);
         const uint32_t w8[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
@@ -279,23 +309,24 @@ qfwd_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
           }
         }
       }
-      uint32_t o[32];
-      {
-        uint32_t o0[16], o1[16];
-        dq::unit32_natural<BITS, FOLD>(w[0], z[0], sc[0], o0);
-        dq::unit32_natural<BITS, FOLD>(w[1], z[1], sc[1], o1);
+      uint32_t o0[16], o1[16];
+      dq::unit32_natural<BITS, FOLD>(w[0], z[0], sc[0], o0);
+      dq::unit32_natural<BITS, FOLD>(w[1], z[1], sc[1], o1);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&bars->pk_empty[q]));   // codes consumed: slot free
+      if (!mbar_wait_cluster(smem_u32(&bars->empty[s]), ((it / PSTAGES) & 1u) ^ 1u, abort_flag)) break;
+      uint8_t* wrow = base + s * PSTAGE_BYTES + PA_BYTES + row * 128;
 #pragma unroll
-        for (int e = 0; e < 16; ++e) { o[e] = o0[e]; o[16 + e] = o1[e]; }
+      for (int c = 0; c < 4; ++c) {
+        *reinterpret_cast<uint4*>(wrow + ((c ^ swz) << 4)) =
+            make_uint4(o0[4 * c], o0[4 * c + 1], o0[4 * c + 2], o0[4 * c + 3]);
+        *reinterpret_cast<uint4*>(wrow + (((4 + c) ^ swz) << 4)) =
+            make_uint4(o1[4 * c], o1[4 * c + 1], o1[4 * c + 2], o1[4 * c + 3]);
       }
+      // make the rows visible to the tensor cores of both CTAs, then tell the leader
+      fence_proxy_async_smem();
       __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&bars->pk_empty[s]));   // codes consumed: slot free
-      if (!mbar_wait_cluster(smem_u32(&bars->empty[s]), ph ^ 1u, abort_flag)) break;
-      tc_fence_after();
-      tmem_st_32x32(tmem_base + ((uint32_t)(q4 * 32) << 16) + P_A_COL + s * (PK / 2), o);
-      tmem_st_wait();
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive_cluster(full_a_leader0 + s * 8);
+      if (lane == 0) mbar_arrive_cluster_release(full_w_leader0 + s * 8);
       z[0] = zn[0]; z[1] = zn[1];
       sc[0] = scn[0]; sc[1] = scn[1];
       cur_kb = next_kb;
@@ -380,9 +411,9 @@ int launch_fwd_pair(const peqa_qweight_t* w, int g, const void* X, int T, void* 
   for (int b = 5; b < 31; ++b)
     if ((1 << b) == g) p.g_shift = b;
   p.T = T;
-  p.r_tiles = (p.N + 2 * PM - 1) / (2 * PM);
-  p.t_tiles = (T + PN - 1) / PN;
-  p.k_blocks = p.K / PK;
+  p.n_tiles = (p.N + 255) / 256;
+  p.t_tiles = (T + 511) / 512;
+  p.k_blocks = (p.K + PK - 1) / PK;
   PEQA_TRY(status_word(&p.status));
   EncodeTiledFn enc = nullptr;
   PEQA_TRY(encode_fn(&enc));
@@ -390,7 +421,7 @@ int launch_fwd_pair(const peqa_qweight_t* w, int g, const void* X, int T, void* 
   {
     cuuint64_t dims[2] = {(cuuint64_t)p.K, (cuuint64_t)T};
     cuuint64_t strides[1] = {(cuuint64_t)p.K * 2};
-    cuuint32_t box[2] = {64, PN / 2};
+    cuuint32_t box[2] = {64, 128};
     cuuint32_t estr[2] = {1, 1};
     if (enc(&tx, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(X), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -401,7 +432,7 @@ int launch_fwd_pair(const peqa_qweight_t* w, int g, const void* X, int T, void* 
     const int wpr = p.K * w->bits / 32;
     cuuint64_t dims[2] = {(cuuint64_t)wpr, (cuuint64_t)p.N};
     cuuint64_t strides[1] = {(cuuint64_t)wpr * 4};
-    cuuint32_t box[2] = {8, PM};
+    cuuint32_t box[2] = {8, 128};
     cuuint32_t estr[2] = {1, 1};
     if (enc(&tq, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<uint32_t*>(w->qweight), dims, strides,
             box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
@@ -411,7 +442,7 @@ int launch_fwd_pair(const peqa_qweight_t* w, int g, const void* X, int T, void* 
   int sms = 0, dev = 0;
   PEQA_CUDA(cudaGetDevice(&dev));
   PEQA_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-  const int tiles = p.r_tiles * p.t_tiles;
+  const int tiles = p.n_tiles * p.t_tiles;
   const int max_pairs = sms / 2;
   const int pairs = tiles < max_pairs ? tiles : max_pairs;
   const bool fold = p.G > 1;

@@ -51,6 +51,14 @@ def test_in_features_not_a_multiple_of_128(bits, g):
         _run_all(d, bits, g)
 
 
+@pytest.mark.parametrize("g", [0, 64, 192])
+def test_token_tail_beyond_one_block(g):
+    # T = 530 leaves 18 tokens in the second 512-token tile; T = 300 fills a block and a bit
+    for T, K in ((530, 192 if g == 192 else 320), (300, 384)):
+        d = synth.custom(300 + g + T, 264, K, T, 4, g, outliers=True, sigma_dy=1e-2)
+        _run_all(d, 4, g)
+
+
 @pytest.mark.parametrize("T", [1, 7, 64, 257, 513])
 def test_token_counts(T):
     d = synth.custom(T, 256, 512, T, 3, 128, sigma_dy=1e-2)
