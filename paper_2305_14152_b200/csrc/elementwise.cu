@@ -41,26 +41,73 @@ __device__ __forceinline__ uint32_t warp_unpack(const uint32_t* src, int lane) {
   return v & ((1u << BITS) - 1u);
 }
 
-// rint(fl(w / s)) with fl() the correctly rounded binary32 quotient.  The product
-// w * (1/s) is within a few ulps of that quotient, so both round to the same
-// integer unless the product sits within a few ulps of a half-integer; only then
-// (or when the product is huge or not finite) is the IEEE division carried out.
-__device__ __forceinline__ float rint_of_quotient(float w, float s, float rs) {
-  const float t = __fmul_rn(w, rs);
-  float k = rintf(t);
-  const float dist = fabsf(__fsub_rn(fabsf(__fsub_rn(t, k)), 0.5f));
-  if (!(fabsf(t) <= 4.0e6f) || dist <= __fmul_rn(fabsf(t), 2.0e-6f)) k = rintf(__fdiv_rn(w, s));
-  return k;
+// Codes of eight consecutive columns of one group, as BITS-wide fields of a word
+// (column e at bits [BITS*e, BITS*e + BITS)).
+//
+// Reference arithmetic (Eq. 1 in binary32): q = clamp(rint(fl(w / s)) + z, 0, qmax).
+// Fast path, same result without a division or a float->int conversion per element:
+//   t  = fl(w * fl(1/s))           within 3 ulp of fl(w / s)
+//   tc = clamp(t, -z - 1/4, qmax - z + 1/4)   rint(tc) + z lands in [0, qmax] and equals
+//                                  the clamped reference whenever rint(t) == rint(fl(w/s))
+//   k  = (tc + 1.5*2^23) - 1.5*2^23           = rint(tc), ties to even, since |tc| < 2^22
+//   word_f += k * 2^(BITS*e)       exact: the fields fill at most 24 bits of an fp32
+// rint(t) can differ from rint(fl(w/s)) only if a half-integer lies within 3 ulp of t
+// (|t| <= 16.25 inside the clamp, so 3 ulp < 6e-6).  The run keeps the smallest distance
+// to a half-integer it has seen; if that is below 1e-5, or 1/s is not a normal number of
+// moderate size, the eight codes are recomputed with the IEEE division.
+template <int BITS>
+__device__ __forceinline__ uint32_t quantize_run8(const float (&x)[8], float s, float z) {
+  constexpr float kMagic = 12582912.0f;   // 1.5 * 2^23
+  const float qmax = (float)((1 << BITS) - 1);
+  const float rs = __frcp_rn(s);
+  const float lo = __fsub_rn(-0.25f, z);
+  const float hi = __fadd_rn(__fsub_rn(qmax, z), 0.25f);
+  float near = 1.0f;
+  uint32_t word;
+  if constexpr (BITS == 3) {
+    float acc = __fmul_rn(z, 2396745.0f);                 // z * sum_e 8^e
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      const float tc = fminf(fmaxf(__fmul_rn(x[e], rs), lo), hi);
+      const float k = __fsub_rn(__fadd_rn(tc, kMagic), kMagic);
+      near = fminf(near, fabsf(__fsub_rn(fabsf(__fsub_rn(tc, k)), 0.5f)));
+      acc = __fmaf_rn(k, (float)(1 << (3 * e)), acc);
+    }
+    word = (uint32_t)acc;
+  } else {
+    float acc0 = __fmul_rn(z, 4369.0f), acc1 = acc0;      // z * sum_{e<4} 16^e
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      const float tc = fminf(fmaxf(__fmul_rn(x[e], rs), lo), hi);
+      const float k = __fsub_rn(__fadd_rn(tc, kMagic), kMagic);
+      near = fminf(near, fabsf(__fsub_rn(fabsf(__fsub_rn(tc, k)), 0.5f)));
+      if (e < 4) acc0 = __fmaf_rn(k, (float)(1 << (4 * e)), acc0);
+      else acc1 = __fmaf_rn(k, (float)(1 << (4 * (e - 4))), acc1);
+    }
+    word = (uint32_t)acc0 | ((uint32_t)acc1 << 16);
+  }
+  if (!(near > 1.0e-5f) || !(rs <= 1.0e30f)) {
+    word = 0u;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      float q = __fadd_rn(rintf(__fdiv_rn(x[e], s)), z);
+      q = fminf(fmaxf(q, 0.0f), qmax);
+      word |= (uint32_t)q << (BITS * e);
+    }
+  }
+  return word;
 }
 
 // One CTA per output row; a thread works on runs of 8 consecutive columns, so
-// a 32-column chunk is 4 adjacent lanes.  Pass 1: min/max per chunk.  Pass 2:
-// per group (s, z) in strict binary32 (division and rounding as single IEEE
-// operations, no FMA).  Pass 3: codes (second read of the row, served by L1/L2)
-// and packing: eight 4-bit codes are exactly one word; eight 3-bit codes are 24
-// bits, and lanes 0..2 of a 4-lane chunk assemble the three words from their
-// own and their right neighbour's piece.
-template <int BITS>
+// a 32-column chunk is 4 adjacent lanes.  Pass 1: read the row (kept in
+// registers when RUNS > 0: run r of a thread is columns 8*(threadIdx.x +
+// r*256)..+7, which covers K <= 2048*RUNS), min/max per chunk.  Pass 2: per
+// group (s, z) in strict binary32 (division and rounding as single IEEE
+// operations, no FMA).  Pass 3: codes and packing: eight 4-bit codes are exactly
+// one word; eight 3-bit codes are 24 bits, and lanes 0..2 of a 4-lane chunk
+// assemble the three words from their own and their right neighbour's piece.
+// RUNS == 0 reads the row a second time in pass 3 instead (any K).
+template <int BITS, int RUNS>
 __global__ void __launch_bounds__(kQuantThreads)
 quantize_rtn_kernel(const float* __restrict__ W, int K, int g, int cpg_shift,
                     uint32_t* __restrict__ qweight, uint8_t* __restrict__ zeros,
@@ -78,15 +125,13 @@ quantize_rtn_kernel(const float* __restrict__ W, int K, int g, int cpg_shift,
   const int cpg = g >> 5;  // chunks per group
   const float4* w4 = reinterpret_cast<const float4*>(W + (size_t)row * K);
   const float qmax = (float)((1 << BITS) - 1);
+  constexpr int NR = RUNS > 0 ? RUNS : 1;
+  float4 ra[NR], rb[NR];
 
   // Every thread runs the same number of iterations (the shuffles name the whole
   // warp); runs past the end of the row are predicated off.  nv8 is a multiple of 4,
   // so the 4 lanes of a chunk are all in or all out.
-  for (int vb = 0; vb < nv8; vb += kQuantThreads) {
-    const int v = vb + threadIdx.x;
-    const bool in = v < nv8;
-    float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
-    if (in) { a = __ldg(w4 + 2 * v); b = __ldg(w4 + 2 * v + 1); }
+  auto minmax_run = [&](int v, bool in, const float4& a, const float4& b) {
     float mn = fminf(fminf(fminf(a.x, a.y), fminf(a.z, a.w)), fminf(fminf(b.x, b.y), fminf(b.z, b.w)));
     float mx = fmaxf(fmaxf(fmaxf(a.x, a.y), fmaxf(a.z, a.w)), fmaxf(fmaxf(b.x, b.y), fmaxf(b.z, b.w)));
 #pragma unroll
@@ -95,6 +140,28 @@ quantize_rtn_kernel(const float* __restrict__ W, int K, int g, int cpg_shift,
       mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
     }
     if (in && (lane & 3) == 0) { cmin[v >> 2] = mn; cmax[v >> 2] = mx; }
+  };
+  if constexpr (RUNS > 0) {
+#pragma unroll
+    for (int r = 0; r < RUNS; ++r) {
+      const int v = r * kQuantThreads + threadIdx.x;
+      ra[r] = make_float4(0.f, 0.f, 0.f, 0.f);
+      rb[r] = ra[r];
+      if (v < nv8) { ra[r] = __ldg(w4 + 2 * v); rb[r] = __ldg(w4 + 2 * v + 1); }
+    }
+#pragma unroll
+    for (int r = 0; r < RUNS; ++r) {
+      const int v = r * kQuantThreads + threadIdx.x;
+      minmax_run(v, v < nv8, ra[r], rb[r]);
+    }
+  } else {
+    for (int vb = 0; vb < nv8; vb += kQuantThreads) {
+      const int v = vb + threadIdx.x;
+      const bool in = v < nv8;
+      float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
+      if (in) { a = __ldg(w4 + 2 * v); b = __ldg(w4 + 2 * v + 1); }
+      minmax_run(v, in, a, b);
+    }
   }
   __syncthreads();
 
@@ -137,23 +204,11 @@ quantize_rtn_kernel(const float* __restrict__ W, int K, int g, int cpg_shift,
   __syncthreads();
 
   uint32_t* qrow = qweight + (size_t)row * chunks * BITS;
-  for (int vb = 0; vb < nv8; vb += kQuantThreads) {
-    const int v = vb + threadIdx.x;
-    const bool in = v < nv8;
-    float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
-    if (in) { a = __ldg(w4 + 2 * v); b = __ldg(w4 + 2 * v + 1); }
+  auto emit_run = [&](int v, bool in, const float4& a, const float4& b) {
     const int chunk = in ? (v >> 2) : 0;
     const int gi = cpg_shift >= 0 ? (chunk >> cpg_shift) : (chunk / cpg);
-    const float s = gscale[gi], z = gzero[gi];
-    const float rs = __frcp_rn(s);
     const float xs[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
-    uint32_t piece = 0u;
-#pragma unroll
-    for (int e = 0; e < 8; ++e) {
-      float q = __fadd_rn(rint_of_quotient(xs[e], s, rs), z);
-      q = fminf(fmaxf(q, 0.0f), qmax);
-      piece |= (uint32_t)q << (BITS * e);
-    }
+    const uint32_t piece = quantize_run8<BITS>(xs, gscale[gi], gzero[gi]);
     if constexpr (BITS == 4) {
       if (in) qrow[v] = piece;
     } else {
@@ -162,6 +217,21 @@ quantize_rtn_kernel(const float* __restrict__ W, int K, int g, int cpg_shift,
       const int j = lane & 3;
       const uint32_t word = (piece >> (8 * j)) | (nextp << (24 - 8 * j));
       if (in && j < 3) qrow[chunk * 3 + j] = word;
+    }
+  };
+  if constexpr (RUNS > 0) {
+#pragma unroll
+    for (int r = 0; r < RUNS; ++r) {
+      const int v = r * kQuantThreads + threadIdx.x;
+      emit_run(v, v < nv8, ra[r], rb[r]);
+    }
+  } else {
+    for (int vb = 0; vb < nv8; vb += kQuantThreads) {
+      const int v = vb + threadIdx.x;
+      const bool in = v < nv8;
+      float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
+      if (in) { a = __ldg(w4 + 2 * v); b = __ldg(w4 + 2 * v + 1); }
+      emit_run(v, in, a, b);
     }
   }
 }
@@ -233,10 +303,28 @@ extern "C" int peqa_quantize_rtn(const float* W, int N, int K, int bits, int gro
   int cpg_shift = -1;
   for (int b = 0; b < 26; ++b)
     if ((32 << b) == g) cpg_shift = b;
-  if (bits == 4)
-    quantize_rtn_kernel<4><<<N, kQuantThreads, 0, st>>>(W, K, g, cpg_shift, qweight, zeros, scales);
-  else
-    quantize_rtn_kernel<3><<<N, kQuantThreads, 0, st>>>(W, K, g, cpg_shift, qweight, zeros, scales);
+  // rows up to 2048 * RUNS columns stay in registers between the passes
+  const int runs = K <= 4096 ? 2 : K <= 8192 ? 4 : K <= 12288 ? 6 : K <= 24576 ? 12 : 0;
+#define PEQA_QUANT_LAUNCH(B, R) \
+  quantize_rtn_kernel<B, R><<<N, kQuantThreads, 0, st>>>(W, K, g, cpg_shift, qweight, zeros, scales)
+  if (bits == 4) {
+    switch (runs) {
+      case 2: PEQA_QUANT_LAUNCH(4, 2); break;
+      case 4: PEQA_QUANT_LAUNCH(4, 4); break;
+      case 6: PEQA_QUANT_LAUNCH(4, 6); break;
+      case 12: PEQA_QUANT_LAUNCH(4, 12); break;
+      default: PEQA_QUANT_LAUNCH(4, 0); break;
+    }
+  } else {
+    switch (runs) {
+      case 2: PEQA_QUANT_LAUNCH(3, 2); break;
+      case 4: PEQA_QUANT_LAUNCH(3, 4); break;
+      case 6: PEQA_QUANT_LAUNCH(3, 6); break;
+      case 12: PEQA_QUANT_LAUNCH(3, 12); break;
+      default: PEQA_QUANT_LAUNCH(3, 0); break;
+    }
+  }
+#undef PEQA_QUANT_LAUNCH
   PEQA_CUDA(cudaGetLastError());
   return PEQA_OK;
 }

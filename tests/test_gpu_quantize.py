@@ -61,6 +61,57 @@ def test_degenerate_rows():
 
 
 @pytest.mark.parametrize("bits", [3, 4])
+def test_quotients_at_and_next_to_ties(bits):
+    """Rows whose quotients w/s sit on half-integers or a few ulps beside them: the
+    rounding decision must be the one of the correctly rounded binary32 division."""
+    qmax = (1 << bits) - 1
+    rng = np.random.default_rng(40 + bits)
+    K = 512
+    rows = []
+    for step in (1.0, 0.5, 0.1, 0.3, 1e-3, 7.7, 3e-5, 1234.5):
+        s = np.float32(step)
+        k = rng.integers(0, qmax, size=K).astype(np.float32)
+        x = ((k + np.float32(0.5)) * s).astype(np.float32)
+        # walk up to 3 representable numbers to either side
+        for _ in range(3):
+            up = rng.integers(0, 3, size=K)
+            toward = np.where(up == 1, np.float32(np.inf), np.float32(-np.inf)).astype(np.float32)
+            x = np.where(up == 0, x, np.nextafter(x, toward)).astype(np.float32)
+        for shift in (0.0, -2.0 * step, 3.0 * step):
+            r = (x + np.float32(shift)).astype(np.float32)
+            # pin the group's range so that s is `step` (up to rounding) in every 32-column group
+            r[0::32] = np.float32(shift)
+            r[1::32] = np.float32(shift) + np.float32(qmax) * s
+            rows.append(r)
+    W = np.stack(rows).astype(np.float32)
+    for g in (0, 32, 128):
+        _compare(W, bits, g)
+
+
+def test_tiny_and_subnormal_scales():
+    K = 256
+    W = np.zeros((6, K), np.float32)
+    j = np.arange(K, dtype=np.float64)
+    W[0] = (1e-39 * j).astype(np.float32)                 # subnormal weights, subnormal scale
+    W[1] = (1e-36 * np.sin(j)).astype(np.float32)         # 1/s beyond 1e30
+    W[2] = (3e-31 * np.cos(j)).astype(np.float32)
+    W[3] = np.float32(1000.0) + (1e-4 * (j % 7)).astype(np.float32)   # large |w/s|
+    W[4] = np.float32(-5e4) + (2e-3 * (j % 5)).astype(np.float32)
+    # the smallest range whose scale does not round to zero (below it Eq. 1 divides by 0)
+    W[5, ::2] = np.float32(3e-44)
+    for bits in (3, 4):
+        for g in (0, 32):
+            _compare(W, bits, g)
+
+
+@pytest.mark.parametrize("K", [8192, 12288, 24576, 24704, 32768])
+def test_row_lengths_across_the_register_budgets(K):
+    d = synth.custom(K, 24, K, 1, 3, 128, outliers=True)
+    _compare(d["W"], 3, 128)
+    _compare(d["W"][:8], 4, 0)
+
+
+@pytest.mark.parametrize("bits", [3, 4])
 def test_pack_unpack_random_codes(bits):
     rng = np.random.default_rng(bits)
     codes = rng.integers(0, 1 << bits, size=(77, 1056), dtype=np.uint8)
