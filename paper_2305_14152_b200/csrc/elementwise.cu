@@ -41,52 +41,83 @@ __device__ __forceinline__ uint32_t warp_unpack(const uint32_t* src, int lane) {
   return v & ((1u << BITS) - 1u);
 }
 
-// Codes of eight consecutive columns of one group, as BITS-wide fields of a word
-// (column e at bits [BITS*e, BITS*e + BITS)).
-//
+__device__ __forceinline__ float min3(float a, float b, float c) {
+  float r;
+  asm("min.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float r;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
+}
+
+// Per-group constants of the fast quantization path, written once per group.
+struct GroupConst {
+  float rs;   // fl(1/s), or NaN when the group must take the division path
+  float zc;   // z * sum of the field weights (the accumulator's start value)
+};
+
 // Reference arithmetic (Eq. 1 in binary32): q = clamp(rint(fl(w / s)) + z, 0, qmax).
-// Fast path, same result without a division or a float->int conversion per element:
-//   t  = fl(w * fl(1/s))           within 3 ulp of fl(w / s)
-//   tc = clamp(t, -z - 1/4, qmax - z + 1/4)   rint(tc) + z lands in [0, qmax] and equals
-//                                  the clamped reference whenever rint(t) == rint(fl(w/s))
-//   k  = (tc + 1.5*2^23) - 1.5*2^23           = rint(tc), ties to even, since |tc| < 2^22
-//   word_f += k * 2^(BITS*e)       exact: the fields fill at most 24 bits of an fp32
-// rint(t) can differ from rint(fl(w/s)) only if a half-integer lies within 3 ulp of t
-// (|t| <= 16.25 inside the clamp, so 3 ulp < 6e-6).  The run keeps the smallest distance
-// to a half-integer it has seen; if that is below 1e-5, or 1/s is not a normal number of
-// moderate size, the eight codes are recomputed with the IEEE division.
+// The fast path computes t = fl(w * fl(1/s)), which is within 3 ulp of fl(w / s), and
+// rounds it without a clamp.  That is only right for a group in which no code needs
+// the clamp: t is monotone in w, so it is enough that the group's extremes satisfy
+// -z - 1/2 < t(min) and t(max) < qmax - z + 1/2 (with a margin of 1e-5).  Groups that
+// fail (all weights of one sign, so that z itself was clamped; an extreme next to a
+// tie), and groups whose 1/s is not a normal number of moderate size, get rs = NaN.
 template <int BITS>
-__device__ __forceinline__ uint32_t quantize_run8(const float (&x)[8], float s, float z) {
-  constexpr float kMagic = 12582912.0f;   // 1.5 * 2^23
+__device__ __forceinline__ GroupConst group_const(float mn, float mx, float s, float z) {
   const float qmax = (float)((1 << BITS) - 1);
-  const float rs = __frcp_rn(s);
-  const float lo = __fsub_rn(-0.25f, z);
-  const float hi = __fadd_rn(__fsub_rn(qmax, z), 0.25f);
-  float near = 1.0f;
+  GroupConst c;
+  c.rs = __frcp_rn(s);
+  const float t_lo = __fmul_rn(mn, c.rs), t_hi = __fmul_rn(mx, c.rs);
+  const bool ok = c.rs <= 1.0e30f && t_lo > __fsub_rn(-0.49999f, z) &&
+                  t_hi < __fadd_rn(__fsub_rn(qmax, z), 0.49999f);
+  if (!ok) c.rs = __int_as_float(0x7fc00000);
+  c.zc = __fmul_rn(z, BITS == 3 ? 2396745.0f : 4369.0f);   // sum_{e<8} 8^e, sum_{e<4} 16^e
+  return c;
+}
+
+// Codes of eight consecutive columns of one group, as BITS-wide fields of a word
+// (column e at bits [BITS*e, BITS*e + BITS)).  Fast path, per element:
+//   t  = fl(w * rs)
+//   k  = (t + 1.5*2^23) - 1.5*2^23   = rint(t), ties to even, since |t| < 2^22
+//   word_f += k * 2^(BITS*e)         exact: the fields fill at most 24 bits of an fp32,
+//                                    and word_f starts at z in every field
+// rint(t) can differ from rint(fl(w/s)) only if a half-integer lies within 3 ulp of t
+// (|t| <= 16.5 in a group that passed group_const, so 3 ulp < 6e-6).  The run keeps the
+// largest |t - k| it has seen; if that is not below 1/2 - 1e-5, or the group's rs is
+// NaN, the eight codes are recomputed with the IEEE division and the clamp.
+template <int BITS>
+__device__ __forceinline__ uint32_t quantize_run8(const float (&x)[8], float s, float z,
+                                                  const GroupConst& c) {
+  constexpr float kMagic = 12582912.0f;   // 1.5 * 2^23
+  float k[8], r[8];
+#pragma unroll
+  for (int e = 0; e < 8; ++e) {
+    const float t = __fmul_rn(x[e], c.rs);
+    k[e] = __fsub_rn(__fadd_rn(t, kMagic), kMagic);
+    r[e] = fabsf(__fsub_rn(t, k[e]));
+  }
+  const float far = max3(max3(r[0], r[1], r[2]), max3(r[3], r[4], r[5]), fmaxf(r[6], r[7]));
   uint32_t word;
   if constexpr (BITS == 3) {
-    float acc = __fmul_rn(z, 2396745.0f);                 // z * sum_e 8^e
+    float acc = c.zc;
 #pragma unroll
-    for (int e = 0; e < 8; ++e) {
-      const float tc = fminf(fmaxf(__fmul_rn(x[e], rs), lo), hi);
-      const float k = __fsub_rn(__fadd_rn(tc, kMagic), kMagic);
-      near = fminf(near, fabsf(__fsub_rn(fabsf(__fsub_rn(tc, k)), 0.5f)));
-      acc = __fmaf_rn(k, (float)(1 << (3 * e)), acc);
-    }
+    for (int e = 0; e < 8; ++e) acc = __fmaf_rn(k[e], (float)(1 << (3 * e)), acc);
     word = (uint32_t)acc;
   } else {
-    float acc0 = __fmul_rn(z, 4369.0f), acc1 = acc0;      // z * sum_{e<4} 16^e
+    float acc0 = c.zc, acc1 = c.zc;
 #pragma unroll
-    for (int e = 0; e < 8; ++e) {
-      const float tc = fminf(fmaxf(__fmul_rn(x[e], rs), lo), hi);
-      const float k = __fsub_rn(__fadd_rn(tc, kMagic), kMagic);
-      near = fminf(near, fabsf(__fsub_rn(fabsf(__fsub_rn(tc, k)), 0.5f)));
-      if (e < 4) acc0 = __fmaf_rn(k, (float)(1 << (4 * e)), acc0);
-      else acc1 = __fmaf_rn(k, (float)(1 << (4 * (e - 4))), acc1);
+    for (int e = 0; e < 4; ++e) {
+      acc0 = __fmaf_rn(k[e], (float)(1 << (4 * e)), acc0);
+      acc1 = __fmaf_rn(k[4 + e], (float)(1 << (4 * e)), acc1);
     }
     word = (uint32_t)acc0 | ((uint32_t)acc1 << 16);
   }
-  if (!(near > 1.0e-5f) || !(rs <= 1.0e30f)) {
+  // max drops a NaN operand, so a NaN rs has to be tested on its own
+  if (!(far < 0.49999f) || c.rs != c.rs) {
+    const float qmax = (float)((1 << BITS) - 1);
     word = 0u;
 #pragma unroll
     for (int e = 0; e < 8; ++e) {
@@ -98,42 +129,54 @@ __device__ __forceinline__ uint32_t quantize_run8(const float (&x)[8], float s, 
   return word;
 }
 
-// One CTA per output row; a thread works on runs of 8 consecutive columns, so
-// a 32-column chunk is 4 adjacent lanes.  Pass 1: read the row (kept in
-// registers when RUNS > 0: run r of a thread is columns 8*(threadIdx.x +
-// r*256)..+7, which covers K <= 2048*RUNS), min/max per chunk.  Pass 2: per
-// group (s, z) in strict binary32 (division and rounding as single IEEE
-// operations, no FMA).  Pass 3: codes and packing: eight 4-bit codes are exactly
-// one word; eight 3-bit codes are 24 bits, and lanes 0..2 of a 4-lane chunk
-// assemble the three words from their own and their right neighbour's piece.
-// RUNS == 0 reads the row a second time in pass 3 instead (any K).
-template <int BITS, int RUNS>
+// A CTA takes rows blockIdx.x, blockIdx.x + gridDim.x, ...; a thread works on
+// runs of 8 consecutive columns, so a 32-column chunk is 4 adjacent lanes.
+// Pass 1: min/max per chunk of the row (kept in registers when RUNS > 0: run r
+// of a thread is columns 8*(threadIdx.x + r*256)..+7, which covers K <=
+// 2048*RUNS).  Pass 2: per group (s, z) in strict binary32 (division and
+// rounding as single IEEE operations, no FMA).  Pass 3: codes and packing:
+// eight 4-bit codes are exactly one word; eight 3-bit codes are 24 bits, and
+// lanes 0..2 of a 4-lane chunk assemble the three words from their own and
+// their right neighbour's piece.  With PREFETCH the loads of the CTA's next
+// row are issued before pass 1 of the current one, so that the memory system
+// stays busy while the row is being reduced and encoded.  RUNS == 0 reads the
+// row a second time in pass 3 instead (any K).
+template <int BITS, int RUNS, bool PREFETCH>
 __global__ void __launch_bounds__(kQuantThreads)
-quantize_rtn_kernel(const float* __restrict__ W, int K, int g, int cpg_shift,
+quantize_rtn_kernel(const float* __restrict__ W, int N, int K, int g, int cpg_shift,
                     uint32_t* __restrict__ qweight, uint8_t* __restrict__ zeros,
                     float* __restrict__ scales) {
-  __shared__ float cmin[kMaxChunks];
-  __shared__ float cmax[kMaxChunks];
-  __shared__ float gscale[kMaxChunks];
-  __shared__ float gzero[kMaxChunks];
-
-  const int row = blockIdx.x;
+  extern __shared__ __align__(16) uint8_t quant_smem[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int chunks = K >> 5;
   const int nv8 = K >> 3;
   const int G = K / g;
+  GroupConst* gconst = reinterpret_cast<GroupConst*>(quant_smem);          // [G]
+  float* gscale = reinterpret_cast<float*>(gconst + G);                    // [G]
+  float* gzero = gscale + G;                                               // [G]
+  float* cmin = gzero + G;                                                 // [chunks]
+  float* cmax = cmin + chunks;                                             // [chunks]
   const int cpg = g >> 5;  // chunks per group
-  const float4* w4 = reinterpret_cast<const float4*>(W + (size_t)row * K);
   const float qmax = (float)((1 << BITS) - 1);
   constexpr int NR = RUNS > 0 ? RUNS : 1;
-  float4 ra[NR], rb[NR];
 
+  auto row_ptr = [&](int row) { return reinterpret_cast<const float4*>(W + (size_t)row * K); };
+  auto load_row = [&](int row, float4 (&a)[NR], float4 (&b)[NR]) {
+    const float4* w4 = row_ptr(row);
+#pragma unroll
+    for (int r = 0; r < NR; ++r) {
+      const int v = r * kQuantThreads + threadIdx.x;
+      a[r] = make_float4(0.f, 0.f, 0.f, 0.f);
+      b[r] = a[r];
+      if (row < N && v < nv8) { a[r] = __ldg(w4 + 2 * v); b[r] = __ldg(w4 + 2 * v + 1); }
+    }
+  };
   // Every thread runs the same number of iterations (the shuffles name the whole
   // warp); runs past the end of the row are predicated off.  nv8 is a multiple of 4,
   // so the 4 lanes of a chunk are all in or all out.
   auto minmax_run = [&](int v, bool in, const float4& a, const float4& b) {
-    float mn = fminf(fminf(fminf(a.x, a.y), fminf(a.z, a.w)), fminf(fminf(b.x, b.y), fminf(b.z, b.w)));
-    float mx = fmaxf(fmaxf(fmaxf(a.x, a.y), fmaxf(a.z, a.w)), fmaxf(fmaxf(b.x, b.y), fmaxf(b.z, b.w)));
+    float mn = min3(min3(a.x, a.y, a.z), min3(a.w, b.x, b.y), fminf(b.z, b.w));
+    float mx = max3(max3(a.x, a.y, a.z), max3(a.w, b.x, b.y), fmaxf(b.z, b.w));
 #pragma unroll
     for (int o = 2; o > 0; o >>= 1) {
       mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
@@ -141,97 +184,120 @@ quantize_rtn_kernel(const float* __restrict__ W, int K, int g, int cpg_shift,
     }
     if (in && (lane & 3) == 0) { cmin[v >> 2] = mn; cmax[v >> 2] = mx; }
   };
-  if constexpr (RUNS > 0) {
-#pragma unroll
-    for (int r = 0; r < RUNS; ++r) {
-      const int v = r * kQuantThreads + threadIdx.x;
-      ra[r] = make_float4(0.f, 0.f, 0.f, 0.f);
-      rb[r] = ra[r];
-      if (v < nv8) { ra[r] = __ldg(w4 + 2 * v); rb[r] = __ldg(w4 + 2 * v + 1); }
-    }
-#pragma unroll
-    for (int r = 0; r < RUNS; ++r) {
-      const int v = r * kQuantThreads + threadIdx.x;
-      minmax_run(v, v < nv8, ra[r], rb[r]);
-    }
-  } else {
-    for (int vb = 0; vb < nv8; vb += kQuantThreads) {
-      const int v = vb + threadIdx.x;
-      const bool in = v < nv8;
-      float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
-      if (in) { a = __ldg(w4 + 2 * v); b = __ldg(w4 + 2 * v + 1); }
-      minmax_run(v, in, a, b);
-    }
-  }
-  __syncthreads();
 
-  auto finish_group = [&](int gi, float mn, float mx) {
-    float s = __fdiv_rn(__fsub_rn(mx, mn), qmax);
-    if (mx == mn) s = 1.0f;
-    float z = rintf(__fdiv_rn(-mn, s));
-    z = fminf(fmaxf(z, 0.0f), qmax);
-    gscale[gi] = s;
-    gzero[gi] = z;
-    scales[(size_t)row * G + gi] = s;
-    zeros[(size_t)row * G + gi] = (uint8_t)z;
-  };
-  if (cpg <= 32) {
-    // narrow groups: one thread per group
-    for (int gi = threadIdx.x; gi < G; gi += kQuantThreads) {
-      float mn = INFINITY, mx = -INFINITY;
-      for (int c = 0; c < cpg; ++c) {
-        mn = fminf(mn, cmin[gi * cpg + c]);
-        mx = fmaxf(mx, cmax[gi * cpg + c]);
-      }
-      finish_group(gi, mn, mx);
-    }
-  } else {
-    // wide groups (per-channel above all): one warp per group
-    for (int gi = warp; gi < G; gi += kQuantWarps) {
-      float mn = INFINITY, mx = -INFINITY;
-      for (int c = lane; c < cpg; c += 32) {
-        mn = fminf(mn, cmin[gi * cpg + c]);
-        mx = fmaxf(mx, cmax[gi * cpg + c]);
-      }
+  // One row, from the registers ra, rb (RUNS > 0) or from memory (RUNS == 0).
+  auto process_row = [&](int row, const float4 (&ra)[NR], const float4 (&rb)[NR]) {
+    const float4* w4 = row_ptr(row);
+    if constexpr (RUNS > 0) {
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
-        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+      for (int r = 0; r < RUNS; ++r) {
+        const int v = r * kQuantThreads + threadIdx.x;
+        minmax_run(v, v < nv8, ra[r], rb[r]);
       }
-      if (lane == 0) finish_group(gi, mn, mx);
-    }
-  }
-  __syncthreads();
-
-  uint32_t* qrow = qweight + (size_t)row * chunks * BITS;
-  auto emit_run = [&](int v, bool in, const float4& a, const float4& b) {
-    const int chunk = in ? (v >> 2) : 0;
-    const int gi = cpg_shift >= 0 ? (chunk >> cpg_shift) : (chunk / cpg);
-    const float xs[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
-    const uint32_t piece = quantize_run8<BITS>(xs, gscale[gi], gzero[gi]);
-    if constexpr (BITS == 4) {
-      if (in) qrow[v] = piece;
     } else {
-      // chunk = 96 bits = pieces p0..p3 of 24 bits: word j = (p_j >> 8j) | (p_{j+1} << (24 - 8j))
-      const uint32_t nextp = __shfl_down_sync(0xffffffffu, piece, 1);
-      const int j = lane & 3;
-      const uint32_t word = (piece >> (8 * j)) | (nextp << (24 - 8 * j));
-      if (in && j < 3) qrow[chunk * 3 + j] = word;
+      for (int vb = 0; vb < nv8; vb += kQuantThreads) {
+        const int v = vb + threadIdx.x;
+        const bool in = v < nv8;
+        float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
+        if (in) { a = __ldg(w4 + 2 * v); b = __ldg(w4 + 2 * v + 1); }
+        minmax_run(v, in, a, b);
+      }
     }
-  };
-  if constexpr (RUNS > 0) {
+    __syncthreads();
+
+    auto finish_group = [&](int gi, float mn, float mx) {
+      float s = __fdiv_rn(__fsub_rn(mx, mn), qmax);
+      if (mx == mn) s = 1.0f;
+      float z = rintf(__fdiv_rn(-mn, s));
+      z = fminf(fmaxf(z, 0.0f), qmax);
+      gscale[gi] = s;
+      gzero[gi] = z;
+      gconst[gi] = group_const<BITS>(mn, mx, s, z);
+      scales[(size_t)row * G + gi] = s;
+      zeros[(size_t)row * G + gi] = (uint8_t)z;
+    };
+    if (cpg <= 32) {
+      // narrow groups: one thread per group
+      for (int gi = threadIdx.x; gi < G; gi += kQuantThreads) {
+        float mn = INFINITY, mx = -INFINITY;
+        for (int c = 0; c < cpg; ++c) {
+          mn = fminf(mn, cmin[gi * cpg + c]);
+          mx = fmaxf(mx, cmax[gi * cpg + c]);
+        }
+        finish_group(gi, mn, mx);
+      }
+    } else {
+      // wide groups (per-channel above all): one warp per group
+      for (int gi = warp; gi < G; gi += kQuantWarps) {
+        float mn = INFINITY, mx = -INFINITY;
+        for (int c = lane; c < cpg; c += 32) {
+          mn = fminf(mn, cmin[gi * cpg + c]);
+          mx = fmaxf(mx, cmax[gi * cpg + c]);
+        }
 #pragma unroll
-    for (int r = 0; r < RUNS; ++r) {
-      const int v = r * kQuantThreads + threadIdx.x;
-      emit_run(v, v < nv8, ra[r], rb[r]);
+        for (int o = 16; o > 0; o >>= 1) {
+          mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        }
+        if (lane == 0) finish_group(gi, mn, mx);
+      }
+    }
+    __syncthreads();
+
+    uint32_t* qrow = qweight + (size_t)row * chunks * BITS;
+    auto emit_run = [&](int v, bool in, const float4& a, const float4& b) {
+      const int chunk = in ? (v >> 2) : 0;
+      const int gi = cpg_shift >= 0 ? (chunk >> cpg_shift) : (chunk / cpg);
+      const float xs[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+      const uint32_t piece = quantize_run8<BITS>(xs, gscale[gi], gzero[gi], gconst[gi]);
+      if constexpr (BITS == 4) {
+        if (in) qrow[v] = piece;
+      } else {
+        // chunk = 96 bits = pieces p0..p3 of 24 bits: word j = (p_j >> 8j) | (p_{j+1} << (24 - 8j))
+        const uint32_t nextp = __shfl_down_sync(0xffffffffu, piece, 1);
+        const int j = lane & 3;
+        const uint32_t word = (piece >> (8 * j)) | (nextp << (24 - 8 * j));
+        if (in && j < 3) qrow[chunk * 3 + j] = word;
+      }
+    };
+    if constexpr (RUNS > 0) {
+#pragma unroll
+      for (int r = 0; r < RUNS; ++r) {
+        const int v = r * kQuantThreads + threadIdx.x;
+        emit_run(v, v < nv8, ra[r], rb[r]);
+      }
+    } else {
+      for (int vb = 0; vb < nv8; vb += kQuantThreads) {
+        const int v = vb + threadIdx.x;
+        const bool in = v < nv8;
+        float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
+        if (in) { a = __ldg(w4 + 2 * v); b = __ldg(w4 + 2 * v + 1); }
+        emit_run(v, in, a, b);
+      }
+    }
+    // The next row's pass 1 rewrites cmin/cmax, which pass 2 of this row has finished
+    // with (second barrier above); its pass 2 rewrites the group arrays only after its
+    // own first barrier, which every thread reaches after it has left this pass 3.
+  };
+
+  float4 a0[NR], b0[NR];
+  if constexpr (RUNS > 0 && PREFETCH) {
+    float4 a1[NR], b1[NR];
+    int row = blockIdx.x;
+    load_row(row, a0, b0);
+    while (row < N) {
+      load_row(row + gridDim.x, a1, b1);
+      process_row(row, a0, b0);
+      row += gridDim.x;
+      if (row >= N) break;
+      load_row(row + gridDim.x, a0, b0);
+      process_row(row, a1, b1);
+      row += gridDim.x;
     }
   } else {
-    for (int vb = 0; vb < nv8; vb += kQuantThreads) {
-      const int v = vb + threadIdx.x;
-      const bool in = v < nv8;
-      float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
-      if (in) { a = __ldg(w4 + 2 * v); b = __ldg(w4 + 2 * v + 1); }
-      emit_run(v, in, a, b);
+    for (int row = blockIdx.x; row < N; row += gridDim.x) {
+      if constexpr (RUNS > 0) load_row(row, a0, b0);
+      process_row(row, a0, b0);
     }
   }
 }
@@ -303,25 +369,40 @@ extern "C" int peqa_quantize_rtn(const float* W, int N, int K, int bits, int gro
   int cpg_shift = -1;
   for (int b = 0; b < 26; ++b)
     if ((32 << b) == g) cpg_shift = b;
-  // rows up to 2048 * RUNS columns stay in registers between the passes
+  // rows up to 2048 * RUNS columns stay in registers between the passes; short rows also
+  // prefetch the CTA's next row
   const int runs = K <= 4096 ? 2 : K <= 8192 ? 4 : K <= 12288 ? 6 : K <= 24576 ? 12 : 0;
-#define PEQA_QUANT_LAUNCH(B, R) \
-  quantize_rtn_kernel<B, R><<<N, kQuantThreads, 0, st>>>(W, K, g, cpg_shift, qweight, zeros, scales)
+  const size_t smem = (size_t)(K / g) * (sizeof(GroupConst) + 8) + (size_t)(K >> 5) * 8;
+  int sms = 0, dev = 0;
+  PEQA_CUDA(cudaGetDevice(&dev));
+  PEQA_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+#define PEQA_QUANT_LAUNCH(B, R, P)                                                                     \
+  do {                                                                                                 \
+    auto kern = quantize_rtn_kernel<B, R, P>;                                                          \
+    if (smem > 48 * 1024)                                                                              \
+      PEQA_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));   \
+    int per_sm = 0;                                                                                    \
+    PEQA_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kQuantThreads, smem));      \
+    if (per_sm < 1) per_sm = 1;                                                                        \
+    const long long resident = (long long)sms * per_sm;                                                \
+    const int grid = (int)(N < resident ? N : resident);                                               \
+    kern<<<grid, kQuantThreads, smem, st>>>(W, N, K, g, cpg_shift, qweight, zeros, scales);            \
+  } while (0)
   if (bits == 4) {
     switch (runs) {
-      case 2: PEQA_QUANT_LAUNCH(4, 2); break;
-      case 4: PEQA_QUANT_LAUNCH(4, 4); break;
-      case 6: PEQA_QUANT_LAUNCH(4, 6); break;
-      case 12: PEQA_QUANT_LAUNCH(4, 12); break;
-      default: PEQA_QUANT_LAUNCH(4, 0); break;
+      case 2: PEQA_QUANT_LAUNCH(4, 2, true); break;
+      case 4: PEQA_QUANT_LAUNCH(4, 4, true); break;
+      case 6: PEQA_QUANT_LAUNCH(4, 6, false); break;
+      case 12: PEQA_QUANT_LAUNCH(4, 12, false); break;
+      default: PEQA_QUANT_LAUNCH(4, 0, false); break;
     }
   } else {
     switch (runs) {
-      case 2: PEQA_QUANT_LAUNCH(3, 2); break;
-      case 4: PEQA_QUANT_LAUNCH(3, 4); break;
-      case 6: PEQA_QUANT_LAUNCH(3, 6); break;
-      case 12: PEQA_QUANT_LAUNCH(3, 12); break;
-      default: PEQA_QUANT_LAUNCH(3, 0); break;
+      case 2: PEQA_QUANT_LAUNCH(3, 2, true); break;
+      case 4: PEQA_QUANT_LAUNCH(3, 4, true); break;
+      case 6: PEQA_QUANT_LAUNCH(3, 6, false); break;
+      case 12: PEQA_QUANT_LAUNCH(3, 12, false); break;
+      default: PEQA_QUANT_LAUNCH(3, 0, false); break;
     }
   }
 #undef PEQA_QUANT_LAUNCH
