@@ -440,6 +440,7 @@ size_t decode_workspace_bytes(const peqa_qweight_t*, int, int) { return 0; }
 int launch_decode(const peqa_qweight_t* w, int g, const void* X, int M, void* Y,
                   void* workspace, size_t workspace_bytes, cudaStream_t st) {
   (void)workspace; (void)workspace_bytes;
+  if (decode_stream_supported(w, g, M)) return launch_decode_stream(w, g, X, M, Y, st);
   DecodeParams p;
   p.qw = w->qweight;
   p.zeros = w->zeros;
@@ -498,7 +499,7 @@ int launch_decode(const peqa_qweight_t* w, int g, const void* X, int M, void* Y,
     cuuint32_t estr[2] = {1, 1};
     if (enc(&tmap_q, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<uint32_t*>(w->qweight), dims,
             strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B,
-            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return cuda_fail(cudaErrorInvalidValue);
   }
   const bool fold = p.G > 1;

@@ -94,6 +94,25 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst_smem, const CUtensorMap
       : "memory");
 }
 
+// 16-byte asynchronous copy global -> shared memory through the load/store unit
+// (not TMA), bypassing L1; both addresses 16-byte aligned.
+__device__ __forceinline__ void cp_async_16(uint32_t dst_smem, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst_smem),
+               "l"(reinterpret_cast<uint64_t>(src))
+               : "memory");
+}
+// One arrival on `bar` once all cp.async copies this thread has issued so far have
+// landed.  The arrival is not added to the barrier's pending count: the count the
+// barrier was initialised with must include it.
+__device__ __forceinline__ void cp_async_mbar_arrive_noinc(uint32_t bar) {
+  asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+// Barrier `id` (1..15) among `nthreads` threads of the CTA (a multiple of 32).
+__device__ __forceinline__ void named_barrier_sync(int id, int nthreads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+
 // ----------------------------------------------------------- tensor memory
 __device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols) {
   asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem),

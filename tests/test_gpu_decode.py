@@ -47,6 +47,20 @@ def test_c4_llama65b_shapes(M):
         _check(d, 3, 0, M)
 
 
+@pytest.mark.parametrize("bits,g,M", [(3, 128, 1), (4, 128, 3), (3, 256, 2), (4, 0, 1), (3, 128, 9)])
+def test_several_row_blocks_per_cta(bits, g, M):
+    # N=5120 gives every CTA of the streaming kernel 40 rows (a full 32-row block and a
+    # quarter of one); K=2048 is four 512-column steps, so warps beyond the fourth idle
+    d = synth.custom(50 + bits + g + M, 5120, 2048, 16, bits, g, outliers=True)
+    _check(d, bits, g, M)
+
+
+def test_ring_reuse_with_long_rows():
+    # 152 rows x 43 steps per CTA: the ring is refilled several times
+    d = synth.custom(77, 22016 // 4, 22016 // 2, 2, 3, 128)
+    _check(d, 3, 128, 1)
+
+
 def test_unit_scale_integer_inputs_are_exact():
     rng = np.random.default_rng(0)
     N, K, M = 256, 1024, 5
