@@ -49,8 +49,9 @@ def measured_traffic(kernel_name):
         with open(os.path.join(ROOT, "profiles", "dram_traffic_c2.json")) as f:
             doc = json.load(f)
         h = hashlib.sha256()
-        for name in ("gemm_sm100.cu", "dequant.cuh", "sm100_ptx.cuh", "decode.cu", "elementwise.cu"):
-            with open(os.path.join(ROOT, "paper_2305_14152_b200", "csrc", name), "rb") as f:
+        csrc = os.path.join(ROOT, "paper_2305_14152_b200", "csrc")
+        for name in sorted(os.listdir(csrc)):
+            with open(os.path.join(csrc, name), "rb") as f:
                 h.update(f.read())
         if h.hexdigest() != doc["kernel_sources_sha256"] or doc.get("workload") != WORKLOAD:
             return None
