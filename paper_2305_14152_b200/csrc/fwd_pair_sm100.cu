@@ -262,16 +262,37 @@ qfwd_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     int pf_tile = pair, pf_kb = grp;
     while (pf_kb >= p.k_blocks) { pf_kb -= p.k_blocks; pf_tile += n_pairs; }
     int pf_r = (pf_tile % p.n_tiles) * 256 + (int)rank * 128 + row;
+    // every lane reads another row, so each load of a warp touches 32 sectors: the two
+    // units of a stage share one load when they share a group (g >= 64, or one scale per
+    // channel), and one 2-byte / 8-byte load when the groups are 32 columns wide
+    const bool one_group = p.G == 1 || (p.g & 63) == 0;
+    const bool pair_load = !one_group && p.g == 32 && (p.G & 1) == 0;
     auto load_zs = [&](uint32_t (&z)[2], float (&sc)[2]) {
-#pragma unroll
-      for (int u = 0; u < 2; ++u) {
-        z[u] = 0u;
-        sc[u] = 0.0f;
-        const int col = pf_kb * PK + 32 * u;
-        if (pf_r < p.N && col < p.K) {
-          const size_t gi = (size_t)pf_r * p.G + pair_group_of(p, col);
-          z[u] = __ldg(p.zeros + gi);
-          if (FOLD) sc[u] = __ldg(p.scales + gi);
+      z[0] = z[1] = 0u;
+      sc[0] = sc[1] = 0.0f;
+      const int col = pf_kb * PK;
+      if (pf_r < p.N && col < p.K) {
+        const size_t gi = (size_t)pf_r * p.G + pair_group_of(p, col);
+        if (one_group) {
+          z[0] = z[1] = __ldg(p.zeros + gi);
+          if (FOLD) sc[0] = sc[1] = __ldg(p.scales + gi);
+        } else if (pair_load) {
+          const uint32_t z2 = __ldg(reinterpret_cast<const unsigned short*>(p.zeros + gi));
+          z[0] = z2 & 0xFFu;
+          z[1] = z2 >> 8;
+          if (FOLD) {
+            const float2 s2 = __ldg(reinterpret_cast<const float2*>(p.scales + gi));
+            sc[0] = s2.x;
+            sc[1] = s2.y;
+          }
+        } else {
+          z[0] = __ldg(p.zeros + gi);
+          if (FOLD) sc[0] = __ldg(p.scales + gi);
+          if (col + 32 < p.K) {
+            const size_t g1 = (size_t)pf_r * p.G + pair_group_of(p, col + 32);
+            z[1] = __ldg(p.zeros + g1);
+            if (FOLD) sc[1] = __ldg(p.scales + g1);
+          }
         }
       }
       pf_kb += P_GROUPS;
