@@ -168,6 +168,18 @@ def bwd_ds(X_bits, dY_bits, qweight, zeros, bits: int, group_size: int = 0,
     return dS
 
 
+def bwd_ds_from_y(dY_bits, Y_bits, scales) -> np.ndarray:
+    """Per-channel dS[i] = (sum_t dY[t,i] Y[t,i]) / s[i] in fp64, from the stored bf16 output."""
+    dY_bits = _c(dY_bits, np.uint16)
+    Y_bits = _c(Y_bits, np.uint16)
+    T, N = dY_bits.shape
+    assert Y_bits.shape == (T, N)
+    scales = _c(scales, np.float32).reshape(N)
+    dS = np.empty((N, 1), np.float64)
+    _load().oracle_bwd_ds_from_y(_p(dY_bits), _p(Y_bits), _p(scales), T, N, _p(dS))
+    return dS
+
+
 def adamw(s, grad, m, v, lr, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.0, step=1):
     """One AdamW step on the scales, fp64 arithmetic on the fp32 state."""
     s = _c(s, np.float32).ravel()

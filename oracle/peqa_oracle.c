@@ -259,6 +259,25 @@ void oracle_bwd_ds(const uint16_t* X, const uint16_t* dY, int T, const uint8_t* 
     free(Xd);
 }
 
+/* ---------------------------------------- per-channel dS from the saved Y ---
+ * With one scale per output channel (G = 1), Eq. 2 gives Y[t,i] = s[i] * u[t,i] with
+ * u[t,i] = sum_j X[t,j] (Q[i,j] - z[i]), and the chain rule gives
+ * dS[i] = sum_t dY[t,i] u[t,i].  Hence, written out with the stored output,
+ *   dS[i] = ( sum_t dY[t,i] * Y[t,i] ) / s[i].
+ * Y is the bf16 tensor the forward pass stored (its rounding is part of the input here).
+ * dY, Y are bf16 bit patterns [T, N]; scales is fp32 [N]; dS is double [N].
+ */
+void oracle_bwd_ds_from_y(const uint16_t* dY, const uint16_t* Y, const float* scales, int T,
+                          int N, double* dS) {
+#pragma omp parallel for schedule(static)
+    for (int i = 0; i < N; ++i) {
+        double acc = 0.0;
+        for (int t = 0; t < T; ++t)
+            acc += bf16_to_double(dY[(size_t)t * N + i]) * bf16_to_double(Y[(size_t)t * N + i]);
+        dS[i] = acc / (double)scales[i];
+    }
+}
+
 /* -------------------------------------------------------------- AdamW -----
  * One step of AdamW (decoupled weight decay, bias-corrected moments, step
  * counted from 1) on the scales -- App. A names the optimizer, none of its

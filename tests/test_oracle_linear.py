@@ -161,3 +161,48 @@ def test_bf16_input_conversion_is_round_to_nearest_even():
     import torch
     t = torch.from_numpy(a).to(torch.bfloat16).to(torch.float32).numpy()
     assert np.array_equal(b, t)
+
+
+# ---------------------------------------------------------------------------------------------
+# Per-channel dS from the stored output: dS[i] = (sum_t dY[t,i] Y[t,i]) / s[i]  (Eq. 2 with G = 1)
+
+@pytest.mark.parametrize("bits", [3, 4])
+def test_ds_from_saved_output_equals_ds_when_the_output_is_exact(bits):
+    """Power-of-two scales and small integer activations make Y exact in bf16; the two
+    routes to dS (through dY^T X, and through the stored Y) must then agree to rounding."""
+    rng = np.random.default_rng(5 + bits)
+    T, N, K = 23, 12, 64
+    codes = rng.integers(0, 1 << bits, size=(N, K), dtype=np.uint8)
+    zeros = rng.integers(0, 1 << bits, size=(N, 1), dtype=np.uint8)
+    scales = (2.0 ** rng.integers(-3, 2, size=(N, 1))).astype(np.float32)
+    qw = oracle.pack(codes, bits)
+    # at most two non-zero activations per token keeps |Y| <= 2*15*2 = 60 steps of 1/8: exact in bf16
+    Xi = np.zeros((T, K))
+    for t in range(T):
+        Xi[t, rng.choice(K, 2, replace=False)] = rng.integers(-1, 2, size=2)
+    dYi = rng.integers(-3, 4, size=(T, N)).astype(np.float64)
+    Xb = synth.f32_to_bf16_bits(Xi.astype(np.float32))
+    dYb = synth.f32_to_bf16_bits(dYi.astype(np.float32))
+    Y = oracle.fwd(Xb, qw, zeros, scales, bits, 0)
+    Yb = synth.f32_to_bf16_bits(Y.astype(np.float32))
+    assert np.array_equal(_f(Yb), Y)                      # the premise: nothing was rounded
+    a = oracle.bwd_ds(Xb, dYb, qw, zeros, bits, 0)
+    b = oracle.bwd_ds_from_y(dYb, Yb, scales)
+    assert np.allclose(a, b, rtol=1e-13, atol=1e-13)
+
+
+def test_ds_from_saved_output_literal_loop_and_rounded_output():
+    T, N, K = 40, 9, 128
+    d, codes, zeros, scales, qw = _case(11, N, K, T, 4, 0, sigma_dy=1e-2)
+    Y = oracle.fwd(d["X"], qw, zeros, scales, 4, 0)
+    Yb = synth.f32_to_bf16_bits(Y.astype(np.float32))
+    got = oracle.bwd_ds_from_y(d["dY"], Yb, scales)
+    dY = _f(d["dY"])
+    Yr = _f(Yb)
+    for i in range(N):
+        ref = sum(Fraction(float(dY[t, i])) * Fraction(float(Yr[t, i])) for t in range(T)) / Fraction(float(scales[i, 0]))
+        assert abs(got[i, 0] - float(ref)) <= 1e-12 * max(1.0, abs(float(ref)))
+    # against the route through dY^T X: only the bf16 rounding of Y separates them
+    full = oracle.bwd_ds(d["X"], d["dY"], qw, zeros, 4, 0)
+    err = np.linalg.norm(got - full) / np.linalg.norm(full)
+    assert err < 5e-3
