@@ -301,6 +301,11 @@ def run_cuda(args):
     if rank == 0 and not args.only_step:
         decode = bench_decode(binding, dev, peaks)
 
+    # ---- next-row item: per-channel dS from the stored output (HBM bound, 4*T*N bytes)
+    ds_from_y = None
+    if rank == 0 and not args.only_step:
+        ds_from_y = bench_ds_from_y(binding, dev, peaks)
+
     out = {
         "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
@@ -312,7 +317,7 @@ def run_cuda(args):
                    "flop_per_step": flop_step},
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
         "stage_ms": dict(zip(stage_names, stage_ms)),
-        "roofline": roofline, "decode": decode,
+        "roofline": roofline, "decode": decode, "ds_from_y": ds_from_y,
     }
     if rank == 0 and world == 1 and not args.only_step:
         dt, fl, what = oracle_sample(spec, sets[0])
@@ -394,6 +399,39 @@ def bench_decode(binding, dev, peaks, reps=30):
                      "frac_nominal_8000": gbs / 8000.0, "bytes": nbytes, "copies": copies}
         del qs, qws
     return res
+
+
+def bench_ds_from_y(binding, dev, peaks, reps=20):
+    """GB/s of peqa_qlinear_bwd_ds_from_y on the LLaMA-7B MLP gate shape (N=11008, T=4096, 4-bit
+    per-channel): two rotating (dY, Y) pairs of 180 MB each, so every launch streams from HBM."""
+    import torch
+    N, K, T = 11008, 4096, 4096
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(3)
+    q = torch.zeros((N, K * 4 // 32), dtype=torch.int32, device=dev)
+    z = torch.zeros((N, 1), dtype=torch.uint8, device=dev)
+    s = torch.full((N, 1), 0.01, dtype=torch.float32, device=dev)
+    qw = binding.QWeight(4, N, K, 0, q, z, s)
+    pairs = [(torch.randn((T, N), device=dev, generator=gen).to(torch.bfloat16),
+              torch.randn((T, N), device=dev, generator=gen).to(torch.bfloat16)) for _ in range(2)]
+    dS = torch.empty((N, 1), dtype=torch.float32, device=dev)
+    ws = binding.alloc_workspace(binding.OP_BWD_DS_FROM_Y, T, qw)
+    for i in range(3):
+        binding.qlinear_bwd_ds_from_y(qw, pairs[i % 2][0], pairs[i % 2][1], dS, ws)
+    torch.cuda.synchronize()
+    e0 = torch.cuda.Event(enable_timing=True)
+    e1 = torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(reps):
+        binding.qlinear_bwd_ds_from_y(qw, pairs[i % 2][0], pairs[i % 2][1], dS, ws)
+    e1.record()
+    torch.cuda.synchronize()
+    us = e0.elapsed_time(e1) / reps * 1e3
+    nbytes = 4 * T * N + 8 * N
+    gbs = nbytes / (us * 1e-6) / 1e9
+    return {"workload": "N=11008, T=4096 (c3 gate), bf16 dY and Y", "us": us, "GB/s": gbs,
+            "frac_measured_hbm": gbs / peaks["hbm_gbs"], "bytes": nbytes,
+            "replaces": "the dS contraction of the same layer (2*T*N*K flop)"}
 
 
 def main():

@@ -67,7 +67,12 @@ typedef struct {
   const float* scales;     /* [N, G] */
 } peqa_qweight_t;
 
-typedef enum { PEQA_OP_FWD = 0, PEQA_OP_BWD = 1, PEQA_OP_DECODE = 2 } peqa_op;
+typedef enum {
+  PEQA_OP_FWD = 0,
+  PEQA_OP_BWD = 1,
+  PEQA_OP_DECODE = 2,
+  PEQA_OP_BWD_DS_FROM_Y = 3
+} peqa_op;
 
 /* Library version, major*10000 + minor*100 + patch. */
 int peqa_version(void);
@@ -126,6 +131,23 @@ int peqa_qlinear_fwd(const peqa_qweight_t* w, const void* X_bf16, int T, void* Y
 int peqa_qlinear_bwd(const peqa_qweight_t* w, const void* X_bf16, const void* dY_bf16, int T,
                      void* dX_bf16, float* dS, void* workspace, size_t workspace_bytes,
                      void* stream);
+
+/*
+ * Scale gradient of a per-channel layer (group_size 0 or K, the paper's main
+ * setting, Sec. 3.2) from the output the forward pass stored.  Eq. 2 with one
+ * scale per channel reads Y[t,i] = s[i] * sum_j X[t,j] (Q[i,j] - z[i]), so
+ *   dS[i] = ( sum_t dY[t,i] * Y[t,i] ) / s[i]
+ * and the third contraction of the backward pass is not needed: the call reads
+ * dY and Y once (4*T*N bytes).  Y must be the bf16 tensor peqa_qlinear_fwd wrote
+ * for the same X and the same scales; its bf16 rounding carries into dS (about
+ * 1e-3 relative).  A channel whose scale is 0 gets inf or NaN.
+ *   dY, Y  in   bf16 [T, N]        dS  out  fp32 [N]  OVERWRITTEN
+ * Requires one scale per channel (else PEQA_ERR_BAD_SHAPE), N % 8 == 0 and a
+ * workspace of peqa_workspace_bytes(PEQA_OP_BWD_DS_FROM_Y, T, w) bytes.
+ */
+int peqa_qlinear_bwd_ds_from_y(const peqa_qweight_t* w, const void* dY_bf16, const void* Y_bf16,
+                               int T, float* dS, void* workspace, size_t workspace_bytes,
+                               void* stream);
 
 /*
  * Small-batch forward for token generation (the memory-bound matrix-vector

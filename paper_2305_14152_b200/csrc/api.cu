@@ -56,6 +56,7 @@ extern "C" size_t peqa_workspace_bytes(int op, int T, const peqa_qweight_t* w) {
   switch (op) {
     case PEQA_OP_BWD: return ds_workspace_bytes(w, g, T);
     case PEQA_OP_DECODE: return decode_workspace_bytes(w, g, T);
+    case PEQA_OP_BWD_DS_FROM_Y: return g == w->in_features ? ds_from_y_workspace_bytes(w, T) : 0;
     default: return 0;
   }
 }
@@ -99,6 +100,22 @@ extern "C" int peqa_qlinear_bwd(const peqa_qweight_t* w, const void* X, const vo
   if (dX) PEQA_TRY(launch_dx(w, g, dY, T, dX, as_stream(stream)));
   if (dS) PEQA_TRY(launch_ds(w, g, X, dY, T, dS, workspace, workspace_bytes, as_stream(stream)));
   return PEQA_OK;
+}
+
+extern "C" int peqa_qlinear_bwd_ds_from_y(const peqa_qweight_t* w, const void* dY, const void* Y,
+                                          int T, float* dS, void* workspace,
+                                          size_t workspace_bytes, void* stream) {
+  int g = 0, G = 0;
+  PEQA_TRY(check_qweight(w, &g, &G));
+  if (!dY || !Y || !dS) return PEQA_ERR_NULL;
+  if (G != 1) return PEQA_ERR_BAD_SHAPE;          // the identity holds for one scale per channel only
+  if (T <= 0 || w->out_features % 8 != 0) return PEQA_ERR_BAD_SHAPE;
+  if (!aligned16(dY) || !aligned16(Y) || !aligned16(dS)) return PEQA_ERR_ALIGNMENT;
+  PEQA_TRY(check_arch());
+  const size_t need = ds_from_y_workspace_bytes(w, T);
+  if (!workspace || workspace_bytes < need) return PEQA_ERR_WORKSPACE;
+  if (reinterpret_cast<uintptr_t>(workspace) & 255u) return PEQA_ERR_ALIGNMENT;
+  return launch_ds_from_y(w, dY, Y, T, dS, workspace, as_stream(stream));
 }
 
 extern "C" int peqa_qlinear_decode(const peqa_qweight_t* w, const void* X, int M, void* Y,
