@@ -177,7 +177,13 @@ int peqa_scale_adamw(float* scales, const float* dS, float* m, float* v, int64_t
  * copies Y [T,N], dX [T,K] (host bf16) and dS [N,G] (host fp32) back.  Every
  * d_* pointer is device memory of the size of its host counterpart; d_m, d_v
  * are the optimizer state [N,G].  w->scales is updated in place (it must be
- * writable).  Synchronises the stream before returning.
+ * writable).  Synchronises the stream before returning.  The tokens travel in
+ * chunks over two auxiliary streams of the library, so that the copies in, the
+ * kernels and the copies out overlap (pinned host buffers are needed for that);
+ * those streams and a few events are created on the first call on a device
+ * and kept until the process ends, so make that first call outside any stream
+ * capture.  h_* and d_* buffers must not be touched by other work until the
+ * call returns.
  */
 int peqa_train_step_host(const peqa_qweight_t* w, int T,
                          const void* h_X_bf16, const void* h_dY_bf16,

@@ -135,6 +135,48 @@ extern "C" int peqa_qlinear_decode(const peqa_qweight_t* w, const void* X, int M
   return launch_decode(w, g, X, M, Y, workspace, workspace_bytes, as_stream(stream));
 }
 
+namespace {
+
+// Two auxiliary streams and a pool of events per device for peqa_train_step_host, made on
+// the first call on that device and kept until the process ends.
+constexpr int kHostChunksMax = 8;
+struct HostPipe {
+  cudaStream_t in = nullptr, out = nullptr;
+  cudaEvent_t start = nullptr, out_done = nullptr;
+  cudaEvent_t landed[kHostChunksMax] = {};
+  cudaEvent_t computed[kHostChunksMax] = {};
+  bool ready = false;
+};
+
+int host_pipe(HostPipe** out) {
+  static HostPipe pipes[64];
+  int dev = 0;
+  PEQA_CUDA(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return PEQA_ERR_BAD_SHAPE;
+  HostPipe& hp = pipes[dev];
+  if (!hp.ready) {
+    PEQA_CUDA(cudaStreamCreateWithFlags(&hp.in, cudaStreamNonBlocking));
+    PEQA_CUDA(cudaStreamCreateWithFlags(&hp.out, cudaStreamNonBlocking));
+    PEQA_CUDA(cudaEventCreateWithFlags(&hp.start, cudaEventDisableTiming));
+    PEQA_CUDA(cudaEventCreateWithFlags(&hp.out_done, cudaEventDisableTiming));
+    for (int c = 0; c < kHostChunksMax; ++c) {
+      PEQA_CUDA(cudaEventCreateWithFlags(&hp.landed[c], cudaEventDisableTiming));
+      PEQA_CUDA(cudaEventCreateWithFlags(&hp.computed[c], cudaEventDisableTiming));
+    }
+    hp.ready = true;
+  }
+  *out = &hp;
+  return PEQA_OK;
+}
+
+}  // namespace
+
+// The tokens go through in chunks so that the three engines overlap: chunk c+1 is on its
+// way to the device (auxiliary stream `in`) while chunk c runs forward and dX on the
+// caller's stream and chunk c-1 returns Y and dX (auxiliary stream `out`); PCIe carries both
+// directions at once.  dS sums over all tokens, so it runs once after the last chunk, then
+// AdamW.  Forward and dX treat tokens independently, so chunking does not change a bit of
+// their results.
 extern "C" int peqa_train_step_host(const peqa_qweight_t* w, int T,
                                     const void* h_X, const void* h_dY,
                                     void* h_Y, void* h_dX, float* h_dS,
@@ -149,17 +191,50 @@ extern "C" int peqa_train_step_host(const peqa_qweight_t* w, int T,
       !d_m || !d_v)
     return PEQA_ERR_NULL;
   if (T <= 0) return PEQA_ERR_BAD_SHAPE;
+  PEQA_TRY(check_gemm_shape(w, T));
   cudaStream_t st = as_stream(stream);
   const size_t N = w->out_features, K = w->in_features;
-  PEQA_CUDA(cudaMemcpyAsync(d_X, h_X, (size_t)T * K * 2, cudaMemcpyHostToDevice, st));
-  PEQA_CUDA(cudaMemcpyAsync(d_dY, h_dY, (size_t)T * N * 2, cudaMemcpyHostToDevice, st));
-  PEQA_TRY(peqa_qlinear_fwd(w, d_X, T, d_Y, workspace, workspace_bytes, stream));
-  PEQA_CUDA(cudaMemcpyAsync(h_Y, d_Y, (size_t)T * N * 2, cudaMemcpyDeviceToHost, st));
-  PEQA_TRY(peqa_qlinear_bwd(w, d_X, d_dY, T, d_dX, d_dS, workspace, workspace_bytes, stream));
-  PEQA_CUDA(cudaMemcpyAsync(h_dX, d_dX, (size_t)T * K * 2, cudaMemcpyDeviceToHost, st));
+  // chunks of whole 512-token tiles, at most kHostChunksMax of them
+  int chunks = (T + 511) / 512;
+  if (chunks > kHostChunksMax) chunks = kHostChunksMax;
+  const int per = ((T + chunks - 1) / chunks + 7) & ~7;   // rows per chunk, 16-byte aligned slices
+  chunks = (T + per - 1) / per;
+  HostPipe* hp = nullptr;
+  PEQA_TRY(host_pipe(&hp));
+  const char* hX = static_cast<const char*>(h_X);
+  const char* hdY = static_cast<const char*>(h_dY);
+  char* hY = static_cast<char*>(h_Y);
+  char* hdX = static_cast<char*>(h_dX);
+  char* dX_in = static_cast<char*>(d_X);
+  char* ddY = static_cast<char*>(d_dY);
+  char* dY_out = static_cast<char*>(d_Y);
+  char* ddX = static_cast<char*>(d_dX);
+  // the auxiliary streams start after whatever the caller's stream already holds
+  PEQA_CUDA(cudaEventRecord(hp->start, st));
+  PEQA_CUDA(cudaStreamWaitEvent(hp->in, hp->start, 0));
+  PEQA_CUDA(cudaStreamWaitEvent(hp->out, hp->start, 0));
+  for (int c = 0; c < chunks; ++c) {
+    const size_t t0 = (size_t)c * per;
+    const size_t tc = (size_t)T - t0 < (size_t)per ? (size_t)T - t0 : (size_t)per;
+    PEQA_CUDA(cudaMemcpyAsync(dX_in + t0 * K * 2, hX + t0 * K * 2, tc * K * 2, cudaMemcpyHostToDevice, hp->in));
+    PEQA_CUDA(cudaMemcpyAsync(ddY + t0 * N * 2, hdY + t0 * N * 2, tc * N * 2, cudaMemcpyHostToDevice, hp->in));
+    PEQA_CUDA(cudaEventRecord(hp->landed[c], hp->in));
+    PEQA_CUDA(cudaStreamWaitEvent(st, hp->landed[c], 0));
+    PEQA_TRY(peqa_qlinear_fwd(w, dX_in + t0 * K * 2, (int)tc, dY_out + t0 * N * 2, workspace,
+                              workspace_bytes, stream));
+    PEQA_TRY(peqa_qlinear_bwd(w, nullptr, ddY + t0 * N * 2, (int)tc, ddX + t0 * K * 2, nullptr,
+                              workspace, workspace_bytes, stream));
+    PEQA_CUDA(cudaEventRecord(hp->computed[c], st));
+    PEQA_CUDA(cudaStreamWaitEvent(hp->out, hp->computed[c], 0));
+    PEQA_CUDA(cudaMemcpyAsync(hY + t0 * N * 2, dY_out + t0 * N * 2, tc * N * 2, cudaMemcpyDeviceToHost, hp->out));
+    PEQA_CUDA(cudaMemcpyAsync(hdX + t0 * K * 2, ddX + t0 * K * 2, tc * K * 2, cudaMemcpyDeviceToHost, hp->out));
+  }
+  PEQA_CUDA(cudaEventRecord(hp->out_done, hp->out));
+  PEQA_TRY(peqa_qlinear_bwd(w, d_X, d_dY, T, nullptr, d_dS, workspace, workspace_bytes, stream));
   PEQA_CUDA(cudaMemcpyAsync(h_dS, d_dS, N * (size_t)G * 4, cudaMemcpyDeviceToHost, st));
   PEQA_TRY(peqa_scale_adamw(const_cast<float*>(w->scales), d_dS, d_m, d_v, (int64_t)(N * G), lr,
                             beta1, beta2, eps, weight_decay, step, stream));
+  PEQA_CUDA(cudaStreamWaitEvent(st, hp->out_done, 0));
   PEQA_CUDA(cudaStreamSynchronize(st));
   return PEQA_OK;
 }
