@@ -168,6 +168,22 @@ def bwd_ds(X_bits, dY_bits, qweight, zeros, bits: int, group_size: int = 0,
     return dS
 
 
+def bwd_dz(X_bits, dY_bits, scales, group_size: int = 0, rows=None) -> np.ndarray:
+    """dZ[i,g] = -s[i,g] sum_{j in g} (dY^T X)[i,j] in fp64 (App. K: trainable zero-points)."""
+    X_bits = _c(X_bits, np.uint16)
+    dY_bits = _c(dY_bits, np.uint16)
+    T, K = X_bits.shape
+    N = dY_bits.shape[1]
+    assert dY_bits.shape[0] == T
+    g = _group(K, group_size)
+    scales = _c(scales, np.float32).reshape(N, K // g)
+    keep, n_sel, ptr = _sel(rows)
+    nrows = n_sel if rows is not None else N
+    dZ = np.empty((nrows, K // g), np.float64)
+    _load().oracle_bwd_dz(_p(X_bits), _p(dY_bits), T, _p(scales), N, K, g, ptr, n_sel, _p(dZ))
+    return dZ
+
+
 def bwd_ds_from_y(dY_bits, Y_bits, scales) -> np.ndarray:
     """Per-channel dS[i] = (sum_t dY[t,i] Y[t,i]) / s[i] in fp64, from the stored bf16 output."""
     dY_bits = _c(dY_bits, np.uint16)

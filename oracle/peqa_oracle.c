@@ -259,6 +259,33 @@ void oracle_bwd_ds(const uint16_t* X, const uint16_t* dY, int T, const uint8_t* 
     free(Xd);
 }
 
+/* ------------------------------------------------- zero-point gradient -----
+ * App. K trains the zero-points as well; by the chain rule on Eq. 2,
+ * d W_hat[i,j] / d z[i,g] = -s[i,g] for the columns j of group g, so
+ *   dZ[i,g] = -s[i,g] * sum_{j in g} (dY^T X)[i,j].
+ * X [T,K], dY [T,N] bf16 bit patterns; scales fp32 [N,G]; row_sel as in oracle_bwd_ds;
+ * dZ is [n_sel, G] double.
+ */
+void oracle_bwd_dz(const uint16_t* X, const uint16_t* dY, int T, const float* scales, int N,
+                   int K, int g, const int32_t* row_sel, int n_sel, double* dZ) {
+    const int G = n_groups(K, g);
+    if (!row_sel) n_sel = N;
+#pragma omp parallel for schedule(static)
+    for (int r = 0; r < n_sel; ++r) {
+        int i = row_sel ? row_sel[r] : r;
+        for (int gi = 0; gi < G; ++gi) {
+            double acc = 0.0;
+            for (int j = gi * g; j < (gi + 1) * g; ++j) {
+                double dw = 0.0;
+                for (int t = 0; t < T; ++t)
+                    dw += bf16_to_double(dY[(size_t)t * N + i]) * bf16_to_double(X[(size_t)t * K + j]);
+                acc += dw;
+            }
+            dZ[(size_t)r * G + gi] = -(double)scales[(size_t)i * G + gi] * acc;
+        }
+    }
+}
+
 /* ---------------------------------------- per-channel dS from the saved Y ---
  * With one scale per output channel (G = 1), Eq. 2 gives Y[t,i] = s[i] * u[t,i] with
  * u[t,i] = sum_j X[t,j] (Q[i,j] - z[i]), and the chain rule gives

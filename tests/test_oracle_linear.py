@@ -206,3 +206,46 @@ def test_ds_from_saved_output_literal_loop_and_rounded_output():
     full = oracle.bwd_ds(d["X"], d["dY"], qw, zeros, 4, 0)
     err = np.linalg.norm(got - full) / np.linalg.norm(full)
     assert err < 5e-3
+
+
+# ---------------------------------------------------------------------------------------------
+# Zero-point gradient (App. K): dZ[i,g] = -s[i,g] sum_{j in g} (dY^T X)[i,j]
+
+@pytest.mark.parametrize("bits,g", [(4, 0), (3, 32), (4, 64)])
+def test_dz_is_the_derivative_of_the_loss_in_a_real_valued_zero_point(bits, g):
+    """L(z) = <dY, X W_hat(z)^T> is linear in z, so a finite difference with any step is exact
+    up to rounding; W_hat(z) is formed here in numpy fp64 with z made real-valued."""
+    T, N, K = 11, 6, 128
+    d, codes, zeros, scales, qw = _case(21 + bits + g, N, K, T, bits, g)
+    gg = K if g == 0 else g
+    G = K // gg
+    X, dY = _f(d["X"]), _f(d["dY"])
+    s64 = scales.astype(np.float64)
+
+    def loss(z):
+        What = np.repeat(s64, gg, axis=1) * (codes.astype(np.float64) - np.repeat(z, gg, axis=1))
+        return float(np.sum(dY * (X @ What.T)))
+
+    z0 = zeros.astype(np.float64)
+    dZ = oracle.bwd_dz(d["X"], d["dY"], scales, g)
+    base = loss(z0)
+    for i in range(N):
+        for gi in range(G):
+            z1 = z0.copy()
+            z1[i, gi] += 0.5
+            fd = (loss(z1) - base) / 0.5
+            assert abs(dZ[i, gi] - fd) <= 1e-9 * max(1.0, abs(fd), abs(base))
+
+
+def test_dz_through_group_sums_of_the_activations():
+    """sum_{j in g} (dY^T X)[i,j] = sum_t dY[t,i] * (sum_{j in g} X[t,j]): the same number by a
+    route that never forms dY^T X."""
+    T, N, K, g = 19, 8, 192, 64
+    d, codes, zeros, scales, qw = _case(31, N, K, T, 3, g)
+    X, dY = _f(d["X"]), _f(d["dY"])
+    Xg = X.reshape(T, K // g, g).sum(axis=2)                 # [T, G]
+    ref = -scales.astype(np.float64) * (dY.T @ Xg)           # [N, G]
+    got = oracle.bwd_dz(d["X"], d["dY"], scales, g)
+    assert np.allclose(got, ref, rtol=1e-12, atol=1e-12)
+    rows = np.array([5, 0, 3], np.int32)
+    assert np.allclose(oracle.bwd_dz(d["X"], d["dY"], scales, g, rows=rows), ref[rows], rtol=1e-12, atol=1e-12)
