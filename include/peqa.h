@@ -71,7 +71,8 @@ typedef enum {
   PEQA_OP_FWD = 0,
   PEQA_OP_BWD = 1,
   PEQA_OP_DECODE = 2,
-  PEQA_OP_BWD_DS_FROM_Y = 3
+  PEQA_OP_BWD_DS_FROM_Y = 3,
+  PEQA_OP_BWD_DSDZ = 4
 } peqa_op;
 
 /* Library version, major*10000 + minor*100 + patch. */
@@ -131,6 +132,21 @@ int peqa_qlinear_fwd(const peqa_qweight_t* w, const void* X_bf16, int T, void* Y
 int peqa_qlinear_bwd(const peqa_qweight_t* w, const void* X_bf16, const void* dY_bf16, int T,
                      void* dX_bf16, float* dS, void* workspace, size_t workspace_bytes,
                      void* stream);
+
+/*
+ * Scale gradient and zero-point gradient together (App. K trains z as well as
+ * s).  By the chain rule on Eq. 2, with dW = dY^T X never leaving the chip,
+ *   dS[i,gi] = sum_{j in group gi} (Q[i,j] - z[i,gi]) * dW[i,j]     (as peqa_qlinear_bwd)
+ *   dZ[i,gi] = -s[i,gi] * sum_{j in group gi} dW[i,j]
+ * Both come from the same dW tiles in one pass.  z itself stays the stored
+ * integer: the gradient is what an optimizer of a real-valued copy would use.
+ *   X  in  bf16 [T, K]   dY  in  bf16 [T, N]   dS, dZ  out  fp32 [N, G]  OVERWRITTEN
+ * Requires K % 64 == 0, N % 8 == 0, T >= 1 and a workspace of
+ * peqa_workspace_bytes(PEQA_OP_BWD_DSDZ, T, w) bytes when that is non-zero.
+ */
+int peqa_qlinear_bwd_dsdz(const peqa_qweight_t* w, const void* X_bf16, const void* dY_bf16, int T,
+                          float* dS, float* dZ, void* workspace, size_t workspace_bytes,
+                          void* stream);
 
 /*
  * Scale gradient of a per-channel layer (group_size 0 or K, the paper's main

@@ -17,7 +17,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libpeqa_b200.so")
 _lib = None
 
-OP_FWD, OP_BWD, OP_DECODE, OP_BWD_DS_FROM_Y = 0, 1, 2, 3
+OP_FWD, OP_BWD, OP_DECODE, OP_BWD_DS_FROM_Y, OP_BWD_DSDZ = 0, 1, 2, 3, 4
 
 STATUS_NAMES = {
     0: "PEQA_OK", -1: "PEQA_ERR_NULL", -2: "PEQA_ERR_BAD_BITS", -3: "PEQA_ERR_BAD_SHAPE",
@@ -67,6 +67,8 @@ def lib() -> ctypes.CDLL:
         L.peqa_scale_adamw.argtypes = [vp, vp, vp, vp, i64, f32, f32, f32, f32, f32, i64, vp]
         L.peqa_train_step_host.argtypes = [qp, i32] + [vp] * 12 + [f32] * 5 + [i64, vp, sz, vp]
         L.peqa_check_status.argtypes = [vp]
+        L.peqa_qlinear_bwd_dsdz.argtypes = [qp, vp, vp, i32, vp, vp, vp, sz, vp]
+        L.peqa_qlinear_bwd_dsdz.restype = ctypes.c_int
         L.peqa_qlinear_bwd_ds_from_y.argtypes = [qp, vp, vp, i32, vp, vp, sz, vp]
         L.peqa_qlinear_bwd_ds_from_y.restype = ctypes.c_int
         L.peqa_qlinear_bwd_ds_static.argtypes = [qp, vp, vp, i32, vp, vp]
@@ -237,6 +239,25 @@ def train_step_host(w: QWeight, h_X, h_dY, h_Y, h_dX, h_dS, d_X, d_dY, d_Y, d_dX
         h_dS.data_ptr(), d_X.data_ptr(), d_dY.data_ptr(), d_Y.data_ptr(), d_dX.data_ptr(),
         d_dS.data_ptr(), d_m.data_ptr(), d_v.data_ptr(), lr, beta1, beta2, eps, weight_decay, step,
         wp, wb, _stream()), "peqa_train_step_host")
+
+
+def qlinear_bwd_dsdz(w: QWeight, X: torch.Tensor, dY: torch.Tensor, dS=None, dZ=None, workspace=None):
+    """Scale gradient and zero-point gradient from the same dW tiles."""
+    _dev(X, torch.bfloat16, "X")
+    _dev(dY, torch.bfloat16, "dY")
+    T = dY.shape[0]
+    if dS is None:
+        dS = torch.empty((w.N, w.G), dtype=torch.float32, device=dY.device)
+    if dZ is None:
+        dZ = torch.empty((w.N, w.G), dtype=torch.float32, device=dY.device)
+    if workspace is None:
+        workspace = alloc_workspace(OP_BWD_DSDZ, T, w)
+    cs = w.c_struct()
+    wp, wb = _ws(workspace)
+    _check(lib().peqa_qlinear_bwd_dsdz(ctypes.byref(cs), X.data_ptr(), dY.data_ptr(), T,
+                                       dS.data_ptr(), dZ.data_ptr(), wp, wb, _stream()),
+           "peqa_qlinear_bwd_dsdz")
+    return dS, dZ
 
 
 def qlinear_bwd_ds_from_y(w: QWeight, dY: torch.Tensor, Y: torch.Tensor, dS=None, workspace=None):

@@ -56,6 +56,7 @@ extern "C" size_t peqa_workspace_bytes(int op, int T, const peqa_qweight_t* w) {
   switch (op) {
     case PEQA_OP_BWD: return ds_workspace_bytes(w, g, T);
     case PEQA_OP_DECODE: return decode_workspace_bytes(w, g, T);
+    case PEQA_OP_BWD_DSDZ: return dsdz_workspace_bytes(w, g, T);
     case PEQA_OP_BWD_DS_FROM_Y: return g == w->in_features ? ds_from_y_workspace_bytes(w, T) : 0;
     default: return 0;
   }
@@ -98,8 +99,25 @@ extern "C" int peqa_qlinear_bwd(const peqa_qweight_t* w, const void* X, const vo
     }
   }
   if (dX) PEQA_TRY(launch_dx(w, g, dY, T, dX, as_stream(stream)));
-  if (dS) PEQA_TRY(launch_ds(w, g, X, dY, T, dS, workspace, workspace_bytes, as_stream(stream)));
+  if (dS) PEQA_TRY(launch_ds(w, g, X, dY, T, dS, nullptr, workspace, workspace_bytes, as_stream(stream)));
   return PEQA_OK;
+}
+
+extern "C" int peqa_qlinear_bwd_dsdz(const peqa_qweight_t* w, const void* X, const void* dY, int T,
+                                     float* dS, float* dZ, void* workspace,
+                                     size_t workspace_bytes, void* stream) {
+  int g = 0, G = 0;
+  PEQA_TRY(check_qweight(w, &g, &G));
+  if (!X || !dY || !dS || !dZ) return PEQA_ERR_NULL;
+  PEQA_TRY(check_gemm_shape(w, T));
+  if (!aligned16(X) || !aligned16(dY) || !aligned16(dS) || !aligned16(dZ)) return PEQA_ERR_ALIGNMENT;
+  PEQA_TRY(check_arch());
+  const size_t need = dsdz_workspace_bytes(w, g, T);
+  if (need > 0) {
+    if (!workspace || workspace_bytes < need) return PEQA_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(workspace) & 255u) return PEQA_ERR_ALIGNMENT;
+  }
+  return launch_ds(w, g, X, dY, T, dS, dZ, workspace, workspace_bytes, as_stream(stream));
 }
 
 extern "C" int peqa_qlinear_bwd_ds_from_y(const peqa_qweight_t* w, const void* dY, const void* Y,

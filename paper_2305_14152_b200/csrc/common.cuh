@@ -63,7 +63,8 @@ bool dx_pair_supported(const peqa_qweight_t* w);
 int launch_dx_pair(const peqa_qweight_t* w, int g, const void* dY, int T, void* dX, cudaStream_t st);
 int launch_dx(const peqa_qweight_t* w, int g, const void* dY, int T, void* dX, cudaStream_t st);
 int launch_ds(const peqa_qweight_t* w, int g, const void* X, const void* dY, int T, float* dS,
-              void* workspace, size_t workspace_bytes, cudaStream_t st);
+              float* dZ, void* workspace, size_t workspace_bytes, cudaStream_t st);
+size_t dsdz_workspace_bytes(const peqa_qweight_t* w, int g, int T);
 size_t ds_workspace_bytes(const peqa_qweight_t* w, int g, int T);
 size_t ds_from_y_workspace_bytes(const peqa_qweight_t* w, int T);
 int launch_ds_from_y(const peqa_qweight_t* w, const void* dY, const void* Y, int T, float* dS,

@@ -455,6 +455,8 @@ struct DsParams {
   const uint32_t* qw;
   const uint8_t* zeros;
   float* out;        // [N, K / piece]: dS itself when piece == g, else partial sums
+  float* out_z;      // same shape: dZ (or its partial sums of dW); only read by ds_kernel<.., true>
+  const float* scales;
   int N, K, G, g, T;
   int wpr;
   int piece;         // columns per output piece: 32, 64 or 128; divides g
@@ -480,7 +482,7 @@ struct DsBarriers {
   int abort_flag;
 };
 
-template <int BITS>
+template <int BITS, bool DZ>
 __global__ void __launch_bounds__(kDsThreads, 1)
 ds_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_constant__ CUtensorMap tmap_x,
           const DsParams p) {
@@ -592,7 +594,7 @@ ds_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_constant__ C
       if (!mbar_wait_cluster(smem_u32(&bars->acc_full[buf]), acc_ph, abort_flag)) { ok = false; break; }
       tc_fence_after();
       const int i = i0 + quarter * 32 + lane;
-      float acc = 0.0f;
+      float acc = 0.0f, accz = 0.0f;
 #pragma unroll 1
       for (int cc = 0; cc < 4; ++cc) {
         const int col0 = j0 + half * 128 + cc * 32;
@@ -621,10 +623,20 @@ ds_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_constant__ C
         for (int q = 0; q < 16; ++q) {
           acc = fmaf(__uint_as_float(v[2 * q]), __uint_as_float(o[q] << 16), acc);
           acc = fmaf(__uint_as_float(v[2 * q + 1]), __uint_as_float(o[q] & 0xFFFF0000u), acc);
+          if (DZ) accz += __uint_as_float(v[2 * q]) + __uint_as_float(v[2 * q + 1]);
         }
         if (((cc + 1) % chunks_per_piece) == 0) {
-          if (row_ok) p.out[(size_t)i * npieces + col0 / p.piece] = acc;
+          if (row_ok) {
+            p.out[(size_t)i * npieces + col0 / p.piece] = acc;
+            if (DZ) {
+              // a piece that is a whole group is dZ itself: -s * sum of dW; otherwise the
+              // reduction kernel applies -s after adding the pieces
+              const float f = p.piece == p.g ? -__ldg(p.scales + (size_t)i * p.G + col0 / p.g) : 1.0f;
+              p.out_z[(size_t)i * npieces + col0 / p.piece] = f * accz;
+            }
+          }
           acc = 0.0f;
+          accz = 0.0f;
         }
       }
       tc_fence_before();
@@ -647,15 +659,17 @@ ds_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_constant__ C
   }
 }
 
-// dS[i, gi] = sum of the group's partial pieces, in index order (deterministic).
+// dS[i, gi] = sum of the group's partial pieces, in index order (deterministic); with
+// neg_scales the sum is multiplied by -s[i, gi] (the zero-point gradient).
 __global__ void ds_reduce_kernel(const float* __restrict__ partial, float* __restrict__ dS,
-                                 long long n_out, int pieces_per_group) {
+                                 long long n_out, int pieces_per_group,
+                                 const float* __restrict__ neg_scales) {
   long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (e >= n_out) return;
   const float* src = partial + e * pieces_per_group;
   float acc = 0.0f;
   for (int q = 0; q < pieces_per_group; ++q) acc += src[q];
-  dS[e] = acc;
+  dS[e] = neg_scales ? -neg_scales[e] * acc : acc;
 }
 
 // --------------------------------------------------------------- host side
@@ -808,8 +822,13 @@ size_t ds_workspace_bytes(const peqa_qweight_t* w, int g, int T) {
   return (size_t)w->out_features * (size_t)(w->in_features / piece) * sizeof(float);
 }
 
+// with dZ: a second array of partial sums behind the first
+size_t dsdz_workspace_bytes(const peqa_qweight_t* w, int g, int T) {
+  return 2 * ds_workspace_bytes(w, g, T);
+}
+
 int launch_ds(const peqa_qweight_t* w, int g, const void* X, const void* dY, int T, float* dS,
-              void* workspace, size_t workspace_bytes, cudaStream_t st) {
+              float* dZ, void* workspace, size_t workspace_bytes, cudaStream_t st) {
   (void)workspace_bytes;
   DsParams p;
   p.qw = w->qweight;
@@ -823,6 +842,9 @@ int launch_ds(const peqa_qweight_t* w, int g, const void* X, const void* dY, int
   p.piece = ds_piece(g);
   const bool direct = (p.piece == g);
   p.out = direct ? dS : static_cast<float*>(workspace);
+  p.scales = w->scales;
+  const size_t n_pieces = (size_t)p.N * (size_t)(p.K / p.piece);
+  p.out_z = dZ ? (direct ? dZ : static_cast<float*>(workspace) + n_pieces) : nullptr;
   p.i_tiles = (p.N + 2 * BM - 1) / (2 * BM);   // 256-row pair tiles
   p.j_tiles = (p.K + BN - 1) / BN;
   p.k_blocks = (T + BK - 1) / BK;
@@ -847,19 +869,28 @@ int launch_ds(const peqa_qweight_t* w, int g, const void* X, const void* dY, int
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
+#define PEQA_DS_LAUNCH(B, Z)                                                                          \
+  do {                                                                                               \
+    PEQA_CUDA(cudaFuncSetAttribute(ds_kernel<B, Z>, cudaFuncAttributeMaxDynamicSharedMemorySize,     \
+                                   DS_SMEM_BYTES));                                                  \
+    PEQA_CUDA(cudaLaunchKernelEx(&cfg, ds_kernel<B, Z>, tmap_dy, tmap_x, p));                        \
+  } while (0)
   if (w->bits == 4) {
-    PEQA_CUDA(cudaFuncSetAttribute(ds_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, DS_SMEM_BYTES));
-    PEQA_CUDA(cudaLaunchKernelEx(&cfg, ds_kernel<4>, tmap_dy, tmap_x, p));
+    if (dZ) PEQA_DS_LAUNCH(4, true); else PEQA_DS_LAUNCH(4, false);
   } else {
-    PEQA_CUDA(cudaFuncSetAttribute(ds_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, DS_SMEM_BYTES));
-    PEQA_CUDA(cudaLaunchKernelEx(&cfg, ds_kernel<3>, tmap_dy, tmap_x, p));
+    if (dZ) PEQA_DS_LAUNCH(3, true); else PEQA_DS_LAUNCH(3, false);
   }
+#undef PEQA_DS_LAUNCH
   if (!direct) {
     const long long n_out = (long long)p.N * p.G;
     const int ppg = g / p.piece;
     const int blocks = (int)((n_out + 255) / 256);
-    ds_reduce_kernel<<<blocks, 256, 0, st>>>(p.out, dS, n_out, ppg);
+    ds_reduce_kernel<<<blocks, 256, 0, st>>>(p.out, dS, n_out, ppg, nullptr);
     PEQA_CUDA(cudaGetLastError());
+    if (dZ) {
+      ds_reduce_kernel<<<blocks, 256, 0, st>>>(p.out_z, dZ, n_out, ppg, w->scales);
+      PEQA_CUDA(cudaGetLastError());
+    }
   }
   return PEQA_OK;
 }
