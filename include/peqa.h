@@ -175,6 +175,22 @@ int peqa_qlinear_decode(const peqa_qweight_t* w, const void* X_bf16, int M, void
                         void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Small-batch forward for several tasks at once (Sec. 3.3: one frozen Q and z
+ * serve every task, only the scales are task-specific, so a server switches
+ * tasks by switching s).  Token m is multiplied by the scales of its own task:
+ *   Y[m,i] = S[task_ids[m]][i] * sum_j X[m,j] * (Q[i,j] - z[i])
+ *   scale_table  in  fp32 [n_tasks, N]   (w->scales is not read)
+ *   task_ids     in  int32 [M], device memory; values are clamped to [0, n_tasks-1]
+ *   X  in  bf16 [M, K]     Y  out  bf16 [M, N]     1 <= M <= 16
+ * One scale per channel only (group_size 0 or K), K % 128 == 0, N % 8 == 0, and
+ * M*K small enough for the streaming kernel (M*K <= 32768); otherwise
+ * PEQA_ERR_BAD_SHAPE.
+ */
+int peqa_qlinear_decode_multitask(const peqa_qweight_t* w, const float* scale_table, int n_tasks,
+                                  const int32_t* task_ids, const void* X_bf16, int M,
+                                  void* Y_bf16, void* stream);
+
+/*
  * One AdamW step on the scales, in place (App. A names AdamW; decoupled weight
  * decay, bias-corrected moments, step counted from 1):
  *   s <- s*(1 - lr*wd);  m <- b1*m + (1-b1)*dS;  v <- b2*v + (1-b2)*dS^2

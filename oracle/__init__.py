@@ -168,6 +168,21 @@ def bwd_ds(X_bits, dY_bits, qweight, zeros, bits: int, group_size: int = 0,
     return dS
 
 
+def fwd_multitask(X_bits, qweight, zeros, scale_table, task_ids, bits: int) -> np.ndarray:
+    """Per-channel forward in which token m uses the scales of task task_ids[m] (Sec. 3.3: Q and
+    z are shared by all tasks, s is task-specific).  scale_table is [n_tasks, N]."""
+    X_bits = _c(X_bits, np.uint16)
+    scale_table = _c(scale_table, np.float32)
+    task_ids = np.asarray(task_ids, dtype=np.int64)
+    n_tasks, N = scale_table.shape
+    Y = np.empty((X_bits.shape[0], N), np.float64)
+    for task in range(n_tasks):
+        rows = np.nonzero(task_ids == task)[0]
+        if rows.size:
+            Y[rows] = fwd(X_bits[rows], qweight, zeros, scale_table[task].reshape(N, 1), bits, 0)
+    return Y
+
+
 def bwd_dz(X_bits, dY_bits, scales, group_size: int = 0, rows=None) -> np.ndarray:
     """dZ[i,g] = -s[i,g] sum_{j in g} (dY^T X)[i,j] in fp64 (App. K: trainable zero-points)."""
     X_bits = _c(X_bits, np.uint16)

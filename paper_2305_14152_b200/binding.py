@@ -67,6 +67,8 @@ def lib() -> ctypes.CDLL:
         L.peqa_scale_adamw.argtypes = [vp, vp, vp, vp, i64, f32, f32, f32, f32, f32, i64, vp]
         L.peqa_train_step_host.argtypes = [qp, i32] + [vp] * 12 + [f32] * 5 + [i64, vp, sz, vp]
         L.peqa_check_status.argtypes = [vp]
+        L.peqa_qlinear_decode_multitask.argtypes = [qp, vp, i32, vp, vp, i32, vp, vp]
+        L.peqa_qlinear_decode_multitask.restype = ctypes.c_int
         L.peqa_qlinear_bwd_dsdz.argtypes = [qp, vp, vp, i32, vp, vp, vp, sz, vp]
         L.peqa_qlinear_bwd_dsdz.restype = ctypes.c_int
         L.peqa_qlinear_bwd_ds_from_y.argtypes = [qp, vp, vp, i32, vp, vp, sz, vp]
@@ -239,6 +241,23 @@ def train_step_host(w: QWeight, h_X, h_dY, h_Y, h_dX, h_dS, d_X, d_dY, d_Y, d_dX
         h_dS.data_ptr(), d_X.data_ptr(), d_dY.data_ptr(), d_Y.data_ptr(), d_dX.data_ptr(),
         d_dS.data_ptr(), d_m.data_ptr(), d_v.data_ptr(), lr, beta1, beta2, eps, weight_decay, step,
         wp, wb, _stream()), "peqa_train_step_host")
+
+
+def qlinear_decode_multitask(w: QWeight, scale_table: torch.Tensor, task_ids: torch.Tensor,
+                             X: torch.Tensor, Y=None):
+    """Decode with one scale vector per task: scale_table fp32 [n_tasks, N], task_ids int32 [M]."""
+    _dev(X, torch.bfloat16, "X")
+    _dev(scale_table, torch.float32, "scale_table")
+    _dev(task_ids, torch.int32, "task_ids")
+    M = X.shape[0]
+    if Y is None:
+        Y = torch.empty((M, w.N), dtype=torch.bfloat16, device=X.device)
+    cs = w.c_struct()
+    _check(lib().peqa_qlinear_decode_multitask(ctypes.byref(cs), scale_table.data_ptr(),
+                                               scale_table.shape[0], task_ids.data_ptr(),
+                                               X.data_ptr(), M, Y.data_ptr(), _stream()),
+           "peqa_qlinear_decode_multitask")
+    return Y
 
 
 def qlinear_bwd_dsdz(w: QWeight, X: torch.Tensor, dY: torch.Tensor, dS=None, dZ=None, workspace=None):

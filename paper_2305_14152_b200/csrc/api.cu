@@ -153,6 +153,21 @@ extern "C" int peqa_qlinear_decode(const peqa_qweight_t* w, const void* X, int M
   return launch_decode(w, g, X, M, Y, workspace, workspace_bytes, as_stream(stream));
 }
 
+extern "C" int peqa_qlinear_decode_multitask(const peqa_qweight_t* w, const float* scale_table,
+                                             int n_tasks, const int32_t* task_ids, const void* X,
+                                             int M, void* Y, void* stream) {
+  int g = 0, G = 0;
+  PEQA_TRY(check_qweight(w, &g, &G));
+  if (!scale_table || !task_ids || !X || !Y) return PEQA_ERR_NULL;
+  if (M < 1 || M > 16 || n_tasks < 1) return PEQA_ERR_BAD_SHAPE;
+  if (G != 1) return PEQA_ERR_BAD_SHAPE;          // task-specific scales are per channel here
+  if (w->in_features % 128 != 0 || w->out_features % 8 != 0) return PEQA_ERR_BAD_SHAPE;
+  if (!aligned16(X) || !aligned16(Y) || !aligned16(scale_table)) return PEQA_ERR_ALIGNMENT;
+  PEQA_TRY(check_arch());
+  if (!decode_stream_supported(w, g, M)) return PEQA_ERR_BAD_SHAPE;
+  return launch_decode_stream(w, g, X, M, Y, scale_table, n_tasks, task_ids, as_stream(stream));
+}
+
 namespace {
 
 // Two auxiliary streams and a pool of events per device for peqa_train_step_host, made on

@@ -70,7 +70,9 @@ size_t ds_from_y_workspace_bytes(const peqa_qweight_t* w, int T);
 int launch_ds_from_y(const peqa_qweight_t* w, const void* dY, const void* Y, int T, float* dS,
                      void* workspace, cudaStream_t st);
 bool decode_stream_supported(const peqa_qweight_t* w, int g, int M);
-int launch_decode_stream(const peqa_qweight_t* w, int g, const void* X, int M, void* Y, cudaStream_t st);
+int launch_decode_stream(const peqa_qweight_t* w, int g, const void* X, int M, void* Y,
+                         const float* scale_table, int n_tasks, const int32_t* task_ids,
+                         cudaStream_t st);
 int launch_decode(const peqa_qweight_t* w, int g, const void* X, int M, void* Y,
                   void* workspace, size_t workspace_bytes, cudaStream_t st);
 size_t decode_workspace_bytes(const peqa_qweight_t* w, int g, int M);

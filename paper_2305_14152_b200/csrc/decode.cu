@@ -440,7 +440,7 @@ size_t decode_workspace_bytes(const peqa_qweight_t*, int, int) { return 0; }
 int launch_decode(const peqa_qweight_t* w, int g, const void* X, int M, void* Y,
                   void* workspace, size_t workspace_bytes, cudaStream_t st) {
   (void)workspace; (void)workspace_bytes;
-  if (decode_stream_supported(w, g, M)) return launch_decode_stream(w, g, X, M, Y, st);
+  if (decode_stream_supported(w, g, M)) return launch_decode_stream(w, g, X, M, Y, nullptr, 1, nullptr, st);
   DecodeParams p;
   p.qw = w->qweight;
   p.zeros = w->zeros;

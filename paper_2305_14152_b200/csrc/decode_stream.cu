@@ -82,6 +82,10 @@ struct StreamParams {
   int x_blocks;             // 128-column blocks staged per token (4 * nchunks)
   int x_pitch;              // bytes between staged token rows
   int slots;                // ring depth
+  // multi-task decode (one scale per channel only): token m uses the scales at
+  // scales + clamp(task_ids[m], 0, n_tasks - 1) * N; task_ids == nullptr: one task
+  const int32_t* task_ids;
+  int n_tasks;
   int* status;
 };
 
@@ -399,8 +403,13 @@ decode_stream_kernel(const StreamParams p) {
           for (int wv = 0; wv < kSWarps; ++wv) sum += buf[(wv * 32 + lr) * TOKP + m];
           if (!GROUPED) {
             const float z = (float)__ldg(p.zeros + row);
+            const float* sc = p.scales;
+            if (p.task_ids) {
+              const int task = min(max(__ldg(p.task_ids + m), 0), p.n_tasks - 1);
+              sc += (size_t)task * p.N;
+            }
             sum = (sum - (kBiasLo + z) * xtot[m * 2] - (kBiasHi + z) * xtot[m * 2 + 1]) *
-                  __ldg(p.scales + row);
+                  __ldg(sc + row);
           }
           p.Y[(size_t)m * p.N + row] = __float2bfloat16_rn(sum);
         }
@@ -481,6 +490,7 @@ bool decode_stream_supported(const peqa_qweight_t* w, int g, int M) {
 }
 
 int launch_decode_stream(const peqa_qweight_t* w, int g, const void* X, int M, void* Y,
+                         const float* scale_table, int n_tasks, const int32_t* task_ids,
                          cudaStream_t st) {
   StreamPlan plan;
   PEQA_TRY(plan_stream(w, g, M, &plan));
@@ -488,13 +498,16 @@ int launch_decode_stream(const peqa_qweight_t* w, int g, const void* X, int M, v
   StreamParams p;
   p.qw = w->qweight;
   p.zeros = w->zeros;
-  p.scales = w->scales;
+  p.scales = task_ids ? scale_table : w->scales;
+  p.task_ids = task_ids;
+  p.n_tasks = n_tasks;
   p.X = static_cast<const __nv_bfloat16*>(X);
   p.Y = static_cast<__nv_bfloat16*>(Y);
   p.N = w->out_features;
   p.K = w->in_features;
   p.g = g;
   p.G = p.K / g;
+  if (task_ids && p.G != 1) return PEQA_ERR_BAD_SHAPE;
   p.M = M;
   p.wpr = p.K * w->bits / 32;
   p.nchunks = plan.nchunks;

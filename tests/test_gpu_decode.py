@@ -72,3 +72,37 @@ def test_unit_scale_integer_inputs_are_exact():
     ref = (Xi @ codes.astype(np.int64).T).astype(np.float32)
     exp = synth.bf16_bits_to_f32(synth.f32_to_bf16_bits(ref)).astype(np.float64)
     assert np.array_equal(dev_to_f64(Y), exp)
+
+
+@pytest.mark.parametrize("bits,M", [(3, 1), (4, 5), (3, 16)])
+def test_multitask_scales(bits, M):
+    """Sec. 3.3: one frozen Q, z; token m is decoded with the scale vector of its own task."""
+    N, K = 1032, 1024
+    d = synth.custom(70 + bits + M, N, K, 16, bits, 0, outliers=True)
+    codes, zeros, scales, packed = oracle_layer(d, bits, 0)
+    rng = np.random.default_rng(M)
+    table = (scales[:, 0][None, :] * rng.uniform(0.5, 2.0, size=(3, N))).astype(np.float32)
+    ids = rng.integers(0, 3, size=M).astype(np.int32)
+    qw = to_qweight(packed, zeros, scales, bits, 0, K)
+    Xb = d["X"][:M]
+    Y = binding.qlinear_decode_multitask(qw, torch.from_numpy(table).cuda(),
+                                         torch.from_numpy(ids).cuda(), bf16_to_dev(Xb))
+    torch.cuda.synchronize()
+    binding.check_status()
+    ref = oracle.fwd_multitask(Xb, packed, zeros, table, ids, bits)
+    assert_close(dev_to_f64(Y), ref, "multi-task decode")
+    # ids beyond the table are clamped to its last row
+    Y2 = binding.qlinear_decode_multitask(qw, torch.from_numpy(table).cuda(),
+                                          torch.from_numpy(np.where(ids == 2, 7, ids).astype(np.int32)).cuda(),
+                                          bf16_to_dev(Xb))
+    assert torch.equal(Y, Y2)
+
+
+def test_multitask_rejects_grouped_layers():
+    d = synth.custom(5, 64, 256, 16, 4, 128)
+    codes, zeros, scales, packed = oracle_layer(d, 4, 128)
+    qw = to_qweight(packed, zeros, scales, 4, 128, 256)
+    with pytest.raises(binding.PeqaError):
+        binding.qlinear_decode_multitask(qw, torch.ones((2, 64), device="cuda"),
+                                         torch.zeros(1, dtype=torch.int32, device="cuda"),
+                                         bf16_to_dev(d["X"][:1]))

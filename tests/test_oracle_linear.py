@@ -249,3 +249,22 @@ def test_dz_through_group_sums_of_the_activations():
     assert np.allclose(got, ref, rtol=1e-12, atol=1e-12)
     rows = np.array([5, 0, 3], np.int32)
     assert np.allclose(oracle.bwd_dz(d["X"], d["dY"], scales, g, rows=rows), ref[rows], rtol=1e-12, atol=1e-12)
+
+
+# ---------------------------------------------------------------------------------------------
+# Multi-task forward (Sec. 3.3): shared Q and z, task-specific scales
+
+def test_multitask_forward_rows_are_single_task_forwards():
+    """Row m equals the plain forward under the scales of task_ids[m]; and since per-channel
+    scales factor out of the contraction, Y_task / s_task is the same for every task."""
+    T, N, K = 7, 10, 64
+    d, codes, zeros, scales, qw = _case(41, N, K, T, 4, 0)
+    table = np.stack([scales[:, 0], 2.0 * scales[:, 0], 0.5 * scales[:, 0] + 1e-3]).astype(np.float32)
+    ids = np.array([2, 0, 1, 1, 0, 2, 2])
+    Y = oracle.fwd_multitask(d["X"], qw, zeros, table, ids, 4)
+    X = _f(d["X"])
+    u = X @ (codes.astype(np.float64) - zeros.astype(np.float64)).T       # [T, N], scale-free
+    for m in range(T):
+        assert np.allclose(Y[m], table[ids[m]].astype(np.float64) * u[m], rtol=1e-12, atol=1e-12)
+    same = oracle.fwd_multitask(d["X"], qw, zeros, table, np.zeros(T, int), 4)
+    assert np.array_equal(same, oracle.fwd(d["X"], qw, zeros, scales, 4, 0))
