@@ -206,6 +206,12 @@ def run_cuda(args):
     dev = torch.device("cuda", torch.cuda.current_device())
     peaks, peak_src = load_peaks()
 
+    if args.only_decode:
+        # the decode section alone (what the decode ncu summaries under profiles/ were taken on)
+        print(json.dumps({"decode": bench_decode(binding, dev, peaks, reps=args.steps if args.steps < 30 else 30)}),
+              flush=True)
+        return
+
     spec, sets = draw_sets(N_SETS)
     N, K, T, bits, g = spec.N, spec.K, spec.T, spec.bits, spec.group_size
     G = K // g if g else 1
@@ -440,6 +446,8 @@ def main():
     ap.add_argument("--steps", type=int, default=500)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--only-decode", action="store_true",
+                    help="run only the M=1 decode section on the three LLaMA-65B shapes")
     ap.add_argument("--only-step", action="store_true",
                     help="time the step only: skip the e2e, decode and CPU-baseline sections "
                          "(lean runs under a profiler)")
