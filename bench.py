@@ -231,9 +231,11 @@ def run_cuda(args):
     Yd = torch.empty((1, N), dtype=torch.bfloat16, device=dev)
     ws = binding.alloc_workspace(binding.OP_BWD, T, qws[0])
     lr = 1e-5
-    stage_names = ["quantize_rtn", "qlinear_fwd", "qlinear_bwd_dx", "qlinear_bwd_ds", "scale_adamw",
-                   "qlinear_decode"]
-    launches_per_step = 6 + (1 if ws is not None else 0)
+    # dS and the AdamW step on the scales are one launch (the step is applied where each dS
+    # value becomes final), so the step has five stages
+    stage_names = ["quantize_rtn", "qlinear_fwd", "qlinear_bwd_dx", "qlinear_bwd_ds", "qlinear_decode"]
+    n_stages = len(stage_names)
+    launches_per_step = n_stages + (1 if ws is not None else 0)
 
     def step(i, evs=None):
         r = i % N_SETS
@@ -245,12 +247,11 @@ def run_cuda(args):
         if evs: evs[2].record()
         binding.qlinear_bwd(qw, None, dYs[r], dX=dX, need_ds=False)
         if evs: evs[3].record()
-        binding.qlinear_bwd(qw, Xs[r], dYs[r], dS=dS, workspace=ws, need_dx=False)
+        binding.qlinear_bwd_ds_adamw(qw, Xs[r], dYs[r], m, v, lr, 0.9, 0.999, 1e-8, 0.0, i + 1,
+                                     dS=dS, workspace=ws)
         if evs: evs[4].record()
-        binding.scale_adamw(qw.scales, dS, m, v, lr, 0.9, 0.999, 1e-8, 0.0, i + 1)
-        if evs: evs[5].record()
         binding.qlinear_decode(qw, Xs[r][:1], Yd)
-        if evs: evs[6].record()
+        if evs: evs[5].record()
 
     for i in range(max(args.warmup, 3)):
         step(i)
@@ -258,7 +259,7 @@ def run_cuda(args):
     torch.cuda.synchronize()
 
     sampler = ClockSampler(physical_gpu_index(torch.cuda.current_device()))
-    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(7)] for _ in range(args.steps)]
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(n_stages + 1)] for _ in range(args.steps)]
     if dist is not None:
         dist.barrier()
     torch.cuda.synchronize()
@@ -277,7 +278,7 @@ def run_cuda(args):
     ms_total = aggregate_max(t_start.elapsed_time(t_end), dist, dev)
     ms_step = ms_total / args.steps
     stage_ms = [float(np.mean([evs[i][k].elapsed_time(evs[i][k + 1]) for i in range(args.steps)]))
-                for k in range(6)]
+                for k in range(n_stages)]
 
     flop_step = 6.0 * T * N * K
     value = world * flop_step / (ms_step * 1e-3) / 1e12
@@ -317,7 +318,7 @@ def run_cuda(args):
         "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": f"{WORKLOAD}: LLaMA-7B attention projection N=K=4096, 3-bit, group 128, "
-                               f"T=2048 tokens; step = quantize+pack, fwd, dX, dS, AdamW, decode(M=1)",
+                               f"T=2048 tokens; step = quantize+pack, fwd, dX, dS+AdamW (one launch), decode(M=1)",
                    "l2": f"{N_SETS} rotating input sets (~{N_SETS * 135} MB) exceed the 126 MB L2; no flush kernel",
                    "parallelism": "replicas only" if world > 1 else "single GPU",
                    "flop_per_step": flop_step},

@@ -134,6 +134,21 @@ int peqa_qlinear_bwd(const peqa_qweight_t* w, const void* X_bf16, const void* dY
                      void* stream);
 
 /*
+ * Scale gradient followed at once by the AdamW step on the scales (chain rule
+ * on Eq. 2, then App. A's optimizer): what peqa_qlinear_bwd (dS only) and
+ * peqa_scale_adamw would do in two launches, done where each dS value becomes
+ * final, so the scales, m and v are touched once and no second kernel runs.
+ * Results are bit-identical to the two calls.
+ *   X  in  bf16 [T, K]   dY  in  bf16 [T, N]   dS  out  fp32 [N, G]  OVERWRITTEN
+ *   m, v  in/out  fp32 [N, G];  w->scales is updated in place (it must be writable)
+ * Same shape rules and workspace as peqa_qlinear_bwd; step >= 1.
+ */
+int peqa_qlinear_bwd_ds_adamw(const peqa_qweight_t* w, const void* X_bf16, const void* dY_bf16,
+                              int T, float* dS, float* m, float* v, float lr, float beta1,
+                              float beta2, float eps, float weight_decay, int64_t step,
+                              void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Scale gradient and zero-point gradient together (App. K trains z as well as
  * s).  By the chain rule on Eq. 2, with dW = dY^T X never leaving the chip,
  *   dS[i,gi] = sum_{j in group gi} (Q[i,j] - z[i,gi]) * dW[i,j]     (as peqa_qlinear_bwd)

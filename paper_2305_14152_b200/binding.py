@@ -69,6 +69,8 @@ def lib() -> ctypes.CDLL:
         L.peqa_check_status.argtypes = [vp]
         L.peqa_qlinear_decode_multitask.argtypes = [qp, vp, i32, vp, vp, i32, vp, vp]
         L.peqa_qlinear_decode_multitask.restype = ctypes.c_int
+        L.peqa_qlinear_bwd_ds_adamw.argtypes = [qp, vp, vp, i32, vp, vp, vp, f32, f32, f32, f32, f32, i64, vp, sz, vp]
+        L.peqa_qlinear_bwd_ds_adamw.restype = ctypes.c_int
         L.peqa_qlinear_bwd_dsdz.argtypes = [qp, vp, vp, i32, vp, vp, vp, sz, vp]
         L.peqa_qlinear_bwd_dsdz.restype = ctypes.c_int
         L.peqa_qlinear_bwd_ds_from_y.argtypes = [qp, vp, vp, i32, vp, vp, sz, vp]
@@ -258,6 +260,26 @@ def qlinear_decode_multitask(w: QWeight, scale_table: torch.Tensor, task_ids: to
                                                X.data_ptr(), M, Y.data_ptr(), _stream()),
            "peqa_qlinear_decode_multitask")
     return Y
+
+
+def qlinear_bwd_ds_adamw(w: QWeight, X: torch.Tensor, dY: torch.Tensor, m: torch.Tensor,
+                         v: torch.Tensor, lr: float, beta1=0.9, beta2=0.999, eps=1e-8,
+                         weight_decay=0.0, step=1, dS=None, workspace=None):
+    """dS and the AdamW step on w.scales (in place) in one pass."""
+    _dev(X, torch.bfloat16, "X")
+    _dev(dY, torch.bfloat16, "dY")
+    T = dY.shape[0]
+    if dS is None:
+        dS = torch.empty((w.N, w.G), dtype=torch.float32, device=dY.device)
+    if workspace is None:
+        workspace = alloc_workspace(OP_BWD, T, w)
+    cs = w.c_struct()
+    wp, wb = _ws(workspace)
+    _check(lib().peqa_qlinear_bwd_ds_adamw(ctypes.byref(cs), X.data_ptr(), dY.data_ptr(), T,
+                                           dS.data_ptr(), m.data_ptr(), v.data_ptr(), lr, beta1,
+                                           beta2, eps, weight_decay, step, wp, wb, _stream()),
+           "peqa_qlinear_bwd_ds_adamw")
+    return dS
 
 
 def qlinear_bwd_dsdz(w: QWeight, X: torch.Tensor, dY: torch.Tensor, dS=None, dZ=None, workspace=None):

@@ -99,8 +99,33 @@ extern "C" int peqa_qlinear_bwd(const peqa_qweight_t* w, const void* X, const vo
     }
   }
   if (dX) PEQA_TRY(launch_dx(w, g, dY, T, dX, as_stream(stream)));
-  if (dS) PEQA_TRY(launch_ds(w, g, X, dY, T, dS, nullptr, workspace, workspace_bytes, as_stream(stream)));
+  if (dS) PEQA_TRY(launch_ds(w, g, X, dY, T, dS, nullptr, nullptr, workspace, workspace_bytes, as_stream(stream)));
   return PEQA_OK;
+}
+
+extern "C" int peqa_qlinear_bwd_ds_adamw(const peqa_qweight_t* w, const void* X, const void* dY,
+                                         int T, float* dS, float* m, float* v, float lr,
+                                         float beta1, float beta2, float eps, float weight_decay,
+                                         int64_t step, void* workspace, size_t workspace_bytes,
+                                         void* stream) {
+  int g = 0, G = 0;
+  PEQA_TRY(check_qweight(w, &g, &G));
+  if (!X || !dY || !dS || !m || !v) return PEQA_ERR_NULL;
+  if (step < 1) return PEQA_ERR_BAD_SHAPE;
+  PEQA_TRY(check_gemm_shape(w, T));
+  if (!aligned16(X) || !aligned16(dY) || !aligned16(dS)) return PEQA_ERR_ALIGNMENT;
+  PEQA_TRY(check_arch());
+  const size_t need = ds_workspace_bytes(w, g, T);
+  if (need > 0) {
+    if (!workspace || workspace_bytes < need) return PEQA_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(workspace) & 255u) return PEQA_ERR_ALIGNMENT;
+  }
+  DsAdam adam;
+  adam.c = adamw_consts(lr, beta1, beta2, eps, weight_decay, (long long)step);
+  adam.scales = const_cast<float*>(w->scales);
+  adam.m = m;
+  adam.v = v;
+  return launch_ds(w, g, X, dY, T, dS, nullptr, &adam, workspace, workspace_bytes, as_stream(stream));
 }
 
 extern "C" int peqa_qlinear_bwd_dsdz(const peqa_qweight_t* w, const void* X, const void* dY, int T,
@@ -117,7 +142,7 @@ extern "C" int peqa_qlinear_bwd_dsdz(const peqa_qweight_t* w, const void* X, con
     if (!workspace || workspace_bytes < need) return PEQA_ERR_WORKSPACE;
     if (reinterpret_cast<uintptr_t>(workspace) & 255u) return PEQA_ERR_ALIGNMENT;
   }
-  return launch_ds(w, g, X, dY, T, dS, dZ, workspace, workspace_bytes, as_stream(stream));
+  return launch_ds(w, g, X, dY, T, dS, dZ, nullptr, workspace, workspace_bytes, as_stream(stream));
 }
 
 extern "C" int peqa_qlinear_bwd_ds_from_y(const peqa_qweight_t* w, const void* dY, const void* Y,
@@ -263,10 +288,9 @@ extern "C" int peqa_train_step_host(const peqa_qweight_t* w, int T,
     PEQA_CUDA(cudaMemcpyAsync(hdX + t0 * K * 2, ddX + t0 * K * 2, tc * K * 2, cudaMemcpyDeviceToHost, hp->out));
   }
   PEQA_CUDA(cudaEventRecord(hp->out_done, hp->out));
-  PEQA_TRY(peqa_qlinear_bwd(w, d_X, d_dY, T, nullptr, d_dS, workspace, workspace_bytes, stream));
+  PEQA_TRY(peqa_qlinear_bwd_ds_adamw(w, d_X, d_dY, T, d_dS, d_m, d_v, lr, beta1, beta2, eps,
+                                     weight_decay, step, workspace, workspace_bytes, stream));
   PEQA_CUDA(cudaMemcpyAsync(h_dS, d_dS, N * (size_t)G * 4, cudaMemcpyDeviceToHost, st));
-  PEQA_TRY(peqa_scale_adamw(const_cast<float*>(w->scales), d_dS, d_m, d_v, (int64_t)(N * G), lr,
-                            beta1, beta2, eps, weight_decay, step, stream));
   PEQA_CUDA(cudaStreamWaitEvent(st, hp->out_done, 0));
   PEQA_CUDA(cudaStreamSynchronize(st));
   return PEQA_OK;

@@ -2,6 +2,8 @@
 // CUDA error capture and the device status word.
 #pragma once
 
+#include <math.h>
+
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -55,6 +57,43 @@ int status_word(int** dev_ptr);
 
 inline cudaStream_t as_stream(void* s) { return reinterpret_cast<cudaStream_t>(s); }
 
+// One AdamW step on a scale (App. A; decoupled decay, bias-corrected moments).  The bias
+// corrections 1 - b^t are formed on the host in double and passed as reciprocals, as are
+// 1 - b1 and 1 - b2.  Every operation is a single rounded binary32 operation, so the
+// stand-alone kernel and the kernels that apply the step where dS is produced agree bit
+// for bit.
+struct AdamWConsts {
+  float lr, b1, b2, omb1, omb2, eps, decay, inv_c1, inv_c2;
+};
+
+inline AdamWConsts adamw_consts(float lr, float beta1, float beta2, float eps, float weight_decay,
+                                long long step) {
+  AdamWConsts c;
+  const double c1 = pow((double)beta1, (double)step), c2 = pow((double)beta2, (double)step);
+  c.lr = lr;
+  c.b1 = beta1;
+  c.b2 = beta2;
+  c.omb1 = (float)(1.0 - (double)beta1);
+  c.omb2 = (float)(1.0 - (double)beta2);
+  c.eps = eps;
+  c.decay = (float)(1.0 - (double)lr * (double)weight_decay);
+  c.inv_c1 = (float)(1.0 / (1.0 - c1));
+  c.inv_c2 = (float)(1.0 / (1.0 - c2));
+  return c;
+}
+
+#ifdef __CUDACC__
+__device__ __forceinline__ void adamw_update(float& s, float gr, float& m, float& v,
+                                             const AdamWConsts& c) {
+  const float mn = __fmaf_rn(c.b1, m, __fmul_rn(c.omb1, gr));
+  const float vn = __fmaf_rn(c.b2, v, __fmul_rn(__fmul_rn(c.omb2, gr), gr));
+  const float denom = __fadd_rn(sqrtf(__fmul_rn(vn, c.inv_c2)), c.eps);
+  s = __fsub_rn(__fmul_rn(s, c.decay), __fdiv_rn(__fmul_rn(c.lr, __fmul_rn(mn, c.inv_c1)), denom));
+  m = mn;
+  v = vn;
+}
+#endif
+
 // Entry points implemented in the individual translation units.
 int launch_fwd(const peqa_qweight_t* w, int g, const void* X, int T, void* Y, cudaStream_t st);
 bool fwd_pair_supported(const peqa_qweight_t* w);
@@ -62,8 +101,15 @@ int launch_fwd_pair(const peqa_qweight_t* w, int g, const void* X, int T, void* 
 bool dx_pair_supported(const peqa_qweight_t* w);
 int launch_dx_pair(const peqa_qweight_t* w, int g, const void* dY, int T, void* dX, cudaStream_t st);
 int launch_dx(const peqa_qweight_t* w, int g, const void* dY, int T, void* dX, cudaStream_t st);
+// adam != nullptr: the AdamW step on (w->scales, m, v) is applied where dS is produced
+struct DsAdam {
+  AdamWConsts c;
+  float* scales;
+  float* m;
+  float* v;
+};
 int launch_ds(const peqa_qweight_t* w, int g, const void* X, const void* dY, int T, float* dS,
-              float* dZ, void* workspace, size_t workspace_bytes, cudaStream_t st);
+              float* dZ, const DsAdam* adam, void* workspace, size_t workspace_bytes, cudaStream_t st);
 size_t dsdz_workspace_bytes(const peqa_qweight_t* w, int g, int T);
 size_t ds_workspace_bytes(const peqa_qweight_t* w, int g, int T);
 size_t ds_from_y_workspace_bytes(const peqa_qweight_t* w, int T);

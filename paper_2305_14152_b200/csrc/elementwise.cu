@@ -324,23 +324,18 @@ __global__ void unpack_kernel(const uint32_t* __restrict__ qweight, long long to
     codes[c * 32 + lane] = (uint8_t)warp_unpack<BITS>(qweight + c * BITS, lane);
 }
 
-// Elementwise AdamW in binary32.  The bias corrections 1-b^t are formed on the
-// host in double and passed in as reciprocals, as are 1-b1 and 1-b2 (the
-// arguments are the binary32 values of lr, b1, b2, eps the caller passed).
+// Elementwise AdamW in binary32 (adamw_update in common.cuh).
 __global__ void adamw_kernel(float* __restrict__ s, const float* __restrict__ grad,
                              float* __restrict__ m, float* __restrict__ v, long long n,
-                             float lr, float b1, float b2, float omb1, float omb2, float eps,
-                             float decay, float inv_c1, float inv_c2) {
+                             const AdamWConsts c) {
   long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   const long long stride = (long long)gridDim.x * blockDim.x;
   for (; i < n; i += stride) {
-    const float gr = grad[i];
-    const float mn = b1 * m[i] + omb1 * gr;
-    const float vn = b2 * v[i] + omb2 * gr * gr;
-    const float denom = sqrtf(vn * inv_c2) + eps;
-    s[i] = s[i] * decay - lr * (mn * inv_c1) / denom;
-    m[i] = mn;
-    v[i] = vn;
+    float sv = s[i], mv = m[i], vv = v[i];
+    adamw_update(sv, grad[i], mv, vv, c);
+    s[i] = sv;
+    m[i] = mv;
+    v[i] = vv;
   }
 }
 
@@ -446,14 +441,9 @@ extern "C" int peqa_scale_adamw(float* scales, const float* dS, float* m, float*
   if (!scales || !dS || !m || !v) return PEQA_ERR_NULL;
   if (numel <= 0 || step < 1) return PEQA_ERR_BAD_SHAPE;
   PEQA_TRY(check_arch());
-  const double c1 = 1.0 - pow((double)beta1, (double)step);
-  const double c2 = 1.0 - pow((double)beta2, (double)step);
-  const float decay = (float)(1.0 - (double)lr * (double)weight_decay);
   const int grid = grid_for(numel, 256);
-  adamw_kernel<<<grid, 256, 0, as_stream(stream)>>>(scales, dS, m, v, (long long)numel, lr, beta1,
-                                                   beta2, (float)(1.0 - (double)beta1),
-                                                   (float)(1.0 - (double)beta2), eps, decay,
-                                                   (float)(1.0 / c1), (float)(1.0 / c2));
+  adamw_kernel<<<grid, 256, 0, as_stream(stream)>>>(scales, dS, m, v, (long long)numel,
+                                                   adamw_consts(lr, beta1, beta2, eps, weight_decay, step));
   PEQA_CUDA(cudaGetLastError());
   return PEQA_OK;
 }

@@ -457,6 +457,11 @@ struct DsParams {
   float* out;        // [N, K / piece]: dS itself when piece == g, else partial sums
   float* out_z;      // same shape: dZ (or its partial sums of dW); only read by ds_kernel<.., true>
   const float* scales;
+  // ds_kernel<.., ADAM = true> and the reduction kernel: AdamW applied where dS is final
+  AdamWConsts adam;
+  float* adam_s;
+  float* adam_m;
+  float* adam_v;
   int N, K, G, g, T;
   int wpr;
   int piece;         // columns per output piece: 32, 64 or 128; divides g
@@ -482,7 +487,7 @@ struct DsBarriers {
   int abort_flag;
 };
 
-template <int BITS, bool DZ>
+template <int BITS, bool DZ, bool ADAM>
 __global__ void __launch_bounds__(kDsThreads, 1)
 ds_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_constant__ CUtensorMap tmap_x,
           const DsParams p) {
@@ -628,6 +633,16 @@ ds_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_constant__ C
         if (((cc + 1) % chunks_per_piece) == 0) {
           if (row_ok) {
             p.out[(size_t)i * npieces + col0 / p.piece] = acc;
+            if (ADAM) {
+              // pieces are whole groups here (the launcher only asks for this then): acc is
+              // the final dS of scale (i, group), owned by this thread alone
+              const size_t e = (size_t)i * npieces + col0 / p.piece;
+              float sv = p.adam_s[e], mv = p.adam_m[e], vv = p.adam_v[e];
+              adamw_update(sv, acc, mv, vv, p.adam);
+              p.adam_s[e] = sv;
+              p.adam_m[e] = mv;
+              p.adam_v[e] = vv;
+            }
             if (DZ) {
               // a piece that is a whole group is dZ itself: -s * sum of dW; otherwise the
               // reduction kernel applies -s after adding the pieces
@@ -660,16 +675,26 @@ ds_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_constant__ C
 }
 
 // dS[i, gi] = sum of the group's partial pieces, in index order (deterministic); with
-// neg_scales the sum is multiplied by -s[i, gi] (the zero-point gradient).
+// neg_scales the sum is multiplied by -s[i, gi] (the zero-point gradient); with adam_s the
+// AdamW step on scale e follows at once.
 __global__ void ds_reduce_kernel(const float* __restrict__ partial, float* __restrict__ dS,
                                  long long n_out, int pieces_per_group,
-                                 const float* __restrict__ neg_scales) {
+                                 const float* __restrict__ neg_scales, AdamWConsts adam,
+                                 float* __restrict__ adam_s, float* __restrict__ adam_m,
+                                 float* __restrict__ adam_v) {
   long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (e >= n_out) return;
   const float* src = partial + e * pieces_per_group;
   float acc = 0.0f;
   for (int q = 0; q < pieces_per_group; ++q) acc += src[q];
   dS[e] = neg_scales ? -neg_scales[e] * acc : acc;
+  if (adam_s) {
+    float sv = adam_s[e], mv = adam_m[e], vv = adam_v[e];
+    adamw_update(sv, acc, mv, vv, adam);
+    adam_s[e] = sv;
+    adam_m[e] = mv;
+    adam_v[e] = vv;
+  }
 }
 
 // --------------------------------------------------------------- host side
@@ -828,7 +853,8 @@ size_t dsdz_workspace_bytes(const peqa_qweight_t* w, int g, int T) {
 }
 
 int launch_ds(const peqa_qweight_t* w, int g, const void* X, const void* dY, int T, float* dS,
-              float* dZ, void* workspace, size_t workspace_bytes, cudaStream_t st) {
+              float* dZ, const DsAdam* adam, void* workspace, size_t workspace_bytes, cudaStream_t st) {
+  if (adam && dZ) return PEQA_ERR_BAD_SHAPE;   // dZ reads the scales the step would be rewriting
   (void)workspace_bytes;
   DsParams p;
   p.qw = w->qweight;
@@ -845,6 +871,11 @@ int launch_ds(const peqa_qweight_t* w, int g, const void* X, const void* dY, int
   p.scales = w->scales;
   const size_t n_pieces = (size_t)p.N * (size_t)(p.K / p.piece);
   p.out_z = dZ ? (direct ? dZ : static_cast<float*>(workspace) + n_pieces) : nullptr;
+  p.adam = adam ? adam->c : AdamWConsts{};
+  p.adam_s = adam ? adam->scales : nullptr;
+  p.adam_m = adam ? adam->m : nullptr;
+  p.adam_v = adam ? adam->v : nullptr;
+  const bool adam_in_kernel = adam && direct;
   p.i_tiles = (p.N + 2 * BM - 1) / (2 * BM);   // 256-row pair tiles
   p.j_tiles = (p.K + BN - 1) / BN;
   p.k_blocks = (T + BK - 1) / BK;
@@ -869,26 +900,33 @@ int launch_ds(const peqa_qweight_t* w, int g, const void* X, const void* dY, int
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-#define PEQA_DS_LAUNCH(B, Z)                                                                          \
+#define PEQA_DS_LAUNCH(B, Z, A)                                                                       \
   do {                                                                                               \
-    PEQA_CUDA(cudaFuncSetAttribute(ds_kernel<B, Z>, cudaFuncAttributeMaxDynamicSharedMemorySize,     \
+    auto kern = ds_kernel<B, Z, A>;                                                                  \
+    PEQA_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,                \
                                    DS_SMEM_BYTES));                                                  \
-    PEQA_CUDA(cudaLaunchKernelEx(&cfg, ds_kernel<B, Z>, tmap_dy, tmap_x, p));                        \
+    PEQA_CUDA(cudaLaunchKernelEx(&cfg, kern, tmap_dy, tmap_x, p));                                   \
   } while (0)
   if (w->bits == 4) {
-    if (dZ) PEQA_DS_LAUNCH(4, true); else PEQA_DS_LAUNCH(4, false);
+    if (dZ) PEQA_DS_LAUNCH(4, true, false);
+    else if (adam_in_kernel) PEQA_DS_LAUNCH(4, false, true);
+    else PEQA_DS_LAUNCH(4, false, false);
   } else {
-    if (dZ) PEQA_DS_LAUNCH(3, true); else PEQA_DS_LAUNCH(3, false);
+    if (dZ) PEQA_DS_LAUNCH(3, true, false);
+    else if (adam_in_kernel) PEQA_DS_LAUNCH(3, false, true);
+    else PEQA_DS_LAUNCH(3, false, false);
   }
 #undef PEQA_DS_LAUNCH
   if (!direct) {
     const long long n_out = (long long)p.N * p.G;
     const int ppg = g / p.piece;
     const int blocks = (int)((n_out + 255) / 256);
-    ds_reduce_kernel<<<blocks, 256, 0, st>>>(p.out, dS, n_out, ppg, nullptr);
+    ds_reduce_kernel<<<blocks, 256, 0, st>>>(p.out, dS, n_out, ppg, nullptr, p.adam, p.adam_s,
+                                             p.adam_m, p.adam_v);
     PEQA_CUDA(cudaGetLastError());
     if (dZ) {
-      ds_reduce_kernel<<<blocks, 256, 0, st>>>(p.out_z, dZ, n_out, ppg, w->scales);
+      ds_reduce_kernel<<<blocks, 256, 0, st>>>(p.out_z, dZ, n_out, ppg, w->scales, AdamWConsts{},
+                                               nullptr, nullptr, nullptr);
       PEQA_CUDA(cudaGetLastError());
     }
   }

@@ -45,3 +45,35 @@ def test_zero_gradient_and_first_step_sign():
     binding.scale_adamw(s, g, m, v, 1e-3)
     torch.cuda.synchronize()
     assert torch.allclose(s, 0.5 - 1e-3 * torch.sign(g), atol=1e-7)
+
+
+@pytest.mark.parametrize("bits,g", [(3, 128), (4, 64), (3, 32), (4, 0), (3, 256)])
+def test_step_applied_where_ds_is_produced_equals_the_two_calls(bits, g):
+    """peqa_qlinear_bwd_ds_adamw against peqa_qlinear_bwd followed by peqa_scale_adamw:
+    the same bits in dS, scales, m and v, for groups that the dS kernel finishes itself
+    (g <= 128) and for those that go through the reduction kernel."""
+    from paper_2305_14152_b200 import synth
+    from gpu_util import bf16_to_dev, oracle_layer, to_qweight
+    N, K, T = 328, 768, 300
+    d = synth.custom(800 + bits + g, N, K, T, bits, g, outliers=True, sigma_dy=1e-2)
+    codes, zeros, scales, packed = oracle_layer(d, bits, g)
+    X, dY = bf16_to_dev(d["X"]), bf16_to_dev(d["dY"])
+    G = scales.shape[1]
+    rng = np.random.default_rng(3)
+    m0 = (rng.standard_normal((N, G)) * 1e-3).astype(np.float32)
+    v0 = (rng.random((N, G)) * 1e-5).astype(np.float32)
+    out = []
+    for fused in (False, True):
+        qw = to_qweight(packed, zeros, scales.copy(), bits, g, K)
+        m, v = torch.from_numpy(m0.copy()).cuda(), torch.from_numpy(v0.copy()).cuda()
+        if fused:
+            dS = binding.qlinear_bwd_ds_adamw(qw, X, dY, m, v, 1e-4, weight_decay=0.01, step=7)
+        else:
+            dS = binding.qlinear_bwd(qw, X, dY, need_dx=False)[1]
+            binding.scale_adamw(qw.scales, dS, m, v, 1e-4, 0.9, 0.999, 1e-8, 0.01, 7)
+        torch.cuda.synchronize()
+        out.append((dS.clone(), qw.scales.clone(), m, v))
+    binding.check_status()
+    for a, b in zip(out[0], out[1]):
+        assert torch.equal(a, b)
+    assert not torch.equal(out[0][1].cpu(), torch.from_numpy(scales))      # the scales did move
