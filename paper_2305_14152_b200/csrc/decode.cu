@@ -1,6 +1,8 @@
 // Small-batch forward (token generation): Y[m,i] = sum_j X[m,j] * s[i,g(j)] * (Q[i,j] - z[i,g(j)])
-// for M <= 16 tokens.  The packed weights are streamed from HBM exactly once
-// with 128-bit loads; everything else is sized so that the stream is the bound.
+// for M <= 16 tokens: the cluster kernel, used for groups narrower than 128
+// columns and for batches whose activations do not fit the streaming kernel's
+// staging (decode_stream.cu serves the rest).  The packed weights are read from
+// HBM exactly once, by TMA into a two-slot ring per CTA.
 //
 // Work split: a CTA owns 128 weight rows and one slice of the K range; the
 // CTAs that share the same rows form a thread-block cluster along K and add
@@ -77,20 +79,6 @@ template <int BITS>
 struct RowChunk {
   uint4 v[BITS];
 };
-
-template <int BITS>
-__device__ __forceinline__ RowChunk<BITS> load_chunk(const DecodeParams& p, int row, int col) {
-  RowChunk<BITS> r;
-  if (row < p.N && col < p.K) {
-    const uint4* src = reinterpret_cast<const uint4*>(p.qw + (size_t)row * p.wpr + (col >> 5) * BITS);
-#pragma unroll
-    for (int q = 0; q < BITS; ++q) r.v[q] = __ldg(src + q);
-  } else {
-#pragma unroll
-    for (int q = 0; q < BITS; ++q) r.v[q] = make_uint4(0u, 0u, 0u, 0u);
-  }
-  return r;
-}
 
 template <int BITS>
 __device__ __forceinline__ void unit_words(const RowChunk<BITS>& r, int u, uint32_t (&w)[BITS]) {

@@ -273,10 +273,18 @@ qdx_pair_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_consta
       uint32_t wa[BITS], wb[BITS];
       {
         const uint32_t* src = reinterpret_cast<const uint32_t*>(sm_q + q * XQ_BYTES) + u4 * BITS;
+        if constexpr (BITS == 4) {
+          // a unit is 16 aligned bytes: one vector load per row
+          const uint4 va = *reinterpret_cast<const uint4*>(src + row_a * 16);
+          const uint4 vb = *reinterpret_cast<const uint4*>(src + row_b * 16);
+          wa[0] = va.x; wa[1] = va.y; wa[2] = va.z; wa[3] = va.w;
+          wb[0] = vb.x; wb[1] = vb.y; wb[2] = vb.z; wb[3] = vb.w;
+        } else {
 #pragma unroll
-        for (int e = 0; e < BITS; ++e) {
-          wa[e] = src[row_a * (4 * BITS) + e];
-          wb[e] = src[row_b * (4 * BITS) + e];
+          for (int e = 0; e < BITS; ++e) {
+            wa[e] = src[row_a * (4 * BITS) + e];
+            wb[e] = src[row_b * (4 * BITS) + e];
+          }
         }
       }
       uint32_t oa[16], ob[16];
