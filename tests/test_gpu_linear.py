@@ -59,6 +59,14 @@ def test_token_tail_beyond_one_block(g):
         _run_all(d, 4, g)
 
 
+@pytest.mark.parametrize("bits,g,N,K,T", [(4, 0, 8, 64, 3), (3, 0, 8, 64, 1), (4, 32, 40, 128, 513),
+                                          (3, 128, 24, 128, 9), (4, 64, 8, 4096, 2)])
+def test_layers_smaller_than_one_tile(bits, g, N, K, T):
+    # every TMA box is larger than the tensor it reads; 3-bit K=64 takes the single-CTA kernels
+    d = synth.custom(500 + N + K + T, N, K, T, bits, g, outliers=True, sigma_dy=1e-2)
+    _run_all(d, bits, g)
+
+
 @pytest.mark.parametrize("T", [1, 7, 64, 257, 513])
 def test_token_counts(T):
     d = synth.custom(T, 256, 512, T, 3, 128, sigma_dy=1e-2)
