@@ -29,8 +29,11 @@
 // That lets the codes go to the tensor core as the biased integers (bias + q)
 // they already are after one logic operation, and the group's zero-point and
 // scale are applied to the accumulator once per 128 columns:
-//   y += s * (acc - (bias_lo + z) * sum_lo(x) - (bias_hi + z) * sum_hi(x)),
-// with the sums of the activations per 128-column block tabulated once per CTA.
+//   y += s * (acc - z * sum(x) - sum(bias * x)),
+// with both sums per 128-column block tabulated once per CTA.  Because the
+// order of the contraction is free here (the activations are staged to match),
+// 3-bit codes are taken two pairs per shifted window (stream_lo / stream_hi in
+// dequant.cuh), a fifth fewer integer operations than pairing (k, k+4) only.
 // The products are exact integers times bf16 in fp32, which is also closer to
 // the reference than multiplying by a bf16-rounded scale first.
 //
@@ -104,8 +107,8 @@ __device__ __forceinline__ void smma_16816(float (&d)[4], const uint32_t (&a)[4]
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
-// MMAs of 4 columns (pairs (E, E+4) and (E+1, E+5) of the 8-column block BLK of the lane's
-// 32-column unit, E = 2*HH) for both 16-row halves of the 32-row block.
+// MMA 2*BLK + HH of the lane's 32-column unit (pairs 4*BLK + 2*HH and the next one, see
+// stream_lo in dequant.cuh) for both 16-row halves of the 32-row block.
 template <int BITS, int NT, int BLK, int HH>
 __device__ __forceinline__ void unit_mma(const uint32_t (&w)[4][BITS], const uint8_t* x0,
                                          const uint8_t* x1, float (&acc)[2][NT][4]) {
@@ -115,10 +118,8 @@ __device__ __forceinline__ void unit_mma(const uint32_t (&w)[4][BITS], const uin
 #pragma unroll
   for (int rb = 0; rb < 2; ++rb) {
     uint32_t a[4];
-    a[0] = dq::pair_raw<BITS, 8 * BLK + 2 * HH>(w[2 * rb]);
-    a[2] = dq::pair_raw<BITS, 8 * BLK + 2 * HH + 1>(w[2 * rb]);
-    a[1] = dq::pair_raw<BITS, 8 * BLK + 2 * HH>(w[2 * rb + 1]);
-    a[3] = dq::pair_raw<BITS, 8 * BLK + 2 * HH + 1>(w[2 * rb + 1]);
+    dq::mma_pairs_stream<BITS, 2 * BLK + HH>(w[2 * rb], a[0], a[2]);
+    dq::mma_pairs_stream<BITS, 2 * BLK + HH>(w[2 * rb + 1], a[1], a[3]);
     smma_16816(acc[rb][0], a, b0.x, b0.y);
     if (NT == 2) smma_16816(acc[rb][1], a, b1.x, b1.y);
   }
@@ -129,8 +130,6 @@ __global__ void __launch_bounds__(kSBlock, 1)
 decode_stream_kernel(const StreamParams p) {
   using Geo = StreamGeom<BITS>;
   constexpr int TOKP = 8 * NT;                       // token columns of the MMAs
-  constexpr float kBiasLo = BITS == 4 ? 128.0f : 8.0f;
-  constexpr float kBiasHi = 128.0f;
   extern __shared__ uint8_t stream_smem_raw[];
   uint8_t* ring = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(stream_smem_raw) + 127) &
                                              ~static_cast<uintptr_t>(127));
@@ -151,7 +150,7 @@ decode_stream_kernel(const StreamParams p) {
 
   // The activation loads are issued before the weight copies start: behind a CTA's worth
   // of weight traffic they would wait for microseconds, and everything waits for them.
-  const int blocks8 = p.x_blocks * 16;                 // 8-column blocks per token, zero past K
+  const int units = p.x_blocks * 4;                    // 32-column units per token, zero past K
   uint4 xv[kSMaxXLoads];
   if (threadIdx.x == kSThreads) {
     for (int q = 0; q < p.slots; ++q) {
@@ -162,12 +161,16 @@ decode_stream_kernel(const StreamParams p) {
     ptx::fence_mbar_init();
   } else if (!is_producer) {
 #pragma unroll
-    for (int q = 0; q < kSMaxXLoads; ++q) {
-      const int idx = q * kSThreads + threadIdx.x;
-      const int m = idx / blocks8;
-      const int col = (idx - m * blocks8) * 8;
-      xv[q] = make_uint4(0u, 0u, 0u, 0u);
-      if (m < p.M && col < p.K) xv[q] = __ldg(reinterpret_cast<const uint4*>(p.X + (size_t)m * p.K + col));
+    for (int q = 0; q < kSMaxXLoads / 4; ++q) {
+      const int idx = q * kSThreads + threadIdx.x;       // one 32-column unit of one token
+      const int m = idx / units;
+      const int col = (idx - m * units) * 32;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        xv[4 * q + e] = make_uint4(0u, 0u, 0u, 0u);
+        if (m < p.M && col + 8 * e < p.K)
+          xv[4 * q + e] = __ldg(reinterpret_cast<const uint4*>(p.X + (size_t)m * p.K + col + 8 * e));
+      }
     }
   }
   __syncthreads();
@@ -207,41 +210,64 @@ decode_stream_kernel(const StreamParams p) {
     }
   } else {
     // ------------------------------------------------ stage the activations
-    // blocks of 8 columns stored as (0,4,1,5,2,6,3,7): the order of the bf16 pairs that one
-    // logic operation extracts from the packed codes; columns beyond K are zero
+    // A unit of 32 columns is stored as its 16 pairs (low column, high column) in the order
+    // in which the weights' pairs come out of the packed codes (stream_lo, stream_hi), so that MMA
+    // m of a unit reads its four activations as one 8-byte word; columns beyond K are zero.
 #pragma unroll
-    for (int q = 0; q < kSMaxXLoads; ++q) {
+    for (int q = 0; q < kSMaxXLoads / 4; ++q) {
       const int idx = q * kSThreads + threadIdx.x;
-      const int m = idx / blocks8;
-      const int col = (idx - m * blocks8) * 8;
+      const int m = idx / units;
+      const int col = (idx - m * units) * 32;
       if (m < p.M) {
-        const uint4 v = xv[q];
-        uint8_t* dst = xs + (size_t)m * p.x_pitch + (col >> 7) * kSBlockBytes + (col & 127) * 2;
-        *reinterpret_cast<uint2*>(dst) =
-            make_uint2(dq::prmt(v.x, v.z, 0x5410u), dq::prmt(v.x, v.z, 0x7632u));
-        *reinterpret_cast<uint2*>(dst + 8) =
-            make_uint2(dq::prmt(v.y, v.w, 0x5410u), dq::prmt(v.y, v.w, 0x7632u));
+        const uint32_t src[16] = {xv[4 * q].x, xv[4 * q].y, xv[4 * q].z, xv[4 * q].w,
+                                  xv[4 * q + 1].x, xv[4 * q + 1].y, xv[4 * q + 1].z, xv[4 * q + 1].w,
+                                  xv[4 * q + 2].x, xv[4 * q + 2].y, xv[4 * q + 2].z, xv[4 * q + 2].w,
+                                  xv[4 * q + 3].x, xv[4 * q + 3].y, xv[4 * q + 3].z, xv[4 * q + 3].w};
+        uint32_t outw[16];
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {
+          const int lo = dq::stream_lo(BITS, k), hi = dq::stream_hi(BITS, k);
+          // bytes 0-1: column lo (half lo % 2 of its word), bytes 2-3: column hi
+          const uint32_t sel = (uint32_t)(2 * (lo & 1)) | ((uint32_t)(2 * (lo & 1) + 1) << 4) |
+                               ((uint32_t)(4 + 2 * (hi & 1)) << 8) | ((uint32_t)(5 + 2 * (hi & 1)) << 12);
+          outw[k] = dq::prmt(src[lo >> 1], src[hi >> 1], sel);
+        }
+        // token rows are 8-byte aligned only (their pitch is skewed by 8 bytes)
+        uint2* dst = reinterpret_cast<uint2*>(xs + (size_t)m * p.x_pitch + (col >> 7) * kSBlockBytes +
+                                              (col & 127) * 2);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) dst[e] = make_uint2(outw[2 * e], outw[2 * e + 1]);
       }
     }
     // entries of tokens beyond M are read by the lanes that hold those (unused) columns
     for (int idx = threadIdx.x; idx < p.x_blocks * TOKP * 2; idx += kSThreads) xtab[idx] = 0.0f;
     ptx::named_barrier_sync(1, kSThreads);
-    // Sums of the staged activations per 128-column block, separately over the columns
-    // that land in the low and in the high half of the bf16 pairs (they carry different
-    // biases).  In the staged order every 32-bit word is one (low, high) pair.
+    // Per 128-column block and token: S = sum of the staged activations and B = sum of
+    // (bias of the code that meets it) * activation.  The MMAs see (bias + q), so what has
+    // to come off the accumulator is sum (bias + z) x = z * S + B.  In the staged order every
+    // 32-bit word is one (low, high) pair and word k of a unit is pair k: lane l reads words
+    // l and l + 32 of the block, both pair l % 16.
+    float bias_lo = 128.0f, bias_hi = 128.0f;
+    if (BITS == 3) {
+      const bool alt = (dq::stream_alt_mask3() >> (lane & 15)) & 1u;
+      bias_lo = alt ? 64.0f : 8.0f;
+      bias_hi = alt ? 16.0f : 128.0f;
+    }
     for (int idx = warp; idx < p.x_blocks * p.M; idx += kSWarps) {
       const int blk = idx / p.M, m = idx - blk * p.M;
       const uint32_t* wds =
           reinterpret_cast<const uint32_t*>(xs + (size_t)m * p.x_pitch + blk * kSBlockBytes);
       const uint32_t v0 = wds[lane], v1 = wds[lane + 32];
-      float lo = __uint_as_float(v0 << 16) + __uint_as_float(v1 << 16);
-      float hi = __uint_as_float(v0 & 0xFFFF0000u) + __uint_as_float(v1 & 0xFFFF0000u);
+      const float lo = __uint_as_float(v0 << 16) + __uint_as_float(v1 << 16);
+      const float hi = __uint_as_float(v0 & 0xFFFF0000u) + __uint_as_float(v1 & 0xFFFF0000u);
+      float sm = lo + hi;
+      float bs = fmaf(bias_hi, hi, bias_lo * lo);
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) {
-        lo += __shfl_xor_sync(0xffffffffu, lo, o);
-        hi += __shfl_xor_sync(0xffffffffu, hi, o);
+        sm += __shfl_xor_sync(0xffffffffu, sm, o);
+        bs += __shfl_xor_sync(0xffffffffu, bs, o);
       }
-      if (lane == 0) { xtab[(blk * TOKP + m) * 2] = lo; xtab[(blk * TOKP + m) * 2 + 1] = hi; }
+      if (lane == 0) { xtab[(blk * TOKP + m) * 2] = sm; xtab[(blk * TOKP + m) * 2 + 1] = bs; }
     }
     ptx::named_barrier_sync(1, kSThreads);
     if (!GROUPED && warp < p.M) {
@@ -355,15 +381,14 @@ decode_stream_kernel(const StreamParams p) {
 #pragma unroll
               for (int nt = 0; nt < NT; ++nt) {
                 const float4 xt = *reinterpret_cast<const float4*>(
-                    xtab + ((size_t)(ch * 4 + j) * TOKP + nt * 8 + 2 * c4) * 2);   // lo0 hi0 lo1 hi1
+                    xtab + ((size_t)(ch * 4 + j) * TOKP + nt * 8 + 2 * c4) * 2);   // S0 B0 S1 B1
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
 #pragma unroll
                   for (int q = 0; q < 2; ++q) {      // q = 0: row g8 of the half, q = 1: row g8 + 8
                     const float z = zq[2 * h + q][j], sc = sq[2 * h + q][j];
-                    const float ca = kBiasLo + z, cb = kBiasHi + z;
-                    const float c0 = fmaf(cb, xt.y, ca * xt.x);
-                    const float c1 = fmaf(cb, xt.w, ca * xt.z);
+                    const float c0 = fmaf(z, xt.x, xt.y);      // z * S + B, token tk
+                    const float c1 = fmaf(z, xt.z, xt.w);      // token tk + 1
                     tot[h][nt][2 * q] = fmaf(sc, acc[h][nt][2 * q] - c0, tot[h][nt][2 * q]);
                     tot[h][nt][2 * q + 1] = fmaf(sc, acc[h][nt][2 * q + 1] - c1, tot[h][nt][2 * q + 1]);
                     acc[h][nt][2 * q] = 0.0f;
@@ -408,8 +433,7 @@ decode_stream_kernel(const StreamParams p) {
               const int task = min(max(__ldg(p.task_ids + m), 0), p.n_tasks - 1);
               sc += (size_t)task * p.N;
             }
-            sum = (sum - (kBiasLo + z) * xtot[m * 2] - (kBiasHi + z) * xtot[m * 2 + 1]) *
-                  __ldg(sc + row);
+            sum = (sum - fmaf(z, xtot[m * 2], xtot[m * 2 + 1])) * __ldg(sc + row);
           }
           p.Y[(size_t)m * p.N + row] = __float2bfloat16_rn(sum);
         }

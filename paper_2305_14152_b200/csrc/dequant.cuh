@@ -124,5 +124,95 @@ __device__ __forceinline__ void unit32_natural(const uint32_t (&w)[BITS], uint32
   block8_natural<BITS, 3, FOLD>(w, zc, s2, out + 12);
 }
 
+// ---------------------------------------------------------------------------
+// Pairing for kernels whose contraction order is free (the streaming decode
+// kernel: the activations are staged in whatever order the weights come out).
+//
+// A 3-bit code fits the 7 mantissa bits of a bf16 at any start bit p in 0..4,
+// and with the exponent chosen so that one code step is 1.0 it reads as
+// 2^(7-p) + q.  So one shifted window of the packed string can yield TWO pairs
+// with two logic operations: with column A at bit 4 it holds
+//   (A    at bit 4,  bias 8)   with  (A + 4 at bit 16, bias 128)   "std"
+//   (A - 1 at bit 1, bias 64)  with  (A + 5 at bit 19, bias 16)    "alt"
+// and a lone pair six columns apart can be taken as (bit 1, bit 19).  The 32
+// columns of a unit split into six such double windows and four single ones
+// (ten shifts, one of them by zero, and sixteen logic operations instead of
+// sixteen of each).  Pair k of the unit, k = 0..15, is (stream_lo(k), stream_hi(k)); MMA
+// m of the unit takes pairs 2m and 2m + 1.  4-bit codes have no second start
+// position in a bf16 mantissa: their pairs stay (8b + e, 8b + e + 4).
+// ---------------------------------------------------------------------------
+// windows: A = 1, A = 3, (4,10), (9,13), A = 12, A = 15, (18,22), (21,27), A = 24, A = 26
+__host__ __device__ constexpr int stream_lo(int bits, int k) {
+  constexpr int lo3[16] = {1, 0, 3, 2, 4, 9, 12, 11, 15, 14, 18, 21, 24, 23, 26, 25};
+  return bits == 3 ? lo3[k] : 8 * (k / 4) + k % 4;
+}
+__host__ __device__ constexpr int stream_hi(int bits, int k) {
+  constexpr int hi3[16] = {5, 6, 7, 8, 10, 13, 16, 17, 19, 20, 22, 27, 28, 29, 30, 31};
+  return bits == 3 ? hi3[k] : 8 * (k / 4) + k % 4 + 4;
+}
+// "alt" pairs sit at bits (1, 19) of their window and carry the biases (64, 16); the others
+// sit at bits (4, 16) and carry (8, 128).  4-bit pairs carry (128, 128).
+__host__ __device__ constexpr bool stream_alt(int bits, int k) {
+  constexpr bool alt3[16] = {false, true, false, true, true, false, false, true,
+                             false, true, false, true, false, true, false, true};
+  return bits == 3 ? alt3[k] : false;
+}
+__host__ __device__ constexpr uint32_t stream_alt_mask3() {
+  uint32_t m = 0;
+  for (int k = 0; k < 16; ++k) m |= (stream_alt(3, k) ? 1u : 0u) << k;
+  return m;
+}
+
+// 32-bit window of the 96-bit string starting at bit START (may be -1), of which bits
+// 0..21 are used.
+template <int START>
+__device__ __forceinline__ uint32_t window3_wide(const uint32_t (&w)[3]) {
+  if constexpr (START < 0) {
+    return w[0] << (-START);
+  } else {
+    constexpr int a = START / 32;
+    constexpr int sh = START % 32;
+    if constexpr (sh == 0) {
+      return w[a];
+    } else if constexpr (sh + 22 <= 32 || a == 2) {
+      return w[a] >> sh;
+    } else {
+      return __funnelshift_r(w[a], w[a + 1], sh);
+    }
+  }
+}
+
+// The two biased bf16x2 registers of MMA M (pairs 2M and 2M + 1) of a unit.
+template <int BITS, int M>
+__device__ __forceinline__ void mma_pairs_stream(const uint32_t (&w)[BITS], uint32_t& p0,
+                                                 uint32_t& p1) {
+  if constexpr (BITS == 4) {
+    // pairs (8b + e, +4) and (8b + e + 1, +4) with b = M / 2, e = 2 * (M % 2)
+    p0 = pair_raw<4, 8 * (M / 2) + 2 * (M % 2)>(w);
+    p1 = pair_raw<4, 8 * (M / 2) + 2 * (M % 2) + 1>(w);
+  } else {
+    constexpr uint32_t kStdMask = 0x00070070u, kStdMagic = 0x43004100u;   // bits 4-6 | 16-18
+    constexpr uint32_t kAltMask = 0x0038000Eu, kAltMagic = 0x41804280u;   // bits 1-3 | 19-21
+    constexpr int k0 = 2 * M, k1 = 2 * M + 1;
+    if constexpr (!stream_alt(3, k0) && stream_alt(3, k1) &&
+                  stream_lo(3, k1) == stream_lo(3, k0) - 1) {
+      // a double window: column lo[k0] at bit 4
+      const uint32_t x = window3_wide<3 * stream_lo(3, k0) - 4>(w);
+      p0 = lop3_and_or(x, kStdMask, kStdMagic);
+      p1 = lop3_and_or(x, kAltMask, kAltMagic);
+    } else {
+      // two single windows
+      if constexpr (stream_alt(3, k0))
+        p0 = lop3_and_or(window3_wide<3 * stream_lo(3, k0) - 1>(w), kAltMask, kAltMagic);
+      else
+        p0 = lop3_and_or(window3_wide<3 * stream_lo(3, k0) - 4>(w), kStdMask, kStdMagic);
+      if constexpr (stream_alt(3, k1))
+        p1 = lop3_and_or(window3_wide<3 * stream_lo(3, k1) - 1>(w), kAltMask, kAltMagic);
+      else
+        p1 = lop3_and_or(window3_wide<3 * stream_lo(3, k1) - 4>(w), kStdMask, kStdMagic);
+    }
+  }
+}
+
 }  // namespace dq
 }  // namespace peqa
