@@ -42,7 +42,7 @@ def test_single_step_and_tiny_rows():
 
 @pytest.mark.parametrize("M", [1, 4, 16])
 def test_c4_llama65b_shapes(M):
-    """BASELINE config 4 at full size: 3-bit per-channel, three layer shapes."""
+    """Workload c4 (LLaMA-65B decode shapes) at full size: 3-bit per-channel, three layer shapes."""
     for d in synth.generate("c4"):
         _check(d, 3, 0, M)
 

@@ -39,7 +39,7 @@ def test_matches_the_oracle_on_the_same_stored_output(bits, N, K, T):
 
 
 def test_c3_gate_projection_full_size():
-    """BASELINE config 3 (LLaMA-7B MLP, 4-bit per-channel) at full size, every channel."""
+    """Workload c3 (LLaMA-7B MLP, 4-bit per-channel) at full size, every channel."""
     d = next(synth.generate("c3"))
     codes, zeros, scales, packed = oracle_layer(d, 4, 0)
     K = d["W"].shape[1]

@@ -130,7 +130,7 @@ def test_skipping_outputs_and_workspace_errors():
 
 
 def test_c2_llama7b_attention_projection_full():
-    """BASELINE config 2 at full size; the oracle finishes each tensor in seconds."""
+    """Workload c2 (LLaMA-7B attention projection) at full size; the oracle finishes each tensor in seconds."""
     d = next(synth.generate("c2"))
     res = _run_all(d, 3, 128)
     print("c2 errors (rel-L2, max-abs):", res)
