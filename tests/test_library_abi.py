@@ -58,6 +58,21 @@ def test_argument_validation_needs_no_gpu(L):
     assert L.peqa_qlinear_fwd(ctypes.byref(w3), p16, 8, p16, 0, 0, 0) == -3      # N % 8
     assert L.peqa_qlinear_decode(ctypes.byref(w), p16, 17, p16, 0, 0, 0) == -3
     assert L.peqa_qlinear_bwd(ctypes.byref(w), p16, 0, 8, p16, 0, 0, 0, 0) == -1
+    # the entry points beyond the basic five: null pointers, shapes and modes they do not take
+    wg = binding._QWeight(4, 128, 256, 128, p16, p16, p16)           # two groups per row
+    assert L.peqa_qlinear_bwd_ds_from_y(ctypes.byref(w), p16, 0, 8, p16, p16, 4096, 0) == -1
+    assert L.peqa_qlinear_bwd_ds_from_y(ctypes.byref(wg), p16, p16, 8, p16, p16, 4096, 0) == -3
+    assert L.peqa_qlinear_bwd_ds_from_y(ctypes.byref(w), p16, p16, 0, p16, p16, 4096, 0) == -3
+    assert L.peqa_qlinear_bwd_dsdz(ctypes.byref(w), p16, p16, 8, p16, 0, 0, 0, 0) == -1
+    assert L.peqa_qlinear_bwd_dsdz(ctypes.byref(w2), p16, p16, 8, p16, p16, 0, 0, 0) == -3
+    assert L.peqa_qlinear_bwd_ds_adamw(ctypes.byref(w), p16, p16, 8, p16, p16, 0, 1e-3, 0.9, 0.999,
+                                       1e-8, 0.0, 1, 0, 0, 0) == -1
+    assert L.peqa_qlinear_bwd_ds_adamw(ctypes.byref(w), p16, p16, 8, p16, p16, p16, 1e-3, 0.9, 0.999,
+                                       1e-8, 0.0, 0, 0, 0, 0) == -3             # step counts from 1
+    assert L.peqa_qlinear_decode_multitask(ctypes.byref(w), p16, 2, 0, p16, 1, p16, 0) == -1
+    assert L.peqa_qlinear_decode_multitask(ctypes.byref(wg), p16, 2, p16, p16, 1, p16, 0) == -3
+    assert L.peqa_qlinear_decode_multitask(ctypes.byref(w), p16, 0, p16, p16, 1, p16, 0) == -3
+    assert L.peqa_qlinear_decode_multitask(ctypes.byref(w), p16, 2, p16, p16, 17, p16, 0) == -3
 
 
 def test_workspace_query(L):
@@ -66,3 +81,9 @@ def test_workspace_query(L):
     w = binding._QWeight(3, 4096, 4096, 128, 16, 16, 16)
     assert L.peqa_workspace_bytes(binding.OP_BWD, 2048, ctypes.byref(w)) == 0
     assert L.peqa_workspace_bytes(binding.OP_FWD, 2048, ctypes.byref(w)) == 0
+    assert L.peqa_workspace_bytes(binding.OP_BWD_DSDZ, 2048, ctypes.byref(w)) == 0
+    assert L.peqa_workspace_bytes(binding.OP_BWD_DS_FROM_Y, 2048, ctypes.byref(w)) == 0   # grouped: not served
+    w = binding._QWeight(4, 4096, 4096, 0, 16, 16, 16)
+    assert L.peqa_workspace_bytes(binding.OP_BWD_DSDZ, 2048, ctypes.byref(w)) == 2 * 4096 * (4096 // 128) * 4
+    n = L.peqa_workspace_bytes(binding.OP_BWD_DS_FROM_Y, 2048, ctypes.byref(w))
+    assert n > 0 and n % (4096 * 4) == 0
