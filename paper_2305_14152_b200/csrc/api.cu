@@ -201,8 +201,10 @@ constexpr int kHostChunksMax = 8;
 struct HostPipe {
   cudaStream_t in = nullptr, out = nullptr;
   cudaEvent_t start = nullptr, out_done = nullptr;
-  cudaEvent_t landed[kHostChunksMax] = {};
-  cudaEvent_t computed[kHostChunksMax] = {};
+  cudaEvent_t x_landed[kHostChunksMax] = {};
+  cudaEvent_t dy_landed[kHostChunksMax] = {};
+  cudaEvent_t fwd_done[kHostChunksMax] = {};
+  cudaEvent_t dx_done[kHostChunksMax] = {};
   bool ready = false;
 };
 
@@ -218,8 +220,10 @@ int host_pipe(HostPipe** out) {
     PEQA_CUDA(cudaEventCreateWithFlags(&hp.start, cudaEventDisableTiming));
     PEQA_CUDA(cudaEventCreateWithFlags(&hp.out_done, cudaEventDisableTiming));
     for (int c = 0; c < kHostChunksMax; ++c) {
-      PEQA_CUDA(cudaEventCreateWithFlags(&hp.landed[c], cudaEventDisableTiming));
-      PEQA_CUDA(cudaEventCreateWithFlags(&hp.computed[c], cudaEventDisableTiming));
+      PEQA_CUDA(cudaEventCreateWithFlags(&hp.x_landed[c], cudaEventDisableTiming));
+      PEQA_CUDA(cudaEventCreateWithFlags(&hp.dy_landed[c], cudaEventDisableTiming));
+      PEQA_CUDA(cudaEventCreateWithFlags(&hp.fwd_done[c], cudaEventDisableTiming));
+      PEQA_CUDA(cudaEventCreateWithFlags(&hp.dx_done[c], cudaEventDisableTiming));
     }
     hp.ready = true;
   }
@@ -275,16 +279,22 @@ extern "C" int peqa_train_step_host(const peqa_qweight_t* w, int T,
     const size_t t0 = (size_t)c * per;
     const size_t tc = (size_t)T - t0 < (size_t)per ? (size_t)T - t0 : (size_t)per;
     PEQA_CUDA(cudaMemcpyAsync(dX_in + t0 * K * 2, hX + t0 * K * 2, tc * K * 2, cudaMemcpyHostToDevice, hp->in));
+    PEQA_CUDA(cudaEventRecord(hp->x_landed[c], hp->in));
     PEQA_CUDA(cudaMemcpyAsync(ddY + t0 * N * 2, hdY + t0 * N * 2, tc * N * 2, cudaMemcpyHostToDevice, hp->in));
-    PEQA_CUDA(cudaEventRecord(hp->landed[c], hp->in));
-    PEQA_CUDA(cudaStreamWaitEvent(st, hp->landed[c], 0));
+    PEQA_CUDA(cudaEventRecord(hp->dy_landed[c], hp->in));
+    // the forward needs only X: it runs while dY is still on its way
+    PEQA_CUDA(cudaStreamWaitEvent(st, hp->x_landed[c], 0));
     PEQA_TRY(peqa_qlinear_fwd(w, dX_in + t0 * K * 2, (int)tc, dY_out + t0 * N * 2, workspace,
                               workspace_bytes, stream));
+    PEQA_CUDA(cudaEventRecord(hp->fwd_done[c], st));
+    PEQA_CUDA(cudaStreamWaitEvent(st, hp->dy_landed[c], 0));
     PEQA_TRY(peqa_qlinear_bwd(w, nullptr, ddY + t0 * N * 2, (int)tc, ddX + t0 * K * 2, nullptr,
                               workspace, workspace_bytes, stream));
-    PEQA_CUDA(cudaEventRecord(hp->computed[c], st));
-    PEQA_CUDA(cudaStreamWaitEvent(hp->out, hp->computed[c], 0));
+    PEQA_CUDA(cudaEventRecord(hp->dx_done[c], st));
+    // Y goes back while dX is still being computed
+    PEQA_CUDA(cudaStreamWaitEvent(hp->out, hp->fwd_done[c], 0));
     PEQA_CUDA(cudaMemcpyAsync(hY + t0 * N * 2, dY_out + t0 * N * 2, tc * N * 2, cudaMemcpyDeviceToHost, hp->out));
+    PEQA_CUDA(cudaStreamWaitEvent(hp->out, hp->dx_done[c], 0));
     PEQA_CUDA(cudaMemcpyAsync(hdX + t0 * K * 2, ddX + t0 * K * 2, tc * K * 2, cudaMemcpyDeviceToHost, hp->out));
   }
   PEQA_CUDA(cudaEventRecord(hp->out_done, hp->out));
