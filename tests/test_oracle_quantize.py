@@ -32,6 +32,29 @@ def test_eq1_worked_examples_exact():
         assert np.array_equal(scales[0, 0] * (codes[0].astype(np.float32) - zeros[0, 0]), W[0])
 
 
+def test_eq1_exact_ties_round_half_to_even():
+    """Rows whose quotients are exactly k + 1/2: the expected codes are literal hand values."""
+    n = 0
+    for line in _rows("eq1_tie_rows.txt"):
+        bits, zero, h, exp = [part.strip() for part in line.split(";")]
+        bits, zero = int(bits), int(zero)
+        h = np.array([float(x) for x in h.split()], dtype=np.float64)
+        exp = np.array([int(x) for x in exp.split()], dtype=np.uint8)
+        W = (h * 2.0 ** -4).astype(np.float32)[None, :]
+        assert np.array_equal(W.astype(np.float64)[0], h * 2.0 ** -4)      # exactly representable
+        codes, zeros, scales = oracle.quantize_rtn(W, bits)
+        assert scales[0, 0] == np.float32(2.0 ** -4)
+        assert zeros[0, 0] == zero
+        assert np.array_equal(codes[0], exp)
+        # the same row as two groups of 16 columns is not defined (groups are multiples of 32);
+        # as one group of a wider row it must give the same codes
+        W2 = np.concatenate([W, W], axis=1)
+        c2, z2, s2 = oracle.quantize_rtn(W2, bits, 32)
+        assert np.array_equal(c2[0, :32], exp) and np.array_equal(c2[0, 32:], exp)
+        n += 1
+    assert n >= 4
+
+
 def _numpy_rtn(W, bits, g):
     """Independent restatement with numpy binary32 array ops (IEEE, ties-to-even rint)."""
     N, K = W.shape
