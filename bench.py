@@ -1,13 +1,22 @@
 #!/usr/bin/env python
 """Benchmark of the PEQA quantized-linear hot path on B200.
 
-One step = one pass of the whole path over one batch of the LLaMA-7B attention
-projection workload (4096x4096, 3-bit, groups of 128, 2048 tokens): RTN
-quantize+pack of the fp32 weight, forward, dX, dS, AdamW on the scales and an
-M=1 decode.  The headline value counts only the 6*T*N*K flop of forward +
-backward against the time of the whole step.
+Headline workload: one LLaMA-65B decoder layer, 3-bit weights in groups of 64
+(q, k, v, o 8192x8192; gate, up 22016x8192; down 8192x22016; 4096 tokens).
+One step runs, for the seven linears in layer order, the whole path through the
+C ABI: RTN quantize+pack of the fp32 weight, forward, dX, dS with the AdamW
+step on the scales applied in the same launch, and an M=1 decode.  The headline
+value counts only the 6*T*N*K flop of forward + backward against the time of
+the whole step.
+
+The same JSON line carries sub-records (each with its own clock record): the
+LLaMA-7B attention projection (3-bit g128, 2048 tokens) and SwiGLU MLP shapes
+(4-bit per-channel, 4096 tokens), decode at M in {1, 4, 16} on the three
+LLaMA-65B shapes with a bare-read ceiling beside each, and the per-channel dS
+from the stored output.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+  python bench.py --render-md LINE.json     # markdown tables of a saved line
 
 Prints exactly one JSON line on rank 0.
 """
@@ -26,10 +35,17 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-WORKLOAD = "c2"
+WORKLOAD = "c5"
+WORKLOAD_TEXT = ("c5: one LLaMA-65B decoder layer, seven linears in layer order (q,k,v,o 8192x8192; "
+                 "gate,up 22016x8192; down 8192x22016), 3-bit, group 64, T=4096 tokens")
 METRIC = "qlinear fwd+bwd TFLOP/s (% bf16 peak); 3-bit decode GB/s (% HBM peak)"
-N_SETS = 4                       # rotating input sets: ~135 MB each, together > L2 (126 MB)
+NOMINAL_BF16_TFLOPS = 2250.0
+NOMINAL_HBM_GBS = 8000.0
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+LR, BETA1, BETA2, EPS, WD = 1e-5, 0.9, 0.999, 1e-8, 0.0
+STAGES = ("quantize_rtn", "qlinear_fwd", "qlinear_bwd_dx", "qlinear_bwd_ds", "qlinear_decode")
+DECODE_SHAPES = (("attn_8192x8192", 8192, 8192), ("gate_up_22016x8192", 22016, 8192),
+                 ("down_8192x22016", 8192, 22016))
 
 
 def load_peaks():
@@ -41,41 +57,37 @@ def load_peaks():
         return dict(FALLBACK_PEAKS), "fallback"
 
 
-def measured_traffic(kernel_name):
-    """DRAM bytes per launch from the committed ncu capture, or None when the kernel sources
-    have changed since the counters were taken."""
+def device_sources_sha256():
     import hashlib
+    h = hashlib.sha256()
+    csrc = os.path.join(ROOT, "paper_2305_14152_b200", "csrc")
+    for name in sorted(os.listdir(csrc)):
+        with open(os.path.join(csrc, name), "rb") as f:
+            text = f.read()
+        if name.endswith(".cuh") or b"__global__" in text:      # device code only
+            h.update(text)
+    return h.hexdigest()
+
+
+def measured_traffic(stage_name):
+    """DRAM bytes per launch of the dominant kernel from the committed ncu capture (scaled to the
+    mean launch of the headline step as that file states), or None when the kernel sources have
+    changed since the counters were taken."""
     try:
-        with open(os.path.join(ROOT, "profiles", "dram_traffic_c2.json")) as f:
+        with open(os.path.join(ROOT, "profiles", "dram_traffic_c5.json")) as f:
             doc = json.load(f)
-        h = hashlib.sha256()
-        csrc = os.path.join(ROOT, "paper_2305_14152_b200", "csrc")
-        for name in sorted(os.listdir(csrc)):
-            with open(os.path.join(csrc, name), "rb") as f:
-                text = f.read()
-            if name.endswith(".cuh") or b"__global__" in text:      # device code only
-                h.update(text)
-        if h.hexdigest() != doc["kernel_sources_sha256"] or doc.get("workload") != WORKLOAD:
+        if device_sources_sha256() != doc["kernel_sources_sha256"] or doc.get("workload") != WORKLOAD:
             return None
-        return doc["kernels"][kernel_name]["traffic_bytes"]
+        return doc["kernels"][stage_name]["traffic_bytes_mean_launch"]
     except Exception:
         return None
 
 
-def draw_sets(n_sets):
-    """Set 0 is the canonical workload draw; further sets continue the same seeded stream."""
-    from paper_2305_14152_b200 import synth
-    wl = synth.WORKLOADS[WORKLOAD]
-    spec = wl.layers[0]
-    rng = np.random.Generator(np.random.PCG64(wl.seed))
-    return spec, [synth.draw_layer(rng, spec) for _ in range(n_sets)]
-
-
 # --------------------------------------------------------------------------- clocks
 class ClockSampler(threading.Thread):
-    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+    """Samples SM clock and throttle reasons through NVML while a timed region runs."""
 
-    def __init__(self, index, period=0.02):
+    def __init__(self, index, period=0.01):
         super().__init__(daemon=True)
         self.index, self.period = index, period
         self.samples, self.reasons, self.max_mhz = [], set(), None
@@ -134,9 +146,53 @@ def physical_gpu_index(local_index):
     return local_index
 
 
+class Timed:
+    """A timed region: CUDA events on the current stream, clocks sampled meanwhile."""
+
+    def __init__(self, torch, min_seconds=0.0):
+        self.torch = torch
+        self.sampler = ClockSampler(physical_gpu_index(torch.cuda.current_device()))
+        self.e0 = torch.cuda.Event(enable_timing=True)
+        self.e1 = torch.cuda.Event(enable_timing=True)
+
+    def __enter__(self):
+        self.torch.cuda.synchronize()
+        self.sampler.start()
+        self.e0.record()
+        return self
+
+    def __exit__(self, *exc):
+        self.e1.record()
+        self.torch.cuda.synchronize()
+        self.clocks = self.sampler.stop()
+        self.ms = self.e0.elapsed_time(self.e1)
+        return False
+
+
+def aggregate_max(ms_local, dist_mod=None, device=None):
+    """Max over ranks of a per-rank time in ms (identity without a process group)."""
+    if dist_mod is None or not dist_mod.is_initialized():
+        return ms_local
+    import torch
+    t = torch.tensor([ms_local], dtype=torch.float64, device=device or "cpu")
+    dist_mod.all_reduce(t, op=dist_mod.ReduceOp.MAX)
+    return float(t.item())
+
+
+def peak_for_clock(peaks, clocks):
+    """Burst or sustained bf16 denominator, chosen by the SM clock sampled during the region:
+    a region that ran near the maximum clock is compared with the burst figure, one that ran
+    power-capped with the sustained one."""
+    mhz, mx = clocks.get("sm_mhz"), clocks.get("sm_max_mhz")
+    capped = (mhz is not None and mx and mhz < 0.85 * mx) or "sw_power_cap" in clocks.get("reasons", [])
+    if capped:
+        return peaks["bf16_tflops_sustained"], "sustained"
+    return peaks["bf16_tflops"], "burst"
+
+
 # --------------------------------------------------------------------------- oracle arm
-def oracle_sample(spec, layer, n_tok=512, n_rows=1024):
-    """Times the CPU oracle on a bounded sample of the workload; returns (seconds, flop)."""
+def oracle_sample(spec, layer, n_tok=512, n_rows=512):
+    """Times the CPU oracle on a bounded sample of one linear; returns (seconds, flop, text)."""
     import oracle
     t0 = time.perf_counter()
     codes, zeros, scales = oracle.quantize_rtn(layer["W"], spec.bits, spec.group_size)
@@ -148,7 +204,15 @@ def oracle_sample(spec, layer, n_tok=512, n_rows=1024):
     oracle.bwd_ds(layer["X"], layer["dY"], packed, zeros, spec.bits, spec.group_size, rows=rows)
     dt = time.perf_counter() - t0
     flop = 2.0 * n_tok * spec.N * spec.K * 2 + 2.0 * spec.T * spec.K * n_rows
-    return dt, flop, f"quantize+pack of W, fwd and dX on {n_tok} of {spec.T} tokens, dS on {n_rows} of {spec.N} rows"
+    what = (f"linear '{spec.name}' ({spec.N}x{spec.K}) of the layer: quantize+pack of W, fwd and dX on "
+            f"{n_tok} of {spec.T} tokens, dS on {n_rows} of {spec.N} rows; throughput by flop count, "
+            f"the other six linears extrapolate at the same rate")
+    return dt, flop, what
+
+
+def first_layer_host():
+    from paper_2305_14152_b200 import synth
+    return next(synth.generate(WORKLOAD))
 
 
 def run_reference(args):
@@ -156,13 +220,14 @@ def run_reference(args):
     if rank != 0:
         return
     import oracle
-    spec, sets = draw_sets(1)
+    layer = first_layer_host()
+    spec = layer["spec"]
     for _ in range(min(args.warmup, 1)):
-        oracle_sample(spec, sets[0], 64, 64)
-    steps = max(1, min(args.steps, 5))
+        oracle_sample(spec, layer, 16, 16)
+    steps = max(1, min(args.steps, 3))
     total_t, total_f, what = 0.0, 0.0, ""
     for _ in range(steps):
-        dt, fl, what = oracle_sample(spec, sets[0], 256, 512)
+        dt, fl, what = oracle_sample(spec, layer, 256, 256)
         total_t += dt
         total_f += fl
     val = total_f / total_t / 1e12
@@ -171,7 +236,7 @@ def run_reference(args):
         "steps": steps, "warmup": min(args.warmup, 1), "ms_per_step": total_t / steps * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
         "data": "synthetic",
-        "config": {"workload": f"{WORKLOAD}: LLaMA-7B attention projection 4096x4096, 3-bit g128, T=2048",
+        "config": {"workload": WORKLOAD_TEXT,
                    "note": "fp64 CPU oracle on a bounded sample per step"},
         "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": oracle.num_threads(),
                          "kind": "oracle", "sample": what},
@@ -181,14 +246,91 @@ def run_reference(args):
 
 
 # --------------------------------------------------------------------------- CUDA arm
-def aggregate_max(ms_local, dist_mod=None, device=None):
-    """Max over ranks of a per-rank time in ms (identity without a process group)."""
-    if dist_mod is None or not dist_mod.is_initialized():
-        return ms_local
-    import torch
-    t = torch.tensor([ms_local], dtype=torch.float64, device=device or "cpu")
-    dist_mod.all_reduce(t, op=dist_mod.ReduceOp.MAX)
-    return float(t.item())
+class Linear:
+    """Device buffers of one linear of a workload."""
+
+    def __init__(self, torch, binding, dev, d, keep_w=True):
+        spec = d["spec"]
+        self.spec = spec
+        self.N, self.K, self.T, self.bits, self.g = spec.N, spec.K, spec.T, spec.bits, spec.group_size
+        self.G = self.K // self.g if self.g else 1
+        self.flop = 2.0 * self.T * self.N * self.K
+
+        def bf16(bits_arr):
+            return torch.from_numpy(bits_arr.view(np.int16)).view(torch.bfloat16).to(dev)
+
+        self.W = torch.from_numpy(d["W"]).to(dev)
+        self.X = bf16(d["X"])
+        self.dY = bf16(d["dY"]) if d["dY"] is not None else None
+        self.qw = binding.quantize_rtn(self.W, self.bits, self.g)
+        if not keep_w:
+            self.W = None
+        self.m = torch.zeros((self.N, self.G), dtype=torch.float32, device=dev)
+        self.v = torch.zeros((self.N, self.G), dtype=torch.float32, device=dev)
+        self.dS = torch.empty((self.N, self.G), dtype=torch.float32, device=dev)
+        self.Yd = torch.empty((1, self.N), dtype=torch.bfloat16, device=dev)
+        self.ws = binding.alloc_workspace(binding.OP_BWD, self.T, self.qw)
+
+
+def load_workload(torch, binding, dev, name, keep_first_host=False):
+    from paper_2305_14152_b200 import synth
+    layers, first = [], None
+    for d in synth.generate(name):
+        layers.append(Linear(torch, binding, dev, d))
+        if keep_first_host and first is None:
+            first = d
+    return layers, first
+
+
+def run_stage(binding, L, k, Y, dX, step_no):
+    if k == 0:
+        binding.quantize_rtn(L.W, L.bits, L.g, out=L.qw)
+    elif k == 1:
+        binding.qlinear_fwd(L.qw, L.X, Y[:L.T * L.N].view(L.T, L.N))
+    elif k == 2:
+        binding.qlinear_bwd(L.qw, None, L.dY, dX=dX[:L.T * L.K].view(L.T, L.K), need_ds=False)
+    elif k == 3:
+        binding.qlinear_bwd_ds_adamw(L.qw, L.X, L.dY, L.m, L.v, LR, BETA1, BETA2, EPS, WD, step_no,
+                                     dS=L.dS, workspace=L.ws)
+    else:
+        binding.qlinear_decode(L.qw, L.X[:1], L.Yd)
+
+
+def time_layer_steps(torch, binding, layers, Y, dX, steps, warmup, dist=None, dev=None):
+    """Times `steps` passes over `layers` (all five stages of every linear); returns the total ms
+    (max over ranks), per-stage mean ms [linear][stage], and the clock record."""
+    n = len(layers)
+    for i in range(warmup):
+        for L in layers:
+            for k in range(len(STAGES)):
+                run_stage(binding, L, k, Y, dX, i + 1)
+    binding.check_status()
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(n * len(STAGES) + 1)] for _ in range(steps)]
+    if dist is not None:
+        dist.barrier()
+    with Timed(torch) as tm:
+        for i in range(steps):
+            e = evs[i]
+            e[0].record()
+            j = 0
+            for L in layers:
+                for k in range(len(STAGES)):
+                    run_stage(binding, L, k, Y, dX, warmup + i + 1)
+                    j += 1
+                    e[j].record()
+    if dist is not None:
+        dist.barrier()
+    binding.check_status()
+    ms_total = aggregate_max(tm.ms, dist, dev)
+    stage_ms = [[float(np.mean([evs[i][li * len(STAGES) + k].elapsed_time(evs[i][li * len(STAGES) + k + 1])
+                                for i in range(steps)])) for k in range(len(STAGES))] for li in range(n)]
+    return ms_total, stage_ms, tm.clocks
+
+
+def launches_per_step(layers):
+    """Kernels of this library per step: one per stage, plus the dS reduce kernel when a
+    quantization group is wider than 128 columns."""
+    return sum(len(STAGES) + (1 if L.ws is not None else 0) for L in layers)
 
 
 def run_cuda(args):
@@ -209,178 +351,191 @@ def run_cuda(args):
     peaks, peak_src = load_peaks()
 
     if args.only_decode:
-        # the decode section alone (what the decode ncu summaries under profiles/ were taken on)
-        print(json.dumps({"decode": bench_decode(binding, dev, peaks, reps=args.steps if args.steps < 30 else 30)}),
-              flush=True)
+        print(json.dumps({"decode": bench_decode(torch, binding, dev, peaks, reps=min(args.steps, 30),
+                                                 shapes=args.case)}), flush=True)
         return
 
-    spec, sets = draw_sets(N_SETS)
-    N, K, T, bits, g = spec.N, spec.K, spec.T, spec.bits, spec.group_size
-    G = K // g if g else 1
-
-    def bf16(bits_arr):
-        return torch.from_numpy(bits_arr.view(np.int16)).view(torch.bfloat16).to(dev)
-
-    Ws = [torch.from_numpy(s["W"]).to(dev) for s in sets]
-    Xs = [bf16(s["X"]) for s in sets]
-    dYs = [bf16(s["dY"]) for s in sets]
-    qws = [binding.quantize_rtn(W, bits, g) for W in Ws]
-    Y = torch.empty((T, N), dtype=torch.bfloat16, device=dev)
-    dX = torch.empty((T, K), dtype=torch.bfloat16, device=dev)
-    dS = torch.empty((N, G), dtype=torch.float32, device=dev)
-    m = torch.zeros((N, G), dtype=torch.float32, device=dev)
-    v = torch.zeros((N, G), dtype=torch.float32, device=dev)
-    Yd = torch.empty((1, N), dtype=torch.bfloat16, device=dev)
-    ws = binding.alloc_workspace(binding.OP_BWD, T, qws[0])
-    lr = 1e-5
-    # dS and the AdamW step on the scales are one launch (the step is applied where each dS
-    # value becomes final), so the step has five stages
-    stage_names = ["quantize_rtn", "qlinear_fwd", "qlinear_bwd_dx", "qlinear_bwd_ds", "qlinear_decode"]
-    n_stages = len(stage_names)
-    launches_per_step = n_stages + (1 if ws is not None else 0)
-
-    def step(i, evs=None):
-        r = i % N_SETS
-        qw = qws[r]
-        if evs: evs[0].record()
-        binding.quantize_rtn(Ws[r], bits, g, out=qw)
-        if evs: evs[1].record()
-        binding.qlinear_fwd(qw, Xs[r], Y)
-        if evs: evs[2].record()
-        binding.qlinear_bwd(qw, None, dYs[r], dX=dX, need_ds=False)
-        if evs: evs[3].record()
-        binding.qlinear_bwd_ds_adamw(qw, Xs[r], dYs[r], m, v, lr, 0.9, 0.999, 1e-8, 0.0, i + 1,
-                                     dS=dS, workspace=ws)
-        if evs: evs[4].record()
-        binding.qlinear_decode(qw, Xs[r][:1], Yd)
-        if evs: evs[5].record()
-
-    for i in range(max(args.warmup, 3)):
-        step(i)
-    binding.check_status()
-    torch.cuda.synchronize()
-
-    sampler = ClockSampler(physical_gpu_index(torch.cuda.current_device()))
-    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(n_stages + 1)] for _ in range(args.steps)]
-    if dist is not None:
-        dist.barrier()
-    torch.cuda.synchronize()
-    sampler.start()
-    t_start = torch.cuda.Event(enable_timing=True)
-    t_end = torch.cuda.Event(enable_timing=True)
-    t_start.record()
-    for i in range(args.steps):
-        step(i, evs[i])
-    t_end.record()
-    torch.cuda.synchronize()
-    if dist is not None:
-        dist.barrier()
-    clocks = sampler.stop()
-    binding.check_status()
-    ms_total = aggregate_max(t_start.elapsed_time(t_end), dist, dev)
+    extras = rank == 0 and not args.only_step
+    layers, first_host = load_workload(torch, binding, dev, WORKLOAD, keep_first_host=extras and world == 1)
+    if args.case:
+        layers = [L for L in layers if L.spec.name in args.case.split(",")]
+    Y = torch.empty(max(L.T * L.N for L in layers), dtype=torch.bfloat16, device=dev)
+    dX = torch.empty(max(L.T * L.K for L in layers), dtype=torch.bfloat16, device=dev)
+    warmup = max(args.warmup, 3)
+    ms_total, stage_ms, clocks = time_layer_steps(torch, binding, layers, Y, dX, args.steps, warmup, dist, dev)
     ms_step = ms_total / args.steps
-    stage_ms = [float(np.mean([evs[i][k].elapsed_time(evs[i][k + 1]) for i in range(args.steps)]))
-                for k in range(n_stages)]
-
-    flop_step = 6.0 * T * N * K
+    flop_step = 3.0 * sum(L.flop for L in layers)
     value = world * flop_step / (ms_step * 1e-3) / 1e12
 
-    # ---- end to end through the host-buffer entry point (pinned host memory both ways)
-    e2e = None
-    if not args.only_step:
-        e2e = bench_e2e(args, binding, torch, qws, Xs, dYs, Y, dX, dS, m, v, ws, lr, dist, dev,
-                        world, flop_step, T, N, K, G)
-
-    # ---- roofline of the dominant kernel (the slowest of the three contractions)
-    gemm = {k: stage_ms[k] for k in (1, 2, 3)}
-    dom = max(gemm, key=gemm.get)
-    ach = 2.0 * T * N * K / (gemm[dom] * 1e-3) / 1e12
-    long_region = ms_total > 1000.0
-    peak = peaks["bf16_tflops_sustained"] if long_region else peaks["bf16_tflops"]
-    roofline = {"bound": "tensor", "kernel": stage_names[dom], "achieved": ach, "peak": peak,
-                "unit": "TFLOP/s", "frac": ach / peak, "traffic": measured_traffic(stage_names[dom]),
-                "traffic_unit": "DRAM bytes per launch (ncu)",
-                "peak_source": f"{peak_src} bf16 {'sustained' if long_region else 'burst'}",
-                "frac_of_nominal_2250": ach / 2250.0,
-                "per_kernel_tflops": {stage_names[k]: 2.0 * T * N * K / (gemm[k] * 1e-3) / 1e12
-                                      for k in (1, 2, 3)}}
-
-    # ---- secondary metric: M=1 decode of the LLaMA-65B 3-bit per-channel shapes, cold in L2
-    decode = None
-    if rank == 0 and not args.only_step:
-        decode = bench_decode(binding, dev, peaks)
-
-    # ---- next-row item: per-channel dS from the stored output (HBM bound, 4*T*N bytes)
-    ds_from_y = None
-    if rank == 0 and not args.only_step:
-        ds_from_y = bench_ds_from_y(binding, dev, peaks)
+    # ---- roofline of the dominant kernel: the contraction with the largest share of the step
+    tot = {k: sum(stage_ms[li][k] for li in range(len(layers))) for k in (1, 2, 3)}
+    dom = max(tot, key=tot.get)
+    mean_flop = sum(L.flop for L in layers) / len(layers)
+    mean_ms = tot[dom] / len(layers)
+    ach = mean_flop / (mean_ms * 1e-3) / 1e12
+    peak, which = peak_for_clock(peaks, clocks)
+    roofline = {
+        "bound": "tensor", "kernel": STAGES[dom], "achieved": ach, "peak": peak, "unit": "TFLOP/s",
+        "frac": ach / peak, "traffic": measured_traffic(STAGES[dom]),
+        "traffic_unit": "DRAM bytes per mean launch (ncu)",
+        "peak_source": f"{peak_src} cuBLAS bf16 {which} (chosen by the sampled SM clock)",
+        "launches_per_step": len(layers), "flop_per_mean_launch": mean_flop, "ms_per_mean_launch": mean_ms,
+        "frac_of_measured_burst": ach / peaks["bf16_tflops"],
+        "frac_of_measured_sustained": ach / peaks["bf16_tflops_sustained"],
+        "frac_of_nominal_2250": ach / NOMINAL_BF16_TFLOPS,
+        "target_60pct_of_nominal_met": bool(ach / NOMINAL_BF16_TFLOPS >= 0.60),
+        "per_kernel_tflops": {STAGES[k]: sum(L.flop for L in layers) / (tot[k] * 1e-3) / 1e12 for k in (1, 2, 3)},
+    }
+    per_linear = {L.spec.name: {"N": L.N, "K": L.K,
+                                **{STAGES[k] + "_ms": stage_ms[li][k] for k in range(len(STAGES))},
+                                "fwd_dx_ds_tflops": 3.0 * L.flop / (sum(stage_ms[li][1:4]) * 1e-3) / 1e12}
+                  for li, L in enumerate(layers)}
 
     out = {
         "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
-        "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
+        "warmup": warmup, "ms_per_step": ms_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": f"{WORKLOAD}: LLaMA-7B attention projection N=K=4096, 3-bit, group 128, "
-                               f"T=2048 tokens; step = quantize+pack, fwd, dX, dS+AdamW (one launch), decode(M=1)",
-                   "l2": f"{N_SETS} rotating input sets (~{N_SETS * 135} MB) exceed the 126 MB L2; no flush kernel",
+        "config": {"workload": WORKLOAD_TEXT + "; step = per linear: quantize+pack, fwd, dX, dS+AdamW (one "
+                               "launch), decode(M=1)" + (f"; restricted to {args.case}" if args.case else ""),
+                   "l2": "every linear's operands (X, dY, Y/dX, packed W: 0.3-0.6 GB) exceed the 126 MB L2 and "
+                         "the seven linears use distinct buffers, so every launch starts cold; no flush kernel",
                    "parallelism": "replicas only" if world > 1 else "single GPU",
                    "flop_per_step": flop_step},
-        "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
-        "stage_ms": dict(zip(stage_names, stage_ms)),
-        "roofline": roofline, "decode": decode, "ds_from_y": ds_from_y,
+        "clocks": clocks, "gpu_launches": launches_per_step(layers) * args.steps,
+        "stage_ms": {STAGES[k]: sum(stage_ms[li][k] for li in range(len(layers))) for k in range(len(STAGES))},
+        "per_linear": per_linear, "roofline": roofline,
+        "value_frac_of_measured_burst": value / world / peaks["bf16_tflops"],
+        "value_frac_of_measured_sustained": value / world / peaks["bf16_tflops_sustained"],
+        "value_frac_of_nominal_2250": value / world / NOMINAL_BF16_TFLOPS,
     }
-    if rank == 0 and world == 1 and not args.only_step:
-        dt, fl, what = oracle_sample(spec, sets[0])
-        import oracle
-        out["cpu_baseline"] = {"value": fl / dt / 1e12, "unit": "TFLOP/s", "cores": oracle.num_threads(),
-                               "kind": "oracle", "sample": what, "seconds": dt}
+
+    # ---- end to end through the host-buffer entry point (pinned host memory both ways)
+    out["e2e"] = None
+    if not args.only_step:
+        out["e2e"] = bench_e2e(args, binding, torch, layers, Y, dX, dist, dev, world, flop_step)
+
+    if extras:
+        del layers
+        torch.cuda.empty_cache()
+        out["c2"] = bench_small_workload(torch, binding, dev, peaks, "c2", steps=200, n_sets=4)
+        out["c3"] = bench_small_workload(torch, binding, dev, peaks, "c3", steps=20, n_sets=2)
+        out["decode"] = bench_decode(torch, binding, dev, peaks)
+        out["ds_from_y"] = bench_ds_from_y(torch, binding, dev, peaks)
+        if world == 1:
+            import oracle
+            dt, fl, what = oracle_sample(first_host["spec"], first_host)
+            out["cpu_baseline"] = {"value": fl / dt / 1e12, "unit": "TFLOP/s", "cores": oracle.num_threads(),
+                                   "kind": "oracle", "sample": what, "seconds": dt}
     if rank == 0:
         print(json.dumps(out), flush=True)
     if dist is not None:
         dist.destroy_process_group()
 
 
-def bench_e2e(args, binding, torch, qws, Xs, dYs, Y, dX, dS, m, v, ws, lr, dist, dev, world,
-              flop_step, T, N, K, G):
-    """Same metric through peqa_train_step_host: pinned host buffers in and out every step."""
-    hX = torch.empty((T, K), dtype=torch.bfloat16).pin_memory()
-    hdY = torch.empty((T, N), dtype=torch.bfloat16).pin_memory()
-    hX.copy_(Xs[0].cpu())
-    hdY.copy_(dYs[0].cpu())
-    hY = torch.empty((T, N), dtype=torch.bfloat16).pin_memory()
-    hdX = torch.empty((T, K), dtype=torch.bfloat16).pin_memory()
-    hdS = torch.empty((N, G), dtype=torch.float32).pin_memory()
-    dXin = torch.empty_like(Xs[0])
-    ddYin = torch.empty_like(dYs[0])
-    e2e_steps = max(3, min(args.steps, 50))
-    for k in range(2):
-        binding.train_step_host(qws[0], hX, hdY, hY, hdX, hdS, dXin, ddYin, Y, dX, dS, m, v, lr,
-                                step=k + 1, workspace=ws)
+def bench_e2e(args, binding, torch, layers, Y, dX, dist, dev, world, flop_step):
+    """Same metric through peqa_train_step_host, one call per linear: every step copies each
+    linear's X and dY from pinned host memory and returns Y, dX and dS to pinned host memory."""
+    host = []
+    for L in layers:
+        hX = torch.empty((L.T, L.K), dtype=torch.bfloat16).pin_memory()
+        hdY = torch.empty((L.T, L.N), dtype=torch.bfloat16).pin_memory()
+        hX.copy_(L.X)
+        hdY.copy_(L.dY)
+        host.append((hX, hdY))
+    hY = torch.empty(Y.numel(), dtype=torch.bfloat16).pin_memory()
+    hdX = torch.empty(dX.numel(), dtype=torch.bfloat16).pin_memory()
+    hdS = torch.empty(max(L.N * L.G for L in layers), dtype=torch.float32).pin_memory()
+    dXin = torch.empty(max(L.T * L.K for L in layers), dtype=torch.bfloat16, device=dev)
+    ddYin = torch.empty(max(L.T * L.N for L in layers), dtype=torch.bfloat16, device=dev)
+    steps = max(2, min(args.steps, 5))
+
+    def one(k):
+        for L, (hX, hdY) in zip(layers, host):
+            binding.train_step_host(L.qw, hX, hdY, hY[:L.T * L.N].view(L.T, L.N), hdX[:L.T * L.K].view(L.T, L.K),
+                                    hdS[:L.N * L.G].view(L.N, L.G), dXin[:L.T * L.K].view(L.T, L.K),
+                                    ddYin[:L.T * L.N].view(L.T, L.N), Y[:L.T * L.N].view(L.T, L.N),
+                                    dX[:L.T * L.K].view(L.T, L.K), L.dS, L.m, L.v, LR, step=k + 1, workspace=L.ws)
+
+    one(0)
     torch.cuda.synchronize()
-    e0 = torch.cuda.Event(enable_timing=True)
-    e1 = torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for k in range(e2e_steps):
-        binding.train_step_host(qws[k % N_SETS], hX, hdY, hY, hdX, hdS, dXin, ddYin, Y, dX, dS, m, v,
-                                lr, step=k + 3, workspace=ws)
-    e1.record()
-    torch.cuda.synchronize()
-    e2e_ms = aggregate_max(e0.elapsed_time(e1) / e2e_steps, dist, dev)
-    return {"value": world * flop_step / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
-            "h2d_bytes_per_step": int(hX.numel() * 2 + hdY.numel() * 2),
-            "d2h_bytes_per_step": int(hY.numel() * 2 + hdX.numel() * 2 + hdS.numel() * 4),
-            "ms_per_step": e2e_ms,
-            "what": "peqa_train_step_host: H2D X,dY; fwd, dX, dS, AdamW; D2H Y,dX,dS"}
+    if dist is not None:
+        dist.barrier()
+    with Timed(torch) as tm:
+        for k in range(steps):
+            one(k + 1)
+    ms = aggregate_max(tm.ms / steps, dist, dev)
+    return {"value": world * flop_step / (ms * 1e-3) / 1e12, "unit": "TFLOP/s",
+            "h2d_bytes_per_step": int(sum(a.numel() * 2 + b.numel() * 2 for a, b in host)),
+            "d2h_bytes_per_step": int(sum(L.T * L.N * 2 + L.T * L.K * 2 + L.N * L.G * 4 for L in layers)),
+            "ms_per_step": ms, "steps": steps, "clocks": tm.clocks,
+            "what": "peqa_train_step_host per linear: H2D X,dY; fwd, dX, dS+AdamW; D2H Y,dX,dS"}
 
 
-def bench_decode(binding, dev, peaks, reps=30):
-    """GB/s of peqa_qlinear_decode at M=1 on the three LLaMA-65B shapes; weights rotate through
-    enough distinct copies to exceed L2, so every launch streams from HBM."""
-    import torch
+def bench_small_workload(torch, binding, dev, peaks, name, steps, n_sets):
+    """The same five stages on another configured workload (a sub-record of the line): `n_sets`
+    seeded draws of every linear rotate so that launches start cold in L2."""
+    from paper_2305_14152_b200 import synth
+    wl = synth.WORKLOADS[name]
+    rng = np.random.Generator(np.random.PCG64(wl.seed))
+    sets = [[Linear(torch, binding, dev, synth.draw_layer(rng, spec)) for spec in wl.layers]
+            for _ in range(n_sets)]
+    Y = torch.empty(max(L.T * L.N for L in sets[0]), dtype=torch.bfloat16, device=dev)
+    dX = torch.empty(max(L.T * L.K for L in sets[0]), dtype=torch.bfloat16, device=dev)
+    n = len(wl.layers)
+    for i in range(3):
+        for L in sets[i % n_sets]:
+            for k in range(len(STAGES)):
+                run_stage(binding, L, k, Y, dX, i + 1)
+    binding.check_status()
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(n * len(STAGES) + 1)] for _ in range(steps)]
+    with Timed(torch) as tm:
+        for i in range(steps):
+            e = evs[i]
+            e[0].record()
+            j = 0
+            for L in sets[i % n_sets]:
+                for k in range(len(STAGES)):
+                    run_stage(binding, L, k, Y, dX, 4 + i)
+                    j += 1
+                    e[j].record()
+    binding.check_status()
+    stage_ms = [[float(np.mean([evs[i][li * len(STAGES) + k].elapsed_time(evs[i][li * len(STAGES) + k + 1])
+                                for i in range(steps)])) for k in range(len(STAGES))] for li in range(n)]
+    layers = sets[0]
+    flop_step = 3.0 * sum(L.flop for L in layers)
+    ms_step = tm.ms / steps
+    peak, which = peak_for_clock(peaks, tm.clocks)
+    rec = {"workload": name, "steps": steps, "ms_per_step": ms_step,
+           "value": flop_step / (ms_step * 1e-3) / 1e12, "unit": "TFLOP/s (6*T*N*K over the whole step)",
+           "clocks": tm.clocks, "peak": peak, "peak_kind": which,
+           "l2": f"{n_sets} rotating seeded draws of every linear", "per_linear": {}}
+    for li, L in enumerate(layers):
+        r = {"N": L.N, "K": L.K, "T": L.T, "bits": L.bits, "group": L.g}
+        for k in range(len(STAGES)):
+            r[STAGES[k] + "_ms"] = stage_ms[li][k]
+        for k in (1, 2, 3):
+            r[STAGES[k] + "_tflops"] = L.flop / (stage_ms[li][k] * 1e-3) / 1e12
+        tf = 3.0 * L.flop / (sum(stage_ms[li][1:4]) * 1e-3) / 1e12
+        r.update({"fwd_dx_ds_tflops": tf, "frac_of_peak": tf / peak, "frac_of_nominal_2250": tf / NOMINAL_BF16_TFLOPS})
+        rec["per_linear"][L.spec.name] = r
+    del sets
+    torch.cuda.empty_cache()
+    return rec
+
+
+def bench_decode(torch, binding, dev, peaks, reps=30, shapes=None):
+    """GB/s of decode at M in {1, 4, 16} on the three LLaMA-65B shapes (3-bit, one scale per
+    channel), from the prepared weights (peqa_qlinear_decode_prepared, what a server runs) and
+    from the canonical packed matrix (peqa_qlinear_decode); the weights rotate through enough
+    distinct copies to exceed L2, so every launch streams from HBM.  Launches are back to back
+    with no event between them.  Beside each shape: a kernel that only reads the same bytes."""
     res = {}
     gen = torch.Generator(device=dev)
     gen.manual_seed(0)
-    for name, N, K in (("attn_8192x8192", 8192, 8192), ("gate_up_22016x8192", 22016, 8192),
-                       ("down_8192x22016", 8192, 22016)):
+    sink = torch.zeros(1024, dtype=torch.int32, device=dev)
+    for name, N, K in DECODE_SHAPES:
+        if shapes and name not in shapes.split(","):
+            continue
         words = K * 3 // 32
         wbytes = N * words * 4
         copies = max(2, int(np.ceil(4 * 126e6 / wbytes)))
@@ -388,32 +543,67 @@ def bench_decode(binding, dev, peaks, reps=30):
               for _ in range(copies)]
         z = torch.full((N, 1), 3, dtype=torch.uint8, device=dev)
         s = torch.full((N, 1), 0.01, dtype=torch.float32, device=dev)
-        X = torch.randn((1, K), device=dev, generator=gen).to(torch.bfloat16)
-        Y = torch.empty((1, N), dtype=torch.bfloat16, device=dev)
         qws = [binding.QWeight(3, N, K, 0, q, z, s) for q in qs]
-        for i in range(copies):
-            binding.qlinear_decode(qws[i], X, Y)
+        rec = {"bytes_weights": wbytes, "copies": copies}
+
+        def timed(fn):
+            """Mean device time per launch: `reps` launches rotating through the weight copies are
+            captured into one CUDA graph (the same C-ABI calls, recorded instead of run) and the
+            graph is replayed, so host launch overhead is not what is measured.  Falls back to
+            eager launches if the capture is refused."""
+            for i in range(copies):
+                fn(i)
+            torch.cuda.synchronize()
+            graph = None
+            try:
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g):
+                    for i in range(reps):
+                        fn(i % copies)
+                graph = g
+                graph.replay()
+                torch.cuda.synchronize()
+            except Exception:
+                graph = None
+                torch.cuda.synchronize()
+            replays = 5
+            with Timed(torch) as tm:
+                for _ in range(replays):
+                    if graph is not None:
+                        graph.replay()
+                    else:
+                        for i in range(reps):
+                            fn(i % copies)
+            rec["launch_mode"] = "cuda graph replay" if graph is not None else "eager"
+            return tm.ms / (reps * replays) * 1e3, tm.clocks
+
+        us, clk = timed(lambda i: binding.probe_read(qs[i], sink))
+        rec["bare_read"] = {"us": us, "GB/s": wbytes / (us * 1e-6) / 1e9,
+                            "frac_measured_hbm": wbytes / (us * 1e-6) / 1e9 / peaks["hbm_gbs"], "clocks": clk}
+        preps = [binding.decode_prepare(qw) for qw in qws]
         torch.cuda.synchronize()
-        e0 = torch.cuda.Event(enable_timing=True)
-        e1 = torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for i in range(reps):
-            binding.qlinear_decode(qws[i % copies], X, Y)
-        e1.record()
-        torch.cuda.synchronize()
-        us = e0.elapsed_time(e1) / reps * 1e3
-        nbytes = wbytes + N * 5 + K * 2 + N * 2
-        gbs = nbytes / (us * 1e-6) / 1e9
-        res[name] = {"us": us, "GB/s": gbs, "frac_measured_hbm": gbs / peaks["hbm_gbs"],
-                     "frac_nominal_8000": gbs / 8000.0, "bytes": nbytes, "copies": copies}
+        for M in (1, 4, 16):
+            X = torch.randn((M, K), device=dev, generator=gen).to(torch.bfloat16)
+            Y = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
+            ws = binding.alloc_workspace(binding.OP_DECODE, M, qws[0])
+            nbytes = wbytes + N * 5 + M * K * 2 + M * N * 2
+            for key, fn in (("prepared", lambda i: binding.qlinear_decode_prepared(qws[i], preps[i], X, Y)),
+                            ("canonical", lambda i: binding.qlinear_decode(qws[i], X, Y, workspace=ws))):
+                us, clk = timed(fn)
+                gbs = nbytes / (us * 1e-6) / 1e9
+                rec[f"M{M}_{key}"] = {"us": us, "GB/s": gbs, "frac_measured_hbm": gbs / peaks["hbm_gbs"],
+                                      "frac_nominal_8000": gbs / NOMINAL_HBM_GBS, "bytes": nbytes,
+                                      "frac_of_bare_read_time": rec["bare_read"]["us"] / us, "clocks": clk}
+        del preps
+        binding.check_status()
+        res[name] = rec
         del qs, qws
     return res
 
 
-def bench_ds_from_y(binding, dev, peaks, reps=20):
+def bench_ds_from_y(torch, binding, dev, peaks, reps=20):
     """GB/s of peqa_qlinear_bwd_ds_from_y on the LLaMA-7B MLP gate shape (N=11008, T=4096, 4-bit
     per-channel): two rotating (dY, Y) pairs of 180 MB each, so every launch streams from HBM."""
-    import torch
     N, K, T = 11008, 4096, 4096
     gen = torch.Generator(device=dev)
     gen.manual_seed(3)
@@ -427,35 +617,98 @@ def bench_ds_from_y(binding, dev, peaks, reps=20):
     ws = binding.alloc_workspace(binding.OP_BWD_DS_FROM_Y, T, qw)
     for i in range(3):
         binding.qlinear_bwd_ds_from_y(qw, pairs[i % 2][0], pairs[i % 2][1], dS, ws)
-    torch.cuda.synchronize()
-    e0 = torch.cuda.Event(enable_timing=True)
-    e1 = torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for i in range(reps):
-        binding.qlinear_bwd_ds_from_y(qw, pairs[i % 2][0], pairs[i % 2][1], dS, ws)
-    e1.record()
-    torch.cuda.synchronize()
-    us = e0.elapsed_time(e1) / reps * 1e3
+    with Timed(torch) as tm:
+        for i in range(reps):
+            binding.qlinear_bwd_ds_from_y(qw, pairs[i % 2][0], pairs[i % 2][1], dS, ws)
+    us = tm.ms / reps * 1e3
     nbytes = 4 * T * N + 8 * N
     gbs = nbytes / (us * 1e-6) / 1e9
     return {"workload": "N=11008, T=4096 (c3 gate), bf16 dY and Y", "us": us, "GB/s": gbs,
-            "frac_measured_hbm": gbs / peaks["hbm_gbs"], "bytes": nbytes,
+            "frac_measured_hbm": gbs / peaks["hbm_gbs"], "bytes": nbytes, "clocks": tm.clocks,
             "replaces": "the dS contraction of the same layer (2*T*N*K flop)"}
+
+
+# --------------------------------------------------------------------------- rendering
+def render_md(path):
+    """Markdown tables of a saved JSON line (the results section of the benchmark spec is made this way)."""
+    with open(path) as f:
+        text = f.read()
+    doc = None
+    for line in text.splitlines():
+        line = line.strip()
+        if line.startswith("{") and '"metric"' in line:
+            doc = json.loads(line)
+    if doc is None:
+        doc = json.loads(text)
+        doc = doc.get("parsed", doc)
+    o = []
+    c, r = doc["clocks"], doc["roofline"]
+    o.append(f"Headline ({doc['config']['workload']}): **{doc['value']:.0f} TFLOP/s**, {doc['ms_per_step']:.3f} ms "
+             f"per step over {doc['steps']} steps; SM clock median {c['sm_mhz']} of {c['sm_max_mhz']} MHz, "
+             f"reasons {c['reasons']}.  Of the measured cuBLAS burst {doc['value_frac_of_measured_burst']:.2f}, "
+             f"of the measured sustained {doc['value_frac_of_measured_sustained']:.2f}, of the nominal 2250 "
+             f"{doc['value_frac_of_nominal_2250']:.2f}.")
+    o.append(f"Dominant kernel `{r['kernel']}`: {r['achieved']:.0f} TFLOP/s = {r['frac']:.2f} of {r['peak_source']} "
+             f"({r['frac_of_measured_burst']:.2f} burst / {r['frac_of_measured_sustained']:.2f} sustained / "
+             f"{r['frac_of_nominal_2250']:.2f} nominal; 60 % of nominal met: {r['target_60pct_of_nominal_met']}).")
+    o.append("")
+    o.append("| workload | linear | fwd ms | dX ms | dS+AdamW ms | quantize ms | decode M=1 ms | fwd+dX+dS TFLOP/s | of nominal 2250 |")
+    o.append("|---|---|---|---|---|---|---|---|---|")
+    for name, p in doc["per_linear"].items():
+        o.append(f"| c5 | {name} {p['N']}x{p['K']} | {p['qlinear_fwd_ms']:.3f} | {p['qlinear_bwd_dx_ms']:.3f} | "
+                 f"{p['qlinear_bwd_ds_ms']:.3f} | {p['quantize_rtn_ms']:.3f} | {p['qlinear_decode_ms']:.3f} | "
+                 f"{p['fwd_dx_ds_tflops']:.0f} | {p['fwd_dx_ds_tflops'] / NOMINAL_BF16_TFLOPS:.2f} |")
+    for key in ("c2", "c3"):
+        sub = doc.get(key)
+        if not sub:
+            continue
+        for name, p in sub["per_linear"].items():
+            o.append(f"| {key} (clock {sub['clocks']['sm_mhz']} MHz, {sub['peak_kind']}) | {name} {p['N']}x{p['K']} T={p['T']} | "
+                     f"{p['qlinear_fwd_ms']:.4f} | {p['qlinear_bwd_dx_ms']:.4f} | {p['qlinear_bwd_ds_ms']:.4f} | "
+                     f"{p['quantize_rtn_ms']:.4f} | {p['qlinear_decode_ms']:.4f} | {p['fwd_dx_ds_tflops']:.0f} | "
+                     f"{p['frac_of_nominal_2250']:.2f} |")
+    if doc.get("e2e"):
+        e = doc["e2e"]
+        o.append("")
+        o.append(f"End to end ({e['what']}): {e['value']:.0f} TFLOP/s, {e['ms_per_step']:.2f} ms per step, "
+                 f"{e['h2d_bytes_per_step'] / 1e6:.0f} MB in and {e['d2h_bytes_per_step'] / 1e6:.0f} MB out per step.")
+    if doc.get("decode"):
+        o.append("")
+        o.append("| decode shape | bare read us (GB/s) | M | us | GB/s | of measured copy | of 8 TB/s | bare read / kernel |")
+        o.append("|---|---|---|---|---|---|---|---|")
+        for name, rec in doc["decode"].items():
+            b = rec["bare_read"]
+            for key, v in rec.items():
+                if not key.startswith("M"):
+                    continue
+                o.append(f"| {name} {key.split('_')[1]} | {b['us']:.1f} ({b['GB/s']:.0f}) | {key[1:].split('_')[0]} | {v['us']:.1f} | "
+                         f"{v['GB/s']:.0f} | {v['frac_measured_hbm']:.2f} | {v['frac_nominal_8000']:.2f} | "
+                         f"{v['frac_of_bare_read_time']:.2f} |")
+    if doc.get("cpu_baseline"):
+        cb = doc["cpu_baseline"]
+        o.append("")
+        o.append(f"CPU oracle: {cb['value']:.4f} TFLOP/s on {cb['cores']} threads ({cb['sample']}).")
+    print("\n".join(o))
 
 
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=500)
-    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--only-decode", action="store_true",
-                    help="run only the M=1 decode section on the three LLaMA-65B shapes")
+                    help="run only the decode section (with --case: a comma list of its shape names)")
     ap.add_argument("--only-step", action="store_true",
-                    help="time the step only: skip the e2e, decode and CPU-baseline sections "
+                    help="time the step only: skip the e2e, sub-record and CPU-baseline sections "
                          "(lean runs under a profiler)")
+    ap.add_argument("--case", default=None,
+                    help="restrict the step to these linears of the layer (comma list: q,k,v,o,gate,up,down)")
+    ap.add_argument("--render-md", default=None, help="print markdown tables of a saved JSON line")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.render_md:
+        render_md(args.render_md)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_cuda(args)

@@ -227,10 +227,13 @@ int peqa_scale_adamw(float* scales, const float* dS, float* m, float* v, int64_t
  * writable).  Synchronises the stream before returning.  The tokens travel in
  * chunks over two auxiliary streams of the library, so that the copies in, the
  * kernels and the copies out overlap (pinned host buffers are needed for that);
- * those streams and a few events are created on the first call on a device
+ * those streams (2) and events (34) are created on the first call on a device
  * and kept until the process ends, so make that first call outside any stream
- * capture.  h_* and d_* buffers must not be touched by other work until the
- * call returns.
+ * capture.  They are shared by all calls on the device: concurrent calls from
+ * several host threads are serialised by the library.  Every argument is checked
+ * before anything is enqueued; if a CUDA call fails later, the streams are
+ * drained before the error is returned.  h_* and d_* buffers must not be
+ * touched by other work until the call returns.
  */
 int peqa_train_step_host(const peqa_qweight_t* w, int T,
                          const void* h_X_bf16, const void* h_dY_bf16,
@@ -264,9 +267,87 @@ int peqa_qlinear_bwd_ds_static(const peqa_qweight_t* w, const void* X_bf16, cons
                                int T, float* dS, void* stream);
 size_t peqa_bwd_ds_static_capacity_bytes(void);
 
-/* Synchronises `stream`, reads and clears the device status word.  Returns
- * PEQA_OK, PEQA_ERR_DEVICE_TIMEOUT, or PEQA_ERR_CUDA. */
+/*
+ * Decode from a prepared copy of the frozen weights.  Q never changes after
+ * quantization and is shared by every task (Sec. 3.3), so a server may keep it
+ * in the order the small-batch kernel streams best.  The canonical packed
+ * layout above stays the interchange format; the prepared buffer holds exactly
+ * the same bits, rearranged:
+ *   rg = row / 8, r = row % 8, u = column / 128 (U = K / 128), C = bits;
+ *   the 4*bits words of a row's 128-column unit are cut into C chunks of 16
+ *   bytes, and chunk c of unit (row, u) is stored at 16-byte index
+ *   ((rg*C + c)*U + u)*8 + r;
+ *   inside every 32-column run the code of column 2k is stored at code position
+ *   lo(k) and the code of column 2k+1 at position hi(k), k = 0..15, where for
+ *   bits = 4: lo(k) = 8*(k/4) + k%4, hi(k) = lo(k) + 4, and for bits = 3:
+ *   lo = {1,0,3,2,4,9,12,11,15,14,18,21,24,23,26,25},
+ *   hi = {5,6,7,8,10,13,16,17,19,20,22,27,28,29,30,31}
+ *   (code position p = bits [bits*p, bits*p + bits) of the run's bit string).
+ * peqa_decode_unprepare(peqa_decode_prepare(Q)) == Q bit for bit.
+ * Requires K % 128 == 0 and N % 8 == 0; the prepared buffer has
+ * peqa_decode_prepared_bytes(w) = N*K*bits/8 bytes (0 for an unsupported shape)
+ * and must be 16-byte aligned.  Only bits, out_features, in_features and
+ * group_size of *w are read by prepared_bytes and unprepare; prepare also reads
+ * w->qweight.
+ */
+size_t peqa_decode_prepared_bytes(const peqa_qweight_t* w);
+int peqa_decode_prepare(const peqa_qweight_t* w, uint32_t* prepared, void* stream);
+int peqa_decode_unprepare(const peqa_qweight_t* w, const uint32_t* prepared, uint32_t* qweight_out,
+                          void* stream);
+
+/*
+ * Small-batch forward (Sec. 3.1 / 3.3) reading the prepared weights, for layers
+ * with one scale per channel (group_size 0 or K; else PEQA_ERR_BAD_SHAPE):
+ *   Y[m,i] = s_m[i] * sum_j X[m,j] * (Q[i,j] - z[i]),   1 <= M <= 16
+ * where s_m = w->scales, or, when task_ids is not NULL, row
+ * clamp(task_ids[m], 0, n_tasks-1) of scale_table (fp32 [n_tasks, N]): token m is
+ * served with the scales of its own task (Sec. 3.3).  w->qweight is not read.
+ *   X  in  bf16 [M, K]    Y  out  bf16 [M, N]    task_ids  in  int32 [M] (device)
+ * No workspace.  The kernel is launched so that it may begin while earlier work
+ * on `stream` is still draining: it reads `prepared`, w->zeros and the scales
+ * before that work is known to be complete (X is read and Y written only after
+ * it has completed).  These tensors must therefore be final when the call is made
+ * -- synchronise once after peqa_decode_prepare or after loading a scale table.
+ */
+int peqa_qlinear_decode_prepared(const peqa_qweight_t* w, const uint32_t* prepared,
+                                 const void* X_bf16, int M, void* Y_bf16,
+                                 const float* scale_table, int n_tasks, const int32_t* task_ids,
+                                 void* stream);
+
+/*
+ * Measurement aid (the paper has no counterpart): reads `bytes` bytes (a
+ * multiple of 16, 16-byte aligned) with one CTA per SM, each CTA a contiguous
+ * range, and does nothing else.  Its duration is the ceiling for any kernel that
+ * must stream that many bytes from HBM under the same launch conditions; the
+ * benchmark reports decode times next to it (Sec. 3.1: small-batch generation is
+ * bound by the weight read).  sink: device scratch of at least 4 bytes per SM.
+ */
+int peqa_probe_read(const void* src, size_t bytes, uint32_t* sink, size_t sink_bytes, void* stream);
+
+/*
+ * Synchronises `stream`, then reads and clears the status word of that stream.
+ * Returns PEQA_OK, PEQA_ERR_DEVICE_TIMEOUT (a bounded wait of a kernel launched on
+ * `stream` expired since the last check; its outputs are undefined) or
+ * PEQA_ERR_CUDA.  Status words live in the library's device image, one per stream
+ * (the first 31 streams seen on a device get a word of their own, any further
+ * streams share one); entry points without a workspace argument have nowhere
+ * else to report to.  The table is initialised by the first call of any entry
+ * point on a device with a blocking copy: make that call outside stream capture.
+ */
 int peqa_check_status(void* stream);
+
+/*
+ * Self-test of the bounded waits (the paper has no counterpart).  Sets, for
+ * kernels launched afterwards on the current device, the bound of a single
+ * device-side wait to wait_limit_us microseconds (0 restores the default of two
+ * seconds) and, when starve_forward is non-zero, makes peqa_qlinear_fwd's
+ * CTA-pair kernel announce one byte more than its copies deliver, so that its
+ * first stage never fills: the kernel must then leave through its time-out path,
+ * free its tensor memory and report PEQA_ERR_DEVICE_TIMEOUT through
+ * peqa_check_status, leaving the context usable.  Synchronises the device and
+ * clears all status words.  For tests only; never leave it set.
+ */
+int peqa_selftest_configure(int wait_limit_us, int starve_forward);
 
 #ifdef __cplusplus
 }

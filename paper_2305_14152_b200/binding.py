@@ -78,6 +78,18 @@ def lib() -> ctypes.CDLL:
         L.peqa_qlinear_bwd_ds_static.argtypes = [qp, vp, vp, i32, vp, vp]
         L.peqa_qlinear_bwd_ds_static.restype = ctypes.c_int
         L.peqa_bwd_ds_static_capacity_bytes.restype = sz
+        L.peqa_decode_prepared_bytes.argtypes = [qp]
+        L.peqa_decode_prepared_bytes.restype = sz
+        L.peqa_decode_prepare.argtypes = [qp, vp, vp]
+        L.peqa_decode_prepare.restype = ctypes.c_int
+        L.peqa_decode_unprepare.argtypes = [qp, vp, vp, vp]
+        L.peqa_decode_unprepare.restype = ctypes.c_int
+        L.peqa_qlinear_decode_prepared.argtypes = [qp, vp, vp, i32, vp, vp, i32, vp, vp]
+        L.peqa_qlinear_decode_prepared.restype = ctypes.c_int
+        L.peqa_selftest_configure.argtypes = [i32, i32]
+        L.peqa_selftest_configure.restype = ctypes.c_int
+        L.peqa_probe_read.argtypes = [vp, sz, vp, sz, vp]
+        L.peqa_probe_read.restype = ctypes.c_int
         for name in ("peqa_quantize_rtn", "peqa_pack", "peqa_unpack", "peqa_qlinear_fwd",
                      "peqa_qlinear_bwd", "peqa_qlinear_decode", "peqa_scale_adamw",
                      "peqa_train_step_host", "peqa_check_status"):
@@ -333,6 +345,65 @@ def qlinear_bwd_ds_static(w: QWeight, X: torch.Tensor, dY: torch.Tensor, dS: tor
 
 def bwd_ds_static_capacity_bytes() -> int:
     return int(lib().peqa_bwd_ds_static_capacity_bytes())
+
+
+def decode_prepared_bytes(w: QWeight) -> int:
+    cs = w.c_struct()
+    return int(lib().peqa_decode_prepared_bytes(ctypes.byref(cs)))
+
+
+def decode_prepare(w: QWeight) -> torch.Tensor:
+    """Prepared copy of w.qweight for qlinear_decode_prepared (int32 bit patterns, flat)."""
+    n = decode_prepared_bytes(w)
+    if n == 0:
+        raise PeqaError(-3, "peqa_decode_prepared_bytes")
+    out = torch.empty(n // 4, dtype=torch.int32, device=w.qweight.device)
+    cs = w.c_struct()
+    _check(lib().peqa_decode_prepare(ctypes.byref(cs), out.data_ptr(), _stream()), "peqa_decode_prepare")
+    return out
+
+
+def decode_unprepare(w: QWeight, prepared: torch.Tensor) -> torch.Tensor:
+    """Canonical packed matrix rebuilt from a prepared buffer."""
+    _dev(prepared, torch.int32, "prepared")
+    out = torch.empty((w.N, w.K * w.bits // 32), dtype=torch.int32, device=prepared.device)
+    cs = w.c_struct()
+    _check(lib().peqa_decode_unprepare(ctypes.byref(cs), prepared.data_ptr(), out.data_ptr(), _stream()),
+           "peqa_decode_unprepare")
+    return out
+
+
+def qlinear_decode_prepared(w: QWeight, prepared: torch.Tensor, X: torch.Tensor, Y=None,
+                            scale_table=None, task_ids=None):
+    """Decode from the prepared weights; with scale_table [n_tasks, N] and task_ids [M] every
+    token uses the scales of its own task."""
+    _dev(prepared, torch.int32, "prepared")
+    _dev(X, torch.bfloat16, "X")
+    M = X.shape[0]
+    if Y is None:
+        Y = torch.empty((M, w.N), dtype=torch.bfloat16, device=X.device)
+    n_tasks = 0
+    if task_ids is not None:
+        _dev(scale_table, torch.float32, "scale_table")
+        _dev(task_ids, torch.int32, "task_ids")
+        n_tasks = scale_table.shape[0]
+    cs = w.c_struct()
+    _check(lib().peqa_qlinear_decode_prepared(ctypes.byref(cs), prepared.data_ptr(), X.data_ptr(), M,
+                                              Y.data_ptr(), _ptr(scale_table), n_tasks, _ptr(task_ids),
+                                              _stream()), "peqa_qlinear_decode_prepared")
+    return Y
+
+
+def probe_read(buf: torch.Tensor, sink: torch.Tensor) -> None:
+    """Read-only pass over ``buf`` (measurement aid); sink: int32 device tensor, one word per SM."""
+    _check(lib().peqa_probe_read(buf.data_ptr(), buf.numel() * buf.element_size(), sink.data_ptr(),
+                                 sink.numel() * sink.element_size(), _stream()), "peqa_probe_read")
+
+
+def selftest_configure(wait_limit_us: int = 0, starve_forward: bool = False) -> None:
+    """Test knob of the bounded waits; selftest_configure() restores the defaults."""
+    _check(lib().peqa_selftest_configure(int(wait_limit_us), 1 if starve_forward else 0),
+           "peqa_selftest_configure")
 
 
 def check_status() -> None:

@@ -1,18 +1,79 @@
 // C-ABI entry points that only validate and dispatch, plus the library's
 // small amount of per-device state (architecture check, status word).
+#include <mutex>
+
 #include "common.cuh"
+#include "tensor_map.cuh"
 
 namespace peqa {
 
 thread_local int g_last_cuda_error = 0;
 
-// Written by kernels whose bounded waits expire: [0] = status code, [1..3] = where.
-__device__ int g_status_word[4];
+// Written by kernels whose bounded waits expire; one slot per stream (see common.cuh).
+__device__ int g_status_slots[kStatusSlots][kStatusInts];
 
-int status_word(int** dev_ptr) {
-  void* p = nullptr;
-  PEQA_CUDA(cudaGetSymbolAddress(&p, g_status_word));
-  *dev_ptr = static_cast<int*>(p);
+namespace {
+
+constexpr int kMaxDevices = 64;
+constexpr int kDefaultWaitLimitUs = 2000000;   // 2 s
+struct DeviceStatus {
+  int* base = nullptr;                 // device address of g_status_slots
+  cudaStream_t keys[kStatusSlots] = {};
+  int used = 0;
+  int wait_limit_us = kDefaultWaitLimitUs;
+  int selftest_knob = 0;
+};
+std::mutex g_status_mutex;
+DeviceStatus g_device_status[kMaxDevices];
+
+int write_all_slots(const DeviceStatus& ds) {
+  int host[kStatusSlots][kStatusInts] = {};
+  for (int q = 0; q < kStatusSlots; ++q) {
+    host[q][4] = ds.wait_limit_us;
+    host[q][5] = ds.selftest_knob;
+  }
+  PEQA_CUDA(cudaMemcpy(ds.base, host, sizeof(host), cudaMemcpyHostToDevice));
+  return PEQA_OK;
+}
+
+// Caller holds g_status_mutex.
+int device_status(DeviceStatus** out) {
+  int dev = 0;
+  PEQA_CUDA(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return PEQA_ERR_TOO_LARGE;
+  DeviceStatus& ds = g_device_status[dev];
+  if (!ds.base) {
+    void* p = nullptr;
+    PEQA_CUDA(cudaGetSymbolAddress(&p, g_status_slots));
+    ds.base = static_cast<int*>(p);
+    const int rc = write_all_slots(ds);
+    if (rc != PEQA_OK) {
+      ds.base = nullptr;
+      return rc;
+    }
+  }
+  *out = &ds;
+  return PEQA_OK;
+}
+
+}  // namespace
+
+int status_word(cudaStream_t st, int** dev_ptr) {
+  std::lock_guard<std::mutex> lock(g_status_mutex);
+  DeviceStatus* ds = nullptr;
+  PEQA_TRY(device_status(&ds));
+  int slot = -1;
+  for (int q = 0; q < ds->used; ++q)
+    if (ds->keys[q] == st) slot = q;
+  if (slot < 0) {
+    if (ds->used < kStatusSlots - 1) {
+      slot = ds->used++;
+      ds->keys[slot] = st;
+    } else {
+      slot = kStatusSlots - 1;       // shared by every further stream
+    }
+  }
+  *dev_ptr = ds->base + slot * kStatusInts;
   return PEQA_OK;
 }
 
@@ -28,6 +89,36 @@ int check_arch() {
     cached_ok = (major == 10);
   }
   return cached_ok ? PEQA_OK : PEQA_ERR_ARCH;
+}
+
+int tensor_map_encoder(EncodeTiledFn* out) {
+  static std::mutex mu;
+  static EncodeTiledFn cached = nullptr;
+  std::lock_guard<std::mutex> lock(mu);
+  if (!cached) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    PEQA_CUDA(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
+    if (!fn || qres != cudaDriverEntryPointSuccess) return cuda_fail(cudaErrorUnknown);
+    cached = reinterpret_cast<EncodeTiledFn>(fn);
+  }
+  *out = cached;
+  return PEQA_OK;
+}
+
+int sm_count_or(int fallback) {
+  static thread_local int cached_dev = -1;
+  static thread_local int cached_sms = 0;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return fallback;
+  if (dev != cached_dev) {
+    int sms = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+      return fallback;
+    cached_dev = dev;
+    cached_sms = sms;
+  }
+  return cached_sms;
 }
 
 int check_qweight(const peqa_qweight_t* w, int* g, int* G) {
@@ -208,27 +299,52 @@ struct HostPipe {
   bool ready = false;
 };
 
-int host_pipe(HostPipe** out) {
+std::mutex g_pipe_mutex[64];
+
+// Caller holds the device's g_pipe_mutex.  A partly created pipe is torn down again, so a
+// later call starts from scratch instead of leaking.
+int host_pipe(int dev, HostPipe** out) {
   static HostPipe pipes[64];
-  int dev = 0;
-  PEQA_CUDA(cudaGetDevice(&dev));
-  if (dev < 0 || dev >= 64) return PEQA_ERR_BAD_SHAPE;
   HostPipe& hp = pipes[dev];
   if (!hp.ready) {
-    PEQA_CUDA(cudaStreamCreateWithFlags(&hp.in, cudaStreamNonBlocking));
-    PEQA_CUDA(cudaStreamCreateWithFlags(&hp.out, cudaStreamNonBlocking));
-    PEQA_CUDA(cudaEventCreateWithFlags(&hp.start, cudaEventDisableTiming));
-    PEQA_CUDA(cudaEventCreateWithFlags(&hp.out_done, cudaEventDisableTiming));
-    for (int c = 0; c < kHostChunksMax; ++c) {
-      PEQA_CUDA(cudaEventCreateWithFlags(&hp.x_landed[c], cudaEventDisableTiming));
-      PEQA_CUDA(cudaEventCreateWithFlags(&hp.dy_landed[c], cudaEventDisableTiming));
-      PEQA_CUDA(cudaEventCreateWithFlags(&hp.fwd_done[c], cudaEventDisableTiming));
-      PEQA_CUDA(cudaEventCreateWithFlags(&hp.dx_done[c], cudaEventDisableTiming));
+    bool ok = cudaStreamCreateWithFlags(&hp.in, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaStreamCreateWithFlags(&hp.out, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaEventCreateWithFlags(&hp.start, cudaEventDisableTiming) == cudaSuccess &&
+              cudaEventCreateWithFlags(&hp.out_done, cudaEventDisableTiming) == cudaSuccess;
+    for (int c = 0; ok && c < kHostChunksMax; ++c)
+      ok = cudaEventCreateWithFlags(&hp.x_landed[c], cudaEventDisableTiming) == cudaSuccess &&
+           cudaEventCreateWithFlags(&hp.dy_landed[c], cudaEventDisableTiming) == cudaSuccess &&
+           cudaEventCreateWithFlags(&hp.fwd_done[c], cudaEventDisableTiming) == cudaSuccess &&
+           cudaEventCreateWithFlags(&hp.dx_done[c], cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) {
+      const cudaError_t e = cudaGetLastError();
+      if (hp.in) cudaStreamDestroy(hp.in);
+      if (hp.out) cudaStreamDestroy(hp.out);
+      if (hp.start) cudaEventDestroy(hp.start);
+      if (hp.out_done) cudaEventDestroy(hp.out_done);
+      for (int c = 0; c < kHostChunksMax; ++c) {
+        if (hp.x_landed[c]) cudaEventDestroy(hp.x_landed[c]);
+        if (hp.dy_landed[c]) cudaEventDestroy(hp.dy_landed[c]);
+        if (hp.fwd_done[c]) cudaEventDestroy(hp.fwd_done[c]);
+        if (hp.dx_done[c]) cudaEventDestroy(hp.dx_done[c]);
+      }
+      hp = HostPipe();
+      return cuda_fail(e == cudaSuccess ? cudaErrorUnknown : e);
     }
     hp.ready = true;
   }
   *out = &hp;
   return PEQA_OK;
+}
+
+// Everything that can still fail once work is enqueued has been checked before; if a CUDA
+// call fails all the same, the three streams are drained before the error is returned, so no
+// copy into the caller's host buffers is left in flight.
+int drain_and_fail(HostPipe* hp, cudaStream_t st, int rc) {
+  cudaStreamSynchronize(hp->in);
+  cudaStreamSynchronize(hp->out);
+  cudaStreamSynchronize(st);
+  return rc;
 }
 
 }  // namespace
@@ -252,8 +368,17 @@ extern "C" int peqa_train_step_host(const peqa_qweight_t* w, int T,
   if (!h_X || !h_dY || !h_Y || !h_dX || !h_dS || !d_X || !d_dY || !d_Y || !d_dX || !d_dS ||
       !d_m || !d_v)
     return PEQA_ERR_NULL;
-  if (T <= 0) return PEQA_ERR_BAD_SHAPE;
+  if (T <= 0 || step < 1) return PEQA_ERR_BAD_SHAPE;
   PEQA_TRY(check_gemm_shape(w, T));
+  // every check the inner calls would make, before anything is enqueued
+  if (!aligned16(d_X) || !aligned16(d_dY) || !aligned16(d_Y) || !aligned16(d_dX) || !aligned16(d_dS))
+    return PEQA_ERR_ALIGNMENT;
+  const size_t need = ds_workspace_bytes(w, g, T);
+  if (need > 0) {
+    if (!workspace || workspace_bytes < need) return PEQA_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(workspace) & 255u) return PEQA_ERR_ALIGNMENT;
+  }
+  PEQA_TRY(check_arch());
   cudaStream_t st = as_stream(stream);
   const size_t N = w->out_features, K = w->in_features;
   // chunks of whole 512-token tiles, at most kHostChunksMax of them
@@ -261,8 +386,13 @@ extern "C" int peqa_train_step_host(const peqa_qweight_t* w, int T,
   if (chunks > kHostChunksMax) chunks = kHostChunksMax;
   const int per = ((T + chunks - 1) / chunks + 7) & ~7;   // rows per chunk, 16-byte aligned slices
   chunks = (T + per - 1) / per;
+  int dev = 0;
+  PEQA_CUDA(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return PEQA_ERR_TOO_LARGE;
+  // the auxiliary streams and events are shared by all calls on the device: one call at a time
+  std::lock_guard<std::mutex> lock(g_pipe_mutex[dev]);
   HostPipe* hp = nullptr;
-  PEQA_TRY(host_pipe(&hp));
+  PEQA_TRY(host_pipe(dev, &hp));
   const char* hX = static_cast<const char*>(h_X);
   const char* hdY = static_cast<const char*>(h_dY);
   char* hY = static_cast<char*>(h_Y);
@@ -271,46 +401,58 @@ extern "C" int peqa_train_step_host(const peqa_qweight_t* w, int T,
   char* ddY = static_cast<char*>(d_dY);
   char* dY_out = static_cast<char*>(d_Y);
   char* ddX = static_cast<char*>(d_dX);
+#define PIPE_CUDA(expr)                                                        \
+  do {                                                                         \
+    cudaError_t _e = (expr);                                                   \
+    if (_e != cudaSuccess) return drain_and_fail(hp, st, cuda_fail(_e));       \
+  } while (0)
+#define PIPE_TRY(expr)                                                         \
+  do {                                                                         \
+    int _s = (expr);                                                           \
+    if (_s != PEQA_OK) return drain_and_fail(hp, st, _s);                      \
+  } while (0)
   // the auxiliary streams start after whatever the caller's stream already holds
-  PEQA_CUDA(cudaEventRecord(hp->start, st));
-  PEQA_CUDA(cudaStreamWaitEvent(hp->in, hp->start, 0));
-  PEQA_CUDA(cudaStreamWaitEvent(hp->out, hp->start, 0));
+  PIPE_CUDA(cudaEventRecord(hp->start, st));
+  PIPE_CUDA(cudaStreamWaitEvent(hp->in, hp->start, 0));
+  PIPE_CUDA(cudaStreamWaitEvent(hp->out, hp->start, 0));
   for (int c = 0; c < chunks; ++c) {
     const size_t t0 = (size_t)c * per;
     const size_t tc = (size_t)T - t0 < (size_t)per ? (size_t)T - t0 : (size_t)per;
-    PEQA_CUDA(cudaMemcpyAsync(dX_in + t0 * K * 2, hX + t0 * K * 2, tc * K * 2, cudaMemcpyHostToDevice, hp->in));
-    PEQA_CUDA(cudaEventRecord(hp->x_landed[c], hp->in));
-    PEQA_CUDA(cudaMemcpyAsync(ddY + t0 * N * 2, hdY + t0 * N * 2, tc * N * 2, cudaMemcpyHostToDevice, hp->in));
-    PEQA_CUDA(cudaEventRecord(hp->dy_landed[c], hp->in));
+    PIPE_CUDA(cudaMemcpyAsync(dX_in + t0 * K * 2, hX + t0 * K * 2, tc * K * 2, cudaMemcpyHostToDevice, hp->in));
+    PIPE_CUDA(cudaEventRecord(hp->x_landed[c], hp->in));
+    PIPE_CUDA(cudaMemcpyAsync(ddY + t0 * N * 2, hdY + t0 * N * 2, tc * N * 2, cudaMemcpyHostToDevice, hp->in));
+    PIPE_CUDA(cudaEventRecord(hp->dy_landed[c], hp->in));
     // the forward needs only X: it runs while dY is still on its way
-    PEQA_CUDA(cudaStreamWaitEvent(st, hp->x_landed[c], 0));
-    PEQA_TRY(peqa_qlinear_fwd(w, dX_in + t0 * K * 2, (int)tc, dY_out + t0 * N * 2, workspace,
+    PIPE_CUDA(cudaStreamWaitEvent(st, hp->x_landed[c], 0));
+    PIPE_TRY(peqa_qlinear_fwd(w, dX_in + t0 * K * 2, (int)tc, dY_out + t0 * N * 2, workspace,
                               workspace_bytes, stream));
-    PEQA_CUDA(cudaEventRecord(hp->fwd_done[c], st));
-    PEQA_CUDA(cudaStreamWaitEvent(st, hp->dy_landed[c], 0));
-    PEQA_TRY(peqa_qlinear_bwd(w, nullptr, ddY + t0 * N * 2, (int)tc, ddX + t0 * K * 2, nullptr,
+    PIPE_CUDA(cudaEventRecord(hp->fwd_done[c], st));
+    PIPE_CUDA(cudaStreamWaitEvent(st, hp->dy_landed[c], 0));
+    PIPE_TRY(peqa_qlinear_bwd(w, nullptr, ddY + t0 * N * 2, (int)tc, ddX + t0 * K * 2, nullptr,
                               workspace, workspace_bytes, stream));
-    PEQA_CUDA(cudaEventRecord(hp->dx_done[c], st));
+    PIPE_CUDA(cudaEventRecord(hp->dx_done[c], st));
     // Y goes back while dX is still being computed
-    PEQA_CUDA(cudaStreamWaitEvent(hp->out, hp->fwd_done[c], 0));
-    PEQA_CUDA(cudaMemcpyAsync(hY + t0 * N * 2, dY_out + t0 * N * 2, tc * N * 2, cudaMemcpyDeviceToHost, hp->out));
-    PEQA_CUDA(cudaStreamWaitEvent(hp->out, hp->dx_done[c], 0));
-    PEQA_CUDA(cudaMemcpyAsync(hdX + t0 * K * 2, ddX + t0 * K * 2, tc * K * 2, cudaMemcpyDeviceToHost, hp->out));
+    PIPE_CUDA(cudaStreamWaitEvent(hp->out, hp->fwd_done[c], 0));
+    PIPE_CUDA(cudaMemcpyAsync(hY + t0 * N * 2, dY_out + t0 * N * 2, tc * N * 2, cudaMemcpyDeviceToHost, hp->out));
+    PIPE_CUDA(cudaStreamWaitEvent(hp->out, hp->dx_done[c], 0));
+    PIPE_CUDA(cudaMemcpyAsync(hdX + t0 * K * 2, ddX + t0 * K * 2, tc * K * 2, cudaMemcpyDeviceToHost, hp->out));
   }
-  PEQA_CUDA(cudaEventRecord(hp->out_done, hp->out));
-  PEQA_TRY(peqa_qlinear_bwd_ds_adamw(w, d_X, d_dY, T, d_dS, d_m, d_v, lr, beta1, beta2, eps,
+  PIPE_CUDA(cudaEventRecord(hp->out_done, hp->out));
+  PIPE_TRY(peqa_qlinear_bwd_ds_adamw(w, d_X, d_dY, T, d_dS, d_m, d_v, lr, beta1, beta2, eps,
                                      weight_decay, step, workspace, workspace_bytes, stream));
-  PEQA_CUDA(cudaMemcpyAsync(h_dS, d_dS, N * (size_t)G * 4, cudaMemcpyDeviceToHost, st));
-  PEQA_CUDA(cudaStreamWaitEvent(st, hp->out_done, 0));
-  PEQA_CUDA(cudaStreamSynchronize(st));
+  PIPE_CUDA(cudaMemcpyAsync(h_dS, d_dS, N * (size_t)G * 4, cudaMemcpyDeviceToHost, st));
+  PIPE_CUDA(cudaStreamWaitEvent(st, hp->out_done, 0));
+  PIPE_CUDA(cudaStreamSynchronize(st));
+#undef PIPE_CUDA
+#undef PIPE_TRY
   return PEQA_OK;
 }
 
 extern "C" int peqa_check_status(void* stream) {
-  int* dev = nullptr;
-  PEQA_TRY(status_word(&dev));
-  int host[4] = {0, 0, 0, 0};
   cudaStream_t st = as_stream(stream);
+  int* dev = nullptr;
+  PEQA_TRY(status_word(st, &dev));
+  int host[4] = {0, 0, 0, 0};
   PEQA_CUDA(cudaMemcpyAsync(host, dev, sizeof(host), cudaMemcpyDeviceToHost, st));
   PEQA_CUDA(cudaStreamSynchronize(st));
   if (host[0] != 0) {
@@ -319,4 +461,16 @@ extern "C" int peqa_check_status(void* stream) {
     return PEQA_ERR_DEVICE_TIMEOUT;
   }
   return PEQA_OK;
+}
+
+extern "C" int peqa_selftest_configure(int wait_limit_us, int starve_forward) {
+  if (wait_limit_us < 0) return PEQA_ERR_BAD_SHAPE;
+  std::lock_guard<std::mutex> lock(g_status_mutex);
+  DeviceStatus* ds = nullptr;
+  PEQA_TRY(device_status(&ds));
+  PEQA_CUDA(cudaDeviceSynchronize());
+  ds->wait_limit_us = wait_limit_us == 0 ? kDefaultWaitLimitUs : wait_limit_us;
+  ds->selftest_knob = starve_forward ? 1 : 0;
+  // the status codes of all slots are cleared along with the knobs
+  return write_all_slots(*ds);
 }

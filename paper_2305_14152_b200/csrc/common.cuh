@@ -52,8 +52,18 @@ int check_qweight(const peqa_qweight_t* w, int* g, int* G);
 // The current device must be compute capability 10.x (cached per device).
 int check_arch();
 
-// Device address of the library's status word (int[4]) on the current device.
-int status_word(int** dev_ptr);
+// Device address of the status slot kernels launched on `st` report to, on the current
+// device.  A slot is int[8]: [0] status code, [1..3] where, [4] bound of a single device-side
+// wait in microseconds, [5] self-test knob (see peqa_selftest_configure), [6..7] unused.
+// Streams get slots of their own (first come, first served; the last slot is shared by any
+// further streams).  The first call on a device initialises the table with a blocking copy.
+constexpr int kStatusSlots = 32;
+constexpr int kStatusInts = 8;
+int status_word(cudaStream_t st, int** dev_ptr);
+
+// Multiprocessor count of the current device (cached per device); `fallback` when the query
+// fails.
+int sm_count_or(int fallback);
 
 inline cudaStream_t as_stream(void* s) { return reinterpret_cast<cudaStream_t>(s); }
 

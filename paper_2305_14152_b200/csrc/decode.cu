@@ -27,6 +27,7 @@
 #include "common.cuh"
 #include "dequant.cuh"
 #include "sm100_ptx.cuh"
+#include "tensor_map.cuh"
 
 namespace cg = cooperative_groups;
 
@@ -63,6 +64,7 @@ struct DecBarriers {
   uint64_t full[kDecSlots];    // weight step landed in its slot
   uint64_t empty[kDecSlots];   // all compute warps have read the slot
   int abort_flag;
+  int wait_limit_us;    // must follow abort_flag (read by the bounded waits)
 };
 
 __device__ __forceinline__ void mma_16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0,
@@ -148,6 +150,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmap_q, const DecodeParams p) 
       ptx::mbar_init(ptx::smem_u32(&bars->empty[q]), kDecWarps);
     }
     bars->abort_flag = 0;
+    bars->wait_limit_us = p.status[4];
     ptx::fence_mbar_init();
     for (int st = 0; st < nsteps && st < kDecSlots; ++st) issue_step(st);
   }
@@ -465,22 +468,12 @@ int launch_decode(const peqa_qweight_t* w, int g, const void* X, int M, void* Y,
     split *= 2;
   }
   if (smem > 227 * 1024) return PEQA_ERR_TOO_LARGE;
-  PEQA_TRY(status_word(&p.status));
+  PEQA_TRY(status_word(st, &p.status));
   // packed matrix as uint32 [N, wpr]; box = 16 words x 128 rows, 64-byte swizzle
   CUtensorMap tmap_q;
   {
-    typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
-                                      const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
-                                      const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                      CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-    static EncodeTiledFn enc = nullptr;
-    if (!enc) {
-      void* fn = nullptr;
-      cudaDriverEntryPointQueryResult qres;
-      PEQA_CUDA(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
-      if (!fn || qres != cudaDriverEntryPointSuccess) return cuda_fail(cudaErrorUnknown);
-      enc = reinterpret_cast<EncodeTiledFn>(fn);
-    }
+    EncodeTiledFn enc = nullptr;
+    PEQA_TRY(tensor_map_encoder(&enc));
     cuuint64_t dims[2] = {(cuuint64_t)p.wpr, (cuuint64_t)p.N};
     cuuint64_t strides[1] = {(cuuint64_t)p.wpr * 4};
     cuuint32_t box[2] = {16, (cuuint32_t)kRowsPerCta};

@@ -96,6 +96,7 @@ struct StreamBarriers {
   uint64_t full[kSMaxSlots];    // the step's row pieces have landed
   uint64_t empty[kSMaxSlots];   // the warp that owns the step has read it
   int abort_flag;
+  int wait_limit_us;    // must follow abort_flag (read by the bounded waits)
 };
 
 __device__ __forceinline__ void smma_16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0,
@@ -158,6 +159,7 @@ decode_stream_kernel(const StreamParams p) {
       ptx::mbar_init(ptx::smem_u32(&bars->empty[q]), 1);
     }
     bars->abort_flag = 0;
+    bars->wait_limit_us = p.status[4];
     ptx::fence_mbar_init();
   } else if (!is_producer) {
 #pragma unroll
@@ -539,7 +541,7 @@ int launch_decode_stream(const peqa_qweight_t* w, int g, const void* X, int M, v
   p.x_blocks = plan.x_blocks;
   p.x_pitch = plan.x_pitch;
   p.slots = plan.slots;
-  PEQA_TRY(status_word(&p.status));
+  PEQA_TRY(status_word(st, &p.status));
   const bool grouped = p.G > 1;
   const int NT = M <= 8 ? 1 : 2;
   if (w->bits == 4) {

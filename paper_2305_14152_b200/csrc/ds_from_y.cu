@@ -78,7 +78,7 @@ __global__ void ds_from_y_finish_kernel(const float* __restrict__ partial, const
 // Token slices: enough CTAs for a few waves of the machine, at least 32 tokens each.
 int ds_from_y_slices(int N, int T) {
   const int col_blocks = (N + kYCols - 1) / kYCols;
-  int slices = (148 * 8 + col_blocks - 1) / col_blocks;
+  int slices = (sm_count_or(148) * 8 + col_blocks - 1) / col_blocks;
   const int max_slices = (T + 31) / 32;
   if (slices > max_slices) slices = max_slices;
   if (slices < 1) slices = 1;

@@ -25,6 +25,7 @@
 #include "common.cuh"
 #include "dequant.cuh"
 #include "sm100_ptx.cuh"
+#include "tensor_map.cuh"
 
 namespace peqa {
 
@@ -55,6 +56,7 @@ struct DxBarriers {
   uint64_t acc_empty;           // leader: both CTAs' epilogues drained them
   uint32_t tmem_base;
   int abort_flag;
+  int wait_limit_us;    // must follow abort_flag (read by the bounded waits)
 };
 
 struct DxParams {
@@ -98,6 +100,7 @@ qdx_pair_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_consta
     mbar_init(smem_u32(&bars->acc_full), 1);
     mbar_init(smem_u32(&bars->acc_empty), 16);            // 8 epilogue warps in each CTA
     bars->abort_flag = 0;
+    bars->wait_limit_us = p.status[4];
     fence_mbar_init();
     prefetch_tmap(&tmap_dy);
     prefetch_tmap(&tmap_q);
@@ -327,24 +330,6 @@ qdx_pair_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_consta
   }
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
-                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
-                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-int dx_encode_fn(EncodeTiledFn* out) {
-  static EncodeTiledFn cached = nullptr;
-  if (!cached) {
-    void* fn = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    PEQA_CUDA(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
-    if (!fn || qres != cudaDriverEntryPointSuccess) return cuda_fail(cudaErrorUnknown);
-    cached = reinterpret_cast<EncodeTiledFn>(fn);
-  }
-  *out = cached;
-  return PEQA_OK;
-}
-
 template <int BITS>
 int launch_dx_pair_t(const CUtensorMap& ta, const CUtensorMap& tq, const DxParams& p, int pairs,
                      cudaStream_t st) {
@@ -389,9 +374,9 @@ int launch_dx_pair(const peqa_qweight_t* w, int g, const void* dY, int T, void* 
   p.j_tiles = (p.K + 255) / 256;
   p.t_tiles = (T + 511) / 512;
   p.k_blocks = (p.N + XK - 1) / XK;
-  PEQA_TRY(status_word(&p.status));
+  PEQA_TRY(status_word(st, &p.status));
   EncodeTiledFn enc = nullptr;
-  PEQA_TRY(dx_encode_fn(&enc));
+  PEQA_TRY(tensor_map_encoder(&enc));
   CUtensorMap ta, tq;
   {
     cuuint64_t dims[2] = {(cuuint64_t)p.N, (cuuint64_t)T};

@@ -339,7 +339,8 @@ __global__ void adamw_kernel(float* __restrict__ s, const float* __restrict__ gr
   }
 }
 
-int grid_for(long long work_items, int threads, int max_blocks = 148 * 16) {
+int grid_for(long long work_items, int threads, int max_blocks = 0) {
+  if (max_blocks <= 0) max_blocks = sm_count_or(148) * 16;
   long long b = (work_items + threads - 1) / threads;
   if (b < 1) b = 1;
   if (b > max_blocks) b = max_blocks;

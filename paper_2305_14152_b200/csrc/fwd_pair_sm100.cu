@@ -28,6 +28,7 @@
 #include "common.cuh"
 #include "dequant.cuh"
 #include "sm100_ptx.cuh"
+#include "tensor_map.cuh"
 
 namespace peqa {
 
@@ -58,6 +59,7 @@ struct PairBarriers {
   uint64_t acc_empty;           // leader: both CTAs' epilogues drained them
   uint32_t tmem_base;
   int abort_flag;
+  int wait_limit_us;    // must follow abort_flag (read by the bounded waits)
 };
 
 struct PairParams {
@@ -101,6 +103,7 @@ qfwd_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     mbar_init(smem_u32(&bars->acc_full), 1);
     mbar_init(smem_u32(&bars->acc_empty), 16);            // 8 epilogue warps in each CTA
     bars->abort_flag = 0;
+    bars->wait_limit_us = p.status[4];
     fence_mbar_init();
     prefetch_tmap(&tmap_x);
     prefetch_tmap(&tmap_q);
@@ -124,6 +127,9 @@ qfwd_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     if (lane == 0) {
       uint32_t it = 0;
       bool ok = true;
+      // self-test knob (peqa_selftest_configure): announce one byte more than will arrive, so
+      // that the stage never fills and the bounded waits have to end the kernel
+      const uint32_t starve = p.status[5] != 0 ? 1u : 0u;
       for (int tile = pair; ok && tile < total_tiles; tile += n_pairs) {
         const int tt0 = (tile / p.n_tiles) * 512;
         const int blocks = tt0 + 256 < p.T ? 2 : 1;
@@ -132,7 +138,7 @@ qfwd_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
           const int s = it % PSTAGES;
           const uint32_t ph = (it / PSTAGES) & 1u;
           if (!mbar_wait_cluster(smem_u32(&bars->empty[s]), ph ^ 1u, abort_flag)) { ok = false; break; }
-          if (leader) mbar_arrive_expect_tx(smem_u32(&bars->full_act[s]), 2 * blocks * PBLK_BYTES);
+          if (leader) mbar_arrive_expect_tx(smem_u32(&bars->full_act[s]), 2 * blocks * PBLK_BYTES + starve);
           const uint32_t bar = mapa_shared(smem_u32(&bars->full_act[s]), 0);
           tma_load_2d_pair(smem_u32(base + s * PSTAGE_BYTES), &tmap_x, bar, kb * PK, t0);
           if (blocks == 2)
@@ -371,24 +377,6 @@ qfwd_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
   }
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
-                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
-                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-int encode_fn(EncodeTiledFn* out) {
-  static EncodeTiledFn cached = nullptr;
-  if (!cached) {
-    void* fn = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    PEQA_CUDA(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
-    if (!fn || qres != cudaDriverEntryPointSuccess) return cuda_fail(cudaErrorUnknown);
-    cached = reinterpret_cast<EncodeTiledFn>(fn);
-  }
-  *out = cached;
-  return PEQA_OK;
-}
-
 template <int BITS, bool FOLD>
 int launch_pair_t(const CUtensorMap& tx, const CUtensorMap& tq, const PairParams& p, int pairs,
                   cudaStream_t st) {
@@ -435,9 +423,9 @@ int launch_fwd_pair(const peqa_qweight_t* w, int g, const void* X, int T, void* 
   p.n_tiles = (p.N + 255) / 256;
   p.t_tiles = (T + 511) / 512;
   p.k_blocks = (p.K + PK - 1) / PK;
-  PEQA_TRY(status_word(&p.status));
+  PEQA_TRY(status_word(st, &p.status));
   EncodeTiledFn enc = nullptr;
-  PEQA_TRY(encode_fn(&enc));
+  PEQA_TRY(tensor_map_encoder(&enc));
   CUtensorMap tx, tq;
   {
     cuuint64_t dims[2] = {(cuuint64_t)p.K, (cuuint64_t)T};

@@ -31,6 +31,7 @@
 #include "common.cuh"
 #include "dequant.cuh"
 #include "sm100_ptx.cuh"
+#include "tensor_map.cuh"
 
 namespace peqa {
 
@@ -66,6 +67,7 @@ struct Barriers {
   uint64_t acc_empty[2];     // accumulator drained by the epilogue
   uint32_t tmem_base;
   int abort_flag;
+  int wait_limit_us;    // must follow abort_flag (read by the bounded waits)
 };
 
 struct SmemView {
@@ -193,6 +195,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmap_act,
       mbar_init(smem_u32(&bars->acc_empty[b]), 128);
     }
     bars->abort_flag = 0;
+    bars->wait_limit_us = p.status[4];
     fence_mbar_init();
     prefetch_tmap(&tmap_act);
     if (PKTMA) prefetch_tmap(&tmap_pk);
@@ -485,6 +488,7 @@ struct DsBarriers {
   uint64_t acc_empty[2];        // leader: both CTAs' epilogues drained the accumulator
   uint32_t tmem_base;
   int abort_flag;
+  int wait_limit_us;    // must follow abort_flag (read by the bounded waits)
 };
 
 template <int BITS, bool DZ, bool ADAM>
@@ -510,6 +514,7 @@ ds_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_constant__ C
       mbar_init(smem_u32(&bars->acc_empty[b]), 16);   // 8 epilogue warps in each of the 2 CTAs
     }
     bars->abort_flag = 0;
+    bars->wait_limit_us = p.status[4];
     fence_mbar_init();
     prefetch_tmap(&tmap_dy);
     prefetch_tmap(&tmap_x);
@@ -698,30 +703,13 @@ __global__ void ds_reduce_kernel(const float* __restrict__ partial, float* __res
 }
 
 // --------------------------------------------------------------- host side
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
-                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
-                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-int get_encode_fn(EncodeTiledFn* out) {
-  static EncodeTiledFn cached = nullptr;
-  if (!cached) {
-    void* fn = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    PEQA_CUDA(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
-    if (!fn || qres != cudaDriverEntryPointSuccess) return cuda_fail(cudaErrorUnknown);
-    cached = reinterpret_cast<EncodeTiledFn>(fn);
-  }
-  *out = cached;
-  return PEQA_OK;
-}
 
 // bf16 row-major [outer, inner] tensor, box = [box_outer rows, 64 elements], 128B swizzle,
 // out-of-bounds elements read as zero.
 int make_tmap_bf16(CUtensorMap* m, const void* base, uint64_t inner, uint64_t outer,
                    uint32_t box_outer) {
   EncodeTiledFn enc = nullptr;
-  PEQA_TRY(get_encode_fn(&enc));
+  PEQA_TRY(tensor_map_encoder(&enc));
   cuuint64_t dims[2] = {inner, outer};
   cuuint64_t strides[1] = {inner * 2};
   cuuint32_t box[2] = {64, box_outer};
@@ -789,7 +777,7 @@ int launch_qgemm(const peqa_qweight_t* w, int g, const void* act, int T, void* o
   p.r_tiles = (p.R + BM - 1) / BM;
   p.t_tiles = (T + BN - 1) / BN;
   p.k_blocks = (p.C + BK - 1) / BK;
-  PEQA_TRY(status_word(&p.status));
+  PEQA_TRY(status_word(st, &p.status));
   CUtensorMap tmap;
   PEQA_TRY(make_tmap_bf16(&tmap, act, (uint64_t)p.C, (uint64_t)T, BN));
   int sms = 0;
@@ -802,7 +790,7 @@ int launch_qgemm(const peqa_qweight_t* w, int g, const void* act, int T, void* o
   CUtensorMap tmap_pk = tmap;
   if (pktma) {
     EncodeTiledFn enc = nullptr;
-    PEQA_TRY(get_encode_fn(&enc));
+    PEQA_TRY(tensor_map_encoder(&enc));
     cuuint64_t dims[2] = {(cuuint64_t)p.wpr, (cuuint64_t)p.N};
     cuuint64_t strides[1] = {(cuuint64_t)p.wpr * 4};
     cuuint32_t box[2] = {trans ? (cuuint32_t)(4 * w->bits) : 8u, trans ? 64u : 128u};
@@ -879,7 +867,7 @@ int launch_ds(const peqa_qweight_t* w, int g, const void* X, const void* dY, int
   p.i_tiles = (p.N + 2 * BM - 1) / (2 * BM);   // 256-row pair tiles
   p.j_tiles = (p.K + BN - 1) / BN;
   p.k_blocks = (T + BK - 1) / BK;
-  PEQA_TRY(status_word(&p.status));
+  PEQA_TRY(status_word(st, &p.status));
   CUtensorMap tmap_dy, tmap_x;
   PEQA_TRY(make_tmap_bf16(&tmap_dy, dY, (uint64_t)p.N, (uint64_t)T, BK));
   PEQA_TRY(make_tmap_bf16(&tmap_x, X, (uint64_t)p.K, (uint64_t)T, BK));

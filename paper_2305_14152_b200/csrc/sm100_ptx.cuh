@@ -52,7 +52,13 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 
 // Wall-clock bound on any single wait.  A correct launch never comes near it;
 // it exists so that a protocol error ends the kernel instead of hanging the GPU.
-constexpr uint64_t kWaitLimitNs = 2000000000ull;  // 2 s
+// The abort flag of a CTA is the first of two adjacent words in shared memory;
+// the second holds the bound in microseconds (kWaitLimitUs unless the host
+// lowered it for a self-test).
+constexpr uint32_t kWaitLimitUs = 2000000u;  // 2 s
+__device__ __forceinline__ uint64_t wait_limit_ns(volatile int* abort_flag) {
+  return (uint64_t)(uint32_t)abort_flag[1] * 1000ull;
+}
 
 // Waits for the phase with the given parity.  Returns false when the bound ran
 // out or another role already raised `abort_flag` (a word in shared memory).
@@ -65,7 +71,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity,
     if (mbar_try_wait(bar, parity)) return true;
     if ((++spins & 63u) == 0u) {
       if (*abort_flag) return false;
-      if (global_timer_ns() - t0 > kWaitLimitNs) {
+      if (global_timer_ns() - t0 > wait_limit_ns(abort_flag)) {
         *abort_flag = 1;
         return false;
       }
@@ -225,7 +231,7 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity,
     if (mbar_try_wait_cluster(bar, parity)) return true;
     if ((++spins & 63u) == 0u) {
       if (*abort_flag) return false;
-      if (global_timer_ns() - t0 > kWaitLimitNs) {
+      if (global_timer_ns() - t0 > wait_limit_ns(abort_flag)) {
         *abort_flag = 1;
         return false;
       }
