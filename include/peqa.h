@@ -254,10 +254,11 @@ int peqa_train_step_host(const peqa_qweight_t* w, int T,
  * device image (each GPU that loads the library holds it until the process
  * ends); peqa_bwd_ds_static_capacity_bytes() returns that size.  A layer
  * whose peqa_workspace_bytes(PEQA_OP_BWD, T, w) exceeds it is refused with
- * PEQA_ERR_TOO_LARGE and nothing is enqueued.  The call performs no
- * allocation of any kind.  The first call on each device looks the array's
- * device address up (with that device current) and caches it; make that
- * first call outside any stream capture.  All calls on a device share the one
+ * PEQA_ERR_TOO_LARGE and nothing is enqueued.  The first call on each device
+ * looks the array's device address up (with that device current) and caches
+ * it; that lookup and the first launch make the driver load the module that
+ * carries the array, so make that first call outside any stream capture.
+ * After it, a call allocates nothing of any kind.  All calls on a device share the one
  * array: it keeps whatever the previous call left, every value that is read
  * is rewritten first, and two calls whose kernels may overlap on the GPU
  * (different streams) race on it -- serialise them.  Same shape rules and

@@ -16,10 +16,15 @@ def _check(d, bits, g, M, also_fwd=False):
     qw = to_qweight(packed, zeros, scales, bits, g, K)
     Xb = d["X"][:M]
     X = bf16_to_dev(Xb)
-    Y = binding.qlinear_decode(qw, X)
-    torch.cuda.synchronize()
+    # the output sits between two guard rows that must survive
+    N = packed.shape[0]
+    buf = torch.full((M + 2, N), 7.0, dtype=torch.bfloat16, device="cuda")
+    Y = buf[1:M + 1]
+    binding.qlinear_decode(qw, X, Y)
+    binding.check_status()
     ref = oracle.fwd(Xb, packed, zeros, scales, bits, g)
     assert_close(dev_to_f64(Y), ref, f"decode M={M}")
+    assert torch.all(buf[0] == 7.0) and torch.all(buf[M + 1] == 7.0)
     if also_fwd:
         Y2 = binding.qlinear_fwd(qw, X)
         binding.check_status()

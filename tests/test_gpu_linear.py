@@ -18,11 +18,31 @@ def _run_all(d, bits, g, check=("Y", "dX", "dS")):
     X = bf16_to_dev(d["X"])
     dY = bf16_to_dev(d["dY"])
     out = {}
+    T, N = X.shape[0], packed.shape[0]
+    G = scales.shape[1]
+
+    # every output sits between two guard rows that must survive (in place of a memory checker)
+    def guarded(rows, cols, dtype):
+        buf = torch.full((rows + 2, cols), 7.0, dtype=dtype, device="cuda")
+        return buf, buf[1:rows + 1]
+
+    guards = []
     if "Y" in check:
-        Y = binding.qlinear_fwd(qw, X)
+        gb, Y = guarded(T, N, torch.bfloat16)
+        guards.append(gb)
+        binding.qlinear_fwd(qw, X, Y)
         out["Y"] = assert_close(dev_to_f64(Y), oracle.fwd(d["X"], packed, zeros, scales, bits, g), "Y")
-    dX, dS = binding.qlinear_bwd(qw, X, dY, need_dx="dX" in check, need_ds="dS" in check)
+    dX = dS = None
+    if "dX" in check:
+        gb, dX = guarded(T, K, torch.bfloat16)
+        guards.append(gb)
+    if "dS" in check:
+        gb, dS = guarded(N, G, torch.float32)
+        guards.append(gb)
+    dX, dS = binding.qlinear_bwd(qw, X, dY, dX=dX, dS=dS, need_dx="dX" in check, need_ds="dS" in check)
     binding.check_status()
+    for gb in guards:
+        assert torch.all(gb[0] == 7.0) and torch.all(gb[-1] == 7.0), "a kernel wrote outside its output"
     if "dX" in check:
         out["dX"] = assert_close(dev_to_f64(dX), oracle.bwd_dx(d["dY"], packed, zeros, scales, K, bits, g), "dX")
     if "dS" in check:

@@ -38,6 +38,13 @@ def test_static_scratch_matches_workspace_path_twice_in_a_row():
         binding.check_status()
         assert_close(dev_to_f64(got), dev_to_f64(ref), "dS static vs workspace")
         assert_close(dev_to_f64(got), oracle.bwd_ds(d["X"], d["dY"], packed, zeros, qw.bits, 0), "dS static vs oracle")
+        # once a device has seen its first call, further calls leave the amount of free device
+        # memory and torch's own allocator untouched
+        torch.cuda.synchronize()
+        free0, used0 = torch.cuda.mem_get_info()[0], torch.cuda.memory_allocated()
+        binding.qlinear_bwd_ds_static(qw, X, dY, got)
+        torch.cuda.synchronize()
+        assert torch.cuda.mem_get_info()[0] == free0 and torch.cuda.memory_allocated() == used0
 
 
 def test_group_sizes_that_need_no_scratch_and_oversize_refusal():
