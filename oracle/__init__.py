@@ -227,3 +227,67 @@ def adamw(s, grad, m, v, lr, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.0,
     lib.oracle_adamw(_p(s), _p(grad), _p(m), _p(v), n, float(lr), float(beta1), float(beta2),
                      float(eps), float(weight_decay), int(step), _p(so), _p(mo), _p(vo))
     return so, mo, vo
+
+
+def quantize_search(W: np.ndarray, bits: int, group_size: int = 0, n_cand: int = 32):
+    """Eq. 1 with the clipping range searched per (row, group) for the smallest reconstruction
+    error (Sec. 3.2's "initialized to minimize"; the search is this library's reading).
+    Returns (codes, zeros, scales, chosen candidate u8 [N,G], error f64 [N,G])."""
+    W = _c(W, np.float32)
+    N, K = W.shape
+    g = _group(K, group_size)
+    G = K // g
+    codes = np.empty((N, K), np.uint8)
+    zeros = np.empty((N, G), np.uint8)
+    scales = np.empty((N, G), np.float32)
+    chosen = np.empty((N, G), np.uint8)
+    err = np.empty((N, G), np.float64)
+    _load().oracle_quantize_search(_p(W), N, K, bits, g, int(n_cand), _p(codes), _p(zeros), _p(scales),
+                                   _p(chosen), _p(err))
+    return codes, zeros, scales, chosen, err
+
+
+def fwd_zf(X_bits, qweight, zeros_f, scales, bits: int, group_size: int = 0, tokens=None) -> np.ndarray:
+    """Forward with a real-valued zero-point (App. K): Y = X (s*(Q - z))^T, z binary32 [N,G]."""
+    X_bits = _c(X_bits, np.uint16)
+    T, K = X_bits.shape
+    g = _group(K, group_size)
+    codes = unpack(qweight, K, bits)
+    N = codes.shape[0]
+    zeros_f = _c(zeros_f, np.float32).reshape(N, K // g)
+    scales = _c(scales, np.float32).reshape(N, K // g)
+    keep, n_sel, ptr = _sel(tokens)
+    rows = n_sel if tokens is not None else T
+    Y = np.empty((rows, N), np.float64)
+    _load().oracle_fwd_zf(_p(X_bits), T, _p(codes), _p(zeros_f), _p(scales), N, K, g, ptr, n_sel, _p(Y))
+    return Y
+
+
+def bwd_dx_zf(dY_bits, qweight, zeros_f, scales, K: int, bits: int, group_size: int = 0, tokens=None) -> np.ndarray:
+    dY_bits = _c(dY_bits, np.uint16)
+    T, N = dY_bits.shape
+    g = _group(K, group_size)
+    codes = unpack(qweight, K, bits)
+    zeros_f = _c(zeros_f, np.float32).reshape(N, K // g)
+    scales = _c(scales, np.float32).reshape(N, K // g)
+    keep, n_sel, ptr = _sel(tokens)
+    rows = n_sel if tokens is not None else T
+    dX = np.empty((rows, K), np.float64)
+    _load().oracle_bwd_dx_zf(_p(dY_bits), T, _p(codes), _p(zeros_f), _p(scales), N, K, g, ptr, n_sel, _p(dX))
+    return dX
+
+
+def bwd_ds_zf(X_bits, dY_bits, qweight, zeros_f, bits: int, group_size: int = 0, rows=None) -> np.ndarray:
+    X_bits = _c(X_bits, np.uint16)
+    dY_bits = _c(dY_bits, np.uint16)
+    T, K = X_bits.shape
+    N = dY_bits.shape[1]
+    g = _group(K, group_size)
+    G = K // g
+    codes = unpack(qweight, K, bits)
+    zeros_f = _c(zeros_f, np.float32).reshape(N, G)
+    keep, n_sel, ptr = _sel(rows)
+    n_out = n_sel if rows is not None else N
+    dS = np.empty((n_out, G), np.float64)
+    _load().oracle_bwd_ds_zf(_p(X_bits), _p(dY_bits), T, _p(codes), _p(zeros_f), N, K, g, ptr, n_sel, _p(dS))
+    return dS

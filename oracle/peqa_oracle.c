@@ -21,7 +21,11 @@
  * words, brute-force Python loops on tiny shapes, s=1,z=0 integer matmul,
  * g=K == per-channel, linearity of <dY,Y> in s (finite difference == dS),
  * the adjoint identity <dY,fwd(X)> == <dX,X>, and the closed form of the
- * first AdamW step.  No function here is "parity unpinned".
+ * first AdamW step; for the searched quantizer: candidate 0 == plain RTN, a
+ * brute-force search on tiny groups, never worse than RTN; for the real-valued
+ * zero-point: equality with the integer functions on integral z, exact rational
+ * brute force, and finite differences of <dY,Y> in z.  No function here is
+ * "parity unpinned".
  */
 #include <math.h>
 #include <stdint.h>
@@ -302,6 +306,167 @@ void oracle_bwd_ds_from_y(const uint16_t* dY, const uint16_t* Y, const float* sc
         for (int t = 0; t < T; ++t)
             acc += bf16_to_double(dY[(size_t)t * N + i]) * bf16_to_double(Y[(size_t)t * N + i]);
         dS[i] = acc / (double)scales[i];
+    }
+}
+
+/* ------------------------------------- Eq. 1 with a searched clipping range --
+ * Sec. 3.2 says that s0 and z0 "are initialized to minimize" the Frobenius error
+ * of Eq. 1 and gives no procedure (Sec. 4.1 names plain round-to-nearest).  The
+ * reading taken: per (row, group), try n_cand shrunken ranges and keep the one
+ * whose reconstruction error is smallest.  Candidate k = 0 .. n_cand-1 scales the
+ * group's extremes by p_k = 1 - k/64 (k = 0 is the plain min/max range of
+ * oracle_quantize_rtn) and then follows Eq. 1 exactly as above, in binary32:
+ *     lo = p*mn, hi = p*mx;  s = (hi - lo)/(2^b-1)  (s := 1 when hi == lo)
+ *     z = clamp(rint(-lo/s), 0, 2^b-1);  q_j = clamp(rint(w_j/s) + z, 0, 2^b-1)
+ *     r_j = s*(q_j - z);  e_j = w_j - r_j                       (binary32 each)
+ *     err = sum_j e_j^2    in binary64, columns in ascending order
+ * The first candidate with the smallest err wins (a later one must be strictly
+ * better), so the result is never worse than plain round-to-nearest.
+ * chosen[i*G+gi] receives the winning k; err_out (may be NULL) its error.
+ * n_cand <= 64.
+ */
+void oracle_quantize_search(const float* W, int N, int K, int bits, int g, int n_cand,
+                            uint8_t* codes, uint8_t* zeros, float* scales, uint8_t* chosen,
+                            double* err_out) {
+    const float qmax = (float)((1 << bits) - 1);
+    const int G = n_groups(K, g);
+#pragma omp parallel for schedule(static)
+    for (int i = 0; i < N; ++i) {
+        uint8_t* tmp = (uint8_t*)malloc((size_t)g);
+        for (int gi = 0; gi < G; ++gi) {
+            const float* w = W + (size_t)i * K + (size_t)gi * g;
+            uint8_t* out = codes + (size_t)i * K + (size_t)gi * g;
+            float mn = w[0], mx = w[0];
+            for (int j = 1; j < g; ++j) {
+                if (w[j] < mn) mn = w[j];
+                if (w[j] > mx) mx = w[j];
+            }
+            double best = 0.0;
+            int best_k = -1;
+            for (int k = 0; k < n_cand; ++k) {
+                volatile float p = 1.0f - (float)k / 64.0f;
+                volatile float lo = p * mn;
+                volatile float hi = p * mx;
+                volatile float range = hi - lo;
+                volatile float s = range / qmax;
+                if (hi == lo) s = 1.0f;
+                volatile float zq = (-lo) / s;
+                float z = rintf(zq);
+                if (z < 0.0f) z = 0.0f;
+                if (z > qmax) z = qmax;
+                double err = 0.0;
+                for (int j = 0; j < g; ++j) {
+                    volatile float r = w[j] / s;
+                    volatile float q = rintf(r) + z;
+                    float qc = q;
+                    if (qc < 0.0f) qc = 0.0f;
+                    if (qc > qmax) qc = qmax;
+                    volatile float d = qc - z;
+                    volatile float rec = s * d;
+                    volatile float e = w[j] - rec;
+                    err += (double)e * (double)e;
+                    tmp[j] = (uint8_t)qc;
+                }
+                if (best_k < 0 || err < best) {
+                    best = err;
+                    best_k = k;
+                    scales[(size_t)i * G + gi] = s;
+                    zeros[(size_t)i * G + gi] = (uint8_t)z;
+                    memcpy(out, tmp, (size_t)g);
+                }
+            }
+            chosen[(size_t)i * G + gi] = (uint8_t)best_k;
+            if (err_out) err_out[(size_t)i * G + gi] = best;
+        }
+        free(tmp);
+    }
+}
+
+/* --------------------------------------- the layer with a real-valued z -----
+ * App. K also trains the zero-points ("zero-points only", "both"); z then leaves
+ * the integer grid and Eq. 2's weight is W_hat[i,j] = s[i,g] * (Q[i,j] - z[i,g])
+ * with z a binary32 number.  The three functions below are oracle_fwd,
+ * oracle_bwd_dx and oracle_bwd_ds with that z; the zero-point gradient
+ * (oracle_bwd_dz) does not depend on z.
+ */
+static void what_row_zf(const uint8_t* codes, const float* zeros_f, const float* scales,
+                        int K, int g, int i, double* out) {
+    const int G = n_groups(K, g);
+    for (int j = 0; j < K; ++j) {
+        int gi = j / g;
+        double s = (double)scales[(size_t)i * G + gi];
+        double wbar = (double)codes[(size_t)i * K + j] - (double)zeros_f[(size_t)i * G + gi];
+        out[j] = s * wbar;
+    }
+}
+
+void oracle_fwd_zf(const uint16_t* X, int T, const uint8_t* codes, const float* zeros_f,
+                   const float* scales, int N, int K, int g,
+                   const int32_t* tok_sel, int n_sel, double* Y) {
+    if (!tok_sel) n_sel = T;
+#pragma omp parallel
+    {
+        double* w = (double*)malloc((size_t)K * sizeof(double));
+#pragma omp for schedule(static)
+        for (int i = 0; i < N; ++i) {
+            what_row_zf(codes, zeros_f, scales, K, g, i, w);
+            for (int r = 0; r < n_sel; ++r) {
+                int t = tok_sel ? tok_sel[r] : r;
+                double acc = 0.0;
+                for (int j = 0; j < K; ++j) acc += bf16_to_double(X[(size_t)t * K + j]) * w[j];
+                Y[(size_t)r * N + i] = acc;
+            }
+        }
+        free(w);
+    }
+}
+
+void oracle_bwd_dx_zf(const uint16_t* dY, int T, const uint8_t* codes, const float* zeros_f,
+                      const float* scales, int N, int K, int g,
+                      const int32_t* tok_sel, int n_sel, double* dX) {
+    if (!tok_sel) n_sel = T;
+    double* What = (double*)malloc((size_t)N * K * sizeof(double));
+#pragma omp parallel for schedule(static)
+    for (int i = 0; i < N; ++i) what_row_zf(codes, zeros_f, scales, K, g, i, What + (size_t)i * K);
+#pragma omp parallel for schedule(static)
+    for (int r = 0; r < n_sel; ++r) {
+        int t = tok_sel ? tok_sel[r] : r;
+        double* out = dX + (size_t)r * K;
+        for (int j = 0; j < K; ++j) out[j] = 0.0;
+        for (int i = 0; i < N; ++i) {
+            double d = bf16_to_double(dY[(size_t)t * N + i]);
+            const double* w = What + (size_t)i * K;
+            for (int j = 0; j < K; ++j) out[j] += d * w[j];
+        }
+    }
+    free(What);
+}
+
+void oracle_bwd_ds_zf(const uint16_t* X, const uint16_t* dY, int T, const uint8_t* codes,
+                      const float* zeros_f, int N, int K, int g,
+                      const int32_t* row_sel, int n_sel, double* dS) {
+    const int G = n_groups(K, g);
+    if (!row_sel) n_sel = N;
+#pragma omp parallel
+    {
+        double* dw = (double*)malloc((size_t)K * sizeof(double));
+#pragma omp for schedule(static)
+        for (int r = 0; r < n_sel; ++r) {
+            int i = row_sel ? row_sel[r] : r;
+            for (int j = 0; j < K; ++j) dw[j] = 0.0;
+            for (int t = 0; t < T; ++t) {
+                double d = bf16_to_double(dY[(size_t)t * N + i]);
+                for (int j = 0; j < K; ++j) dw[j] += d * bf16_to_double(X[(size_t)t * K + j]);
+            }
+            for (int gi = 0; gi < G; ++gi) {
+                double acc = 0.0;
+                double z = (double)zeros_f[(size_t)i * G + gi];
+                for (int j = gi * g; j < (gi + 1) * g; ++j)
+                    acc += ((double)codes[(size_t)i * K + j] - z) * dw[j];
+                dS[(size_t)r * G + gi] = acc;
+            }
+        }
+        free(dw);
     }
 }
 
