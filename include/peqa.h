@@ -96,6 +96,25 @@ int peqa_last_cuda_error(void);
 int peqa_quantize_rtn(const float* W, int N, int K, int bits, int group_size,
                       uint32_t* qweight, uint8_t* zeros, float* scales, void* stream);
 
+/*
+ * Quantization with a searched clipping range.  Sec. 3.2 says s0 and z0 "are
+ * initialized to minimize" the Frobenius error of Eq. 1 without giving a
+ * procedure; this entry point reads it as a search over shrunken ranges.  Per
+ * (row, group), candidate k = 0 .. n_candidates-1 scales the group's extremes by
+ * p_k = 1 - k/64 and applies Eq. 1 in binary32 exactly as peqa_quantize_rtn does
+ * (lo = p*mn, hi = p*mx, s = (hi-lo)/(2^b-1), z = clamp(rint(-lo/s)),
+ * q = clamp(rint(w/s) + z)); its error is sum_j (w_j - s*(q_j - z))^2 with binary32
+ * terms summed in binary64 in column order.  The first candidate with the smallest
+ * error wins, so the result is never worse than peqa_quantize_rtn (candidate 0).
+ *   W in fp32 [N, K];  qweight, zeros, scales out as in peqa_quantize_rtn;
+ *   chosen  out  uint8 [N, G], the winning k (may be NULL).
+ * 1 <= n_candidates <= 64.  An initialisation step (about n_candidates times the
+ * work of peqa_quantize_rtn), not part of the training or serving loop.
+ */
+int peqa_quantize_search(const float* W, int N, int K, int bits, int group_size, int n_candidates,
+                         uint32_t* qweight, uint8_t* zeros, float* scales, uint8_t* chosen,
+                         void* stream);
+
 /* Pack one code per byte (values in [0, 2^bits-1], upper bits ignored) into the
  * packed layout above, and the inverse.  codes is uint8 [N, K]; K % 32 == 0.
  * (The paper only states that the weights are a b-bit integer matrix, Sec. 3.3.) */
@@ -162,6 +181,33 @@ int peqa_qlinear_bwd_ds_adamw(const peqa_qweight_t* w, const void* X_bf16, const
 int peqa_qlinear_bwd_dsdz(const peqa_qweight_t* w, const void* X_bf16, const void* dY_bf16, int T,
                           float* dS, float* dZ, void* workspace, size_t workspace_bytes,
                           void* stream);
+
+/*
+ * The layer with a real-valued zero-point.  App. K also trains the zero-points
+ * ("zero-points only", "both zero-points and quantization scales"); z then leaves
+ * the integer grid, and Eq. 2's weight is W_hat[i,j] = s[i,g] * (Q[i,j] - z[i,g])
+ * with z a binary32 tensor zeros_f [N, G] that replaces w->zeros (which may be
+ * NULL here).  Forward and dX fold s*(Q - z) into the bf16 operand, for every
+ * group size, as (Q - zi)*s - (z - zi)*s with zi = clamp(rint(z), 0, 2^b-1), one
+ * fused multiply-add on exact integers.  The gradients follow from the chain rule
+ * on Eq. 2:
+ *   dS[i,g] = sum_{j in g} (Q[i,j] - z[i,g]) * dW[i,j]
+ *   dZ[i,g] = -s[i,g] * sum_{j in g} dW[i,j],          dW = dY^T X (never stored)
+ * peqa_qlinear_bwd_zf: dX may be NULL (skipped); dS and dZ are both given or both
+ * NULL; they need X and a workspace of peqa_workspace_bytes(PEQA_OP_BWD_DSDZ, T, w)
+ * bytes when that is non-zero.  Shape rules as peqa_qlinear_fwd / _bwd.
+ * One training step of a mode of App. K is then: peqa_qlinear_fwd_zf,
+ * peqa_qlinear_bwd_zf, and peqa_scale_adamw on s and/or peqa_zero_adamw on z
+ * (the same AdamW step, App. A, applied to the zero-points with dZ).
+ */
+int peqa_qlinear_fwd_zf(const peqa_qweight_t* w, const float* zeros_f, const void* X_bf16, int T,
+                        void* Y_bf16, void* stream);
+int peqa_qlinear_bwd_zf(const peqa_qweight_t* w, const float* zeros_f, const void* X_bf16,
+                        const void* dY_bf16, int T, void* dX_bf16, float* dS, float* dZ,
+                        void* workspace, size_t workspace_bytes, void* stream);
+int peqa_zero_adamw(float* zeros_f, const float* dZ, float* m, float* v, int64_t numel, float lr,
+                    float beta1, float beta2, float eps, float weight_decay, int64_t step,
+                    void* stream);
 
 /*
  * Scale gradient of a per-channel layer (group_size 0 or K, the paper's main

@@ -57,6 +57,8 @@ def lib() -> ctypes.CDLL:
         L.peqa_version.restype = ctypes.c_int
         L.peqa_last_cuda_error.restype = ctypes.c_int
         L.peqa_quantize_rtn.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, vp]
+        L.peqa_quantize_search.argtypes = [vp, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp]
+        L.peqa_quantize_search.restype = ctypes.c_int
         L.peqa_pack.argtypes = [vp, i32, i32, i32, vp, vp]
         L.peqa_unpack.argtypes = [vp, i32, i32, i32, vp, vp]
         L.peqa_workspace_bytes.argtypes = [i32, i32, qp]
@@ -86,6 +88,12 @@ def lib() -> ctypes.CDLL:
         L.peqa_decode_unprepare.restype = ctypes.c_int
         L.peqa_qlinear_decode_prepared.argtypes = [qp, vp, vp, i32, vp, vp, i32, vp, vp]
         L.peqa_qlinear_decode_prepared.restype = ctypes.c_int
+        L.peqa_qlinear_fwd_zf.argtypes = [qp, vp, vp, i32, vp, vp]
+        L.peqa_qlinear_fwd_zf.restype = ctypes.c_int
+        L.peqa_qlinear_bwd_zf.argtypes = [qp, vp, vp, vp, i32, vp, vp, vp, vp, sz, vp]
+        L.peqa_qlinear_bwd_zf.restype = ctypes.c_int
+        L.peqa_zero_adamw.argtypes = [vp, vp, vp, vp, i64, f32, f32, f32, f32, f32, i64, vp]
+        L.peqa_zero_adamw.restype = ctypes.c_int
         L.peqa_selftest_configure.argtypes = [i32, i32]
         L.peqa_selftest_configure.restype = ctypes.c_int
         L.peqa_probe_read.argtypes = [vp, sz, vp, sz, vp]
@@ -156,6 +164,21 @@ def quantize_rtn(W: torch.Tensor, bits: int, group_size: int = 0, out: QWeight |
     _check(lib().peqa_quantize_rtn(W.data_ptr(), N, K, bits, group_size, q.data_ptr(), z.data_ptr(),
                                    s.data_ptr(), _stream()), "peqa_quantize_rtn")
     return out if out is not None else QWeight(bits, N, K, group_size, q, z, s)
+
+
+def quantize_search(W: torch.Tensor, bits: int, group_size: int = 0, n_candidates: int = 32):
+    """Quantize W with the clipping range searched per group; returns (QWeight, chosen u8 [N,G])."""
+    _dev(W, torch.float32, "W")
+    N, K = W.shape
+    G = 1 if group_size in (0, K) else max(K // max(group_size, 1), 1)
+    q = torch.empty((N, max(K * bits // 32, 1)), dtype=torch.int32, device=W.device)
+    z = torch.empty((N, G), dtype=torch.uint8, device=W.device)
+    s = torch.empty((N, G), dtype=torch.float32, device=W.device)
+    chosen = torch.empty((N, G), dtype=torch.uint8, device=W.device)
+    _check(lib().peqa_quantize_search(W.data_ptr(), N, K, bits, group_size, n_candidates, q.data_ptr(),
+                                      z.data_ptr(), s.data_ptr(), chosen.data_ptr(), _stream()),
+           "peqa_quantize_search")
+    return QWeight(bits, N, K, group_size, q, z, s), chosen
 
 
 def pack(codes: torch.Tensor, bits: int) -> torch.Tensor:
@@ -398,6 +421,45 @@ def probe_read(buf: torch.Tensor, sink: torch.Tensor) -> None:
     """Read-only pass over ``buf`` (measurement aid); sink: int32 device tensor, one word per SM."""
     _check(lib().peqa_probe_read(buf.data_ptr(), buf.numel() * buf.element_size(), sink.data_ptr(),
                                  sink.numel() * sink.element_size(), _stream()), "peqa_probe_read")
+
+
+def qlinear_fwd_zf(w: QWeight, zeros_f: torch.Tensor, X: torch.Tensor, Y=None):
+    """Forward with real-valued zero-points zeros_f fp32 [N, G] (App. K)."""
+    _dev(zeros_f, torch.float32, "zeros_f")
+    _dev(X, torch.bfloat16, "X")
+    T = X.shape[0]
+    if Y is None:
+        Y = torch.empty((T, w.N), dtype=torch.bfloat16, device=X.device)
+    cs = w.c_struct()
+    _check(lib().peqa_qlinear_fwd_zf(ctypes.byref(cs), zeros_f.data_ptr(), X.data_ptr(), T, Y.data_ptr(),
+                                     _stream()), "peqa_qlinear_fwd_zf")
+    return Y
+
+
+def qlinear_bwd_zf(w: QWeight, zeros_f: torch.Tensor, X, dY: torch.Tensor, need_dx=True, need_grads=True,
+                   workspace=None):
+    """dX and/or (dS, dZ) with real-valued zero-points; returns (dX, dS, dZ)."""
+    _dev(zeros_f, torch.float32, "zeros_f")
+    _dev(dY, torch.bfloat16, "dY")
+    T = dY.shape[0]
+    dX = torch.empty((T, w.K), dtype=torch.bfloat16, device=dY.device) if need_dx else None
+    dS = torch.empty((w.N, w.G), dtype=torch.float32, device=dY.device) if need_grads else None
+    dZ = torch.empty((w.N, w.G), dtype=torch.float32, device=dY.device) if need_grads else None
+    if need_grads and workspace is None:
+        workspace = alloc_workspace(OP_BWD_DSDZ, T, w)
+    cs = w.c_struct()
+    wp, wb = _ws(workspace)
+    _check(lib().peqa_qlinear_bwd_zf(ctypes.byref(cs), zeros_f.data_ptr(), _ptr(X), dY.data_ptr(), T,
+                                     _ptr(dX), _ptr(dS), _ptr(dZ), wp, wb, _stream()), "peqa_qlinear_bwd_zf")
+    return dX, dS, dZ
+
+
+def zero_adamw(zeros_f, dZ, m, v, lr, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.0, step=1):
+    for t, n in ((zeros_f, "zeros_f"), (dZ, "dZ"), (m, "m"), (v, "v")):
+        _dev(t, torch.float32, n)
+    _check(lib().peqa_zero_adamw(zeros_f.data_ptr(), dZ.data_ptr(), m.data_ptr(), v.data_ptr(),
+                                 zeros_f.numel(), lr, beta1, beta2, eps, weight_decay, step, _stream()),
+           "peqa_zero_adamw")
 
 
 def selftest_configure(wait_limit_us: int = 0, starve_forward: bool = False) -> None:

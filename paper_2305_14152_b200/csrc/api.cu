@@ -121,9 +121,9 @@ int sm_count_or(int fallback) {
   return cached_sms;
 }
 
-int check_qweight(const peqa_qweight_t* w, int* g, int* G) {
+int check_qweight(const peqa_qweight_t* w, int* g, int* G, bool zeros_optional) {
   if (!w) return PEQA_ERR_NULL;
-  if (!w->qweight || !w->zeros || !w->scales) return PEQA_ERR_NULL;
+  if (!w->qweight || (!w->zeros && !zeros_optional) || !w->scales) return PEQA_ERR_NULL;
   PEQA_TRY(check_bits_shape(w->out_features, w->in_features, w->bits, w->group_size));
   if (!aligned16(w->qweight) || !aligned16(w->scales)) return PEQA_ERR_ALIGNMENT;
   *g = effective_group(w->in_features, w->group_size);
@@ -168,7 +168,7 @@ extern "C" int peqa_qlinear_fwd(const peqa_qweight_t* w, const void* X, int T, v
   PEQA_TRY(check_gemm_shape(w, T));
   if (!aligned16(X) || !aligned16(Y)) return PEQA_ERR_ALIGNMENT;
   PEQA_TRY(check_arch());
-  return launch_fwd(w, g, X, T, Y, as_stream(stream));
+  return launch_fwd(w, nullptr, g, X, T, Y, as_stream(stream));
 }
 
 extern "C" int peqa_qlinear_bwd(const peqa_qweight_t* w, const void* X, const void* dY, int T,
@@ -189,8 +189,8 @@ extern "C" int peqa_qlinear_bwd(const peqa_qweight_t* w, const void* X, const vo
       if (reinterpret_cast<uintptr_t>(workspace) & 255u) return PEQA_ERR_ALIGNMENT;
     }
   }
-  if (dX) PEQA_TRY(launch_dx(w, g, dY, T, dX, as_stream(stream)));
-  if (dS) PEQA_TRY(launch_ds(w, g, X, dY, T, dS, nullptr, nullptr, workspace, workspace_bytes, as_stream(stream)));
+  if (dX) PEQA_TRY(launch_dx(w, nullptr, g, dY, T, dX, as_stream(stream)));
+  if (dS) PEQA_TRY(launch_ds(w, nullptr, g, X, dY, T, dS, nullptr, nullptr, workspace, workspace_bytes, as_stream(stream)));
   return PEQA_OK;
 }
 
@@ -216,7 +216,7 @@ extern "C" int peqa_qlinear_bwd_ds_adamw(const peqa_qweight_t* w, const void* X,
   adam.scales = const_cast<float*>(w->scales);
   adam.m = m;
   adam.v = v;
-  return launch_ds(w, g, X, dY, T, dS, nullptr, &adam, workspace, workspace_bytes, as_stream(stream));
+  return launch_ds(w, nullptr, g, X, dY, T, dS, nullptr, &adam, workspace, workspace_bytes, as_stream(stream));
 }
 
 extern "C" int peqa_qlinear_bwd_dsdz(const peqa_qweight_t* w, const void* X, const void* dY, int T,
@@ -233,7 +233,7 @@ extern "C" int peqa_qlinear_bwd_dsdz(const peqa_qweight_t* w, const void* X, con
     if (!workspace || workspace_bytes < need) return PEQA_ERR_WORKSPACE;
     if (reinterpret_cast<uintptr_t>(workspace) & 255u) return PEQA_ERR_ALIGNMENT;
   }
-  return launch_ds(w, g, X, dY, T, dS, dZ, nullptr, workspace, workspace_bytes, as_stream(stream));
+  return launch_ds(w, nullptr, g, X, dY, T, dS, dZ, nullptr, workspace, workspace_bytes, as_stream(stream));
 }
 
 extern "C" int peqa_qlinear_bwd_ds_from_y(const peqa_qweight_t* w, const void* dY, const void* Y,
@@ -250,6 +250,42 @@ extern "C" int peqa_qlinear_bwd_ds_from_y(const peqa_qweight_t* w, const void* d
   if (!workspace || workspace_bytes < need) return PEQA_ERR_WORKSPACE;
   if (reinterpret_cast<uintptr_t>(workspace) & 255u) return PEQA_ERR_ALIGNMENT;
   return launch_ds_from_y(w, dY, Y, T, dS, workspace, as_stream(stream));
+}
+
+extern "C" int peqa_qlinear_fwd_zf(const peqa_qweight_t* w, const float* zeros_f, const void* X,
+                                   int T, void* Y, void* stream) {
+  int g = 0, G = 0;
+  PEQA_TRY(check_qweight(w, &g, &G, true));
+  if (!zeros_f || !X || !Y) return PEQA_ERR_NULL;
+  PEQA_TRY(check_gemm_shape(w, T));
+  if (!aligned16(X) || !aligned16(Y)) return PEQA_ERR_ALIGNMENT;
+  PEQA_TRY(check_arch());
+  return launch_fwd(w, zeros_f, g, X, T, Y, as_stream(stream));
+}
+
+extern "C" int peqa_qlinear_bwd_zf(const peqa_qweight_t* w, const float* zeros_f, const void* X,
+                                   const void* dY, int T, void* dX, float* dS, float* dZ,
+                                   void* workspace, size_t workspace_bytes, void* stream) {
+  int g = 0, G = 0;
+  PEQA_TRY(check_qweight(w, &g, &G, true));
+  if (!zeros_f || !dY) return PEQA_ERR_NULL;
+  if ((dS == nullptr) != (dZ == nullptr)) return PEQA_ERR_NULL;   // both gradients or neither
+  if (dS && !X) return PEQA_ERR_NULL;
+  PEQA_TRY(check_gemm_shape(w, T));
+  if (!aligned16(dY) || (X && !aligned16(X)) || (dX && !aligned16(dX)) || (dS && !aligned16(dS)) ||
+      (dZ && !aligned16(dZ)))
+    return PEQA_ERR_ALIGNMENT;
+  PEQA_TRY(check_arch());
+  if (dS) {
+    const size_t need = dsdz_workspace_bytes(w, g, T);
+    if (need > 0) {
+      if (!workspace || workspace_bytes < need) return PEQA_ERR_WORKSPACE;
+      if (reinterpret_cast<uintptr_t>(workspace) & 255u) return PEQA_ERR_ALIGNMENT;
+    }
+  }
+  if (dX) PEQA_TRY(launch_dx(w, zeros_f, g, dY, T, dX, as_stream(stream)));
+  if (dS) PEQA_TRY(launch_ds(w, zeros_f, g, X, dY, T, dS, dZ, nullptr, workspace, workspace_bytes, as_stream(stream)));
+  return PEQA_OK;
 }
 
 extern "C" int peqa_qlinear_decode(const peqa_qweight_t* w, const void* X, int M, void* Y,

@@ -46,8 +46,9 @@ inline int check_bits_shape(int N, int K, int bits, int group_size) {
   return PEQA_OK;
 }
 
-// Validates a layer descriptor; fills g (effective group) and G.
-int check_qweight(const peqa_qweight_t* w, int* g, int* G);
+// Validates a layer descriptor; fills g (effective group) and G.  With zeros_optional the
+// integer zero-points may be absent (entry points that take real-valued ones).
+int check_qweight(const peqa_qweight_t* w, int* g, int* G, bool zeros_optional = false);
 
 // The current device must be compute capability 10.x (cached per device).
 int check_arch();
@@ -105,12 +106,17 @@ __device__ __forceinline__ void adamw_update(float& s, float gr, float& m, float
 #endif
 
 // Entry points implemented in the individual translation units.
-int launch_fwd(const peqa_qweight_t* w, int g, const void* X, int T, void* Y, cudaStream_t st);
+// zeros_f != nullptr: real-valued zero-points [N, G] (App. K) replace w->zeros
+int launch_fwd(const peqa_qweight_t* w, const float* zeros_f, int g, const void* X, int T, void* Y,
+               cudaStream_t st);
 bool fwd_pair_supported(const peqa_qweight_t* w);
-int launch_fwd_pair(const peqa_qweight_t* w, int g, const void* X, int T, void* Y, cudaStream_t st);
+int launch_fwd_pair(const peqa_qweight_t* w, const float* zeros_f, int g, const void* X, int T,
+                    void* Y, cudaStream_t st);
 bool dx_pair_supported(const peqa_qweight_t* w);
-int launch_dx_pair(const peqa_qweight_t* w, int g, const void* dY, int T, void* dX, cudaStream_t st);
-int launch_dx(const peqa_qweight_t* w, int g, const void* dY, int T, void* dX, cudaStream_t st);
+int launch_dx_pair(const peqa_qweight_t* w, const float* zeros_f, int g, const void* dY, int T,
+                   void* dX, cudaStream_t st);
+int launch_dx(const peqa_qweight_t* w, const float* zeros_f, int g, const void* dY, int T, void* dX,
+              cudaStream_t st);
 // adam != nullptr: the AdamW step on (w->scales, m, v) is applied where dS is produced
 struct DsAdam {
   AdamWConsts c;
@@ -118,8 +124,10 @@ struct DsAdam {
   float* m;
   float* v;
 };
-int launch_ds(const peqa_qweight_t* w, int g, const void* X, const void* dY, int T, float* dS,
-              float* dZ, const DsAdam* adam, void* workspace, size_t workspace_bytes, cudaStream_t st);
+// zeros_f != nullptr needs dZ: dS is then taken with the real-valued zero-point
+int launch_ds(const peqa_qweight_t* w, const float* zeros_f, int g, const void* X, const void* dY,
+              int T, float* dS, float* dZ, const DsAdam* adam, void* workspace,
+              size_t workspace_bytes, cudaStream_t st);
 size_t dsdz_workspace_bytes(const peqa_qweight_t* w, int g, int T);
 size_t ds_workspace_bytes(const peqa_qweight_t* w, int g, int T);
 size_t ds_from_y_workspace_bytes(const peqa_qweight_t* w, int T);

@@ -40,6 +40,14 @@ __device__ __forceinline__ uint32_t bf162_mul(uint32_t a, uint32_t b) {
   return *reinterpret_cast<uint32_t*>(&r);
 }
 
+__device__ __forceinline__ uint32_t bf162_fma(uint32_t a, uint32_t b, uint32_t c) {
+  __nv_bfloat162 x = *reinterpret_cast<__nv_bfloat162*>(&a);
+  __nv_bfloat162 y = *reinterpret_cast<__nv_bfloat162*>(&b);
+  __nv_bfloat162 z = *reinterpret_cast<__nv_bfloat162*>(&c);
+  __nv_bfloat162 r = __hfma2(x, y, z);
+  return *reinterpret_cast<uint32_t*>(&r);
+}
+
 __device__ __forceinline__ uint32_t bf162_broadcast(float s) {
   __nv_bfloat162 r = __float2bfloat162_rn(s);
   return *reinterpret_cast<uint32_t*>(&r);
@@ -122,6 +130,46 @@ __device__ __forceinline__ void unit32_natural(const uint32_t (&w)[BITS], uint32
   block8_natural<BITS, 1, FOLD>(w, zc, s2, out + 4);
   block8_natural<BITS, 2, FOLD>(w, zc, s2, out + 8);
   block8_natural<BITS, 3, FOLD>(w, zc, s2, out + 12);
+}
+
+// A unit of 32 columns with a real-valued zero-point z = zi + delta (App. K trains z):
+//   s*(q - z) = (q - zi)*s + c,  c = -delta*s,
+// formed as one fused multiply-add per pair on the exact integers q - zi, so the operand is
+// the product rounded once (with s and c rounded to bf16 first, as for grouped scales).
+// zi must be an integer in [0, 2^BITS - 1].
+template <int BITS>
+__device__ __forceinline__ void unit32_affine(const uint32_t (&w)[BITS], uint32_t zi, float s, float c,
+                                              uint32_t (&out)[16]) {
+  const uint32_t zc = zero_const<BITS>(zi);
+  const uint32_t s2 = bf162_broadcast(s), c2 = bf162_broadcast(c);
+#pragma unroll
+  for (int blk = 0; blk < 4; ++blk) {
+    uint32_t d[4];
+    if (blk == 0) {
+      d[0] = pair_raw<BITS, 0>(w); d[1] = pair_raw<BITS, 1>(w); d[2] = pair_raw<BITS, 2>(w); d[3] = pair_raw<BITS, 3>(w);
+    } else if (blk == 1) {
+      d[0] = pair_raw<BITS, 8>(w); d[1] = pair_raw<BITS, 9>(w); d[2] = pair_raw<BITS, 10>(w); d[3] = pair_raw<BITS, 11>(w);
+    } else if (blk == 2) {
+      d[0] = pair_raw<BITS, 16>(w); d[1] = pair_raw<BITS, 17>(w); d[2] = pair_raw<BITS, 18>(w); d[3] = pair_raw<BITS, 19>(w);
+    } else {
+      d[0] = pair_raw<BITS, 24>(w); d[1] = pair_raw<BITS, 25>(w); d[2] = pair_raw<BITS, 26>(w); d[3] = pair_raw<BITS, 27>(w);
+    }
+#pragma unroll
+    for (int e = 0; e < 4; ++e) d[e] = bf162_fma(bf162_sub(d[e], zc), s2, c2);
+    out[4 * blk + 0] = prmt(d[0], d[1], 0x5410u);
+    out[4 * blk + 1] = prmt(d[2], d[3], 0x5410u);
+    out[4 * blk + 2] = prmt(d[0], d[1], 0x7632u);
+    out[4 * blk + 3] = prmt(d[2], d[3], 0x7632u);
+  }
+}
+
+// Splits a real-valued zero-point into the integer the exact dequantization can use and
+// the remainder the affine form carries: zi = clamp(rint(z), 0, 2^BITS - 1), delta = z - zi.
+template <int BITS>
+__device__ __forceinline__ void split_zero_point(float z, uint32_t& zi, float& delta) {
+  const float r = fminf(fmaxf(rintf(z), 0.0f), (float)((1 << BITS) - 1));
+  zi = (uint32_t)r;
+  delta = z - r;
 }
 
 // ---------------------------------------------------------------------------

@@ -61,6 +61,7 @@ struct DxBarriers {
 
 struct DxParams {
   const uint8_t* zeros;
+  const float* zeros_f;   // real-valued zero-points (App. K) or nullptr; replaces `zeros`
   const float* scales;
   __nv_bfloat16* out;   // dX [T, K]
   int N, K, G, g, g_shift, T;
@@ -73,7 +74,7 @@ __device__ __forceinline__ int dx_group_of(const DxParams& p, int col) {
   return p.g_shift >= 0 ? (col >> p.g_shift) : (col / p.g);
 }
 
-template <int BITS>
+template <int BITS, bool ZF>
 __global__ void __launch_bounds__(kDxThreads, 1)
 qdx_pair_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_constant__ CUtensorMap tmap_q,
                 const DxParams p) {
@@ -246,16 +247,24 @@ qdx_pair_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_consta
     int pf_tile = pair, pf_kb = grp;
     while (pf_kb >= p.k_blocks) { pf_kb -= p.k_blocks; pf_tile += n_pairs; }
     int pf_col = (pf_tile % p.j_tiles) * 256 + (int)rank * 128 + 32 * u4;
-    auto load_zs = [&](uint32_t (&z)[2], float (&sc)[2]) {
+    // cz: the constant term -delta * s of a real-valued zero-point (ZF), else unused
+    auto load_zs = [&](uint32_t (&z)[2], float (&sc)[2], float (&cz)[2]) {
 #pragma unroll
       for (int k = 0; k < 2; ++k) {
         const int i = pf_kb * XK + (k ? row_b : row_a);
         z[k] = 0u;
         sc[k] = 0.0f;
+        cz[k] = 0.0f;
         if (i < p.N && pf_col < p.K) {
           const size_t gi = (size_t)i * p.G + dx_group_of(p, pf_col);
-          z[k] = __ldg(p.zeros + gi);
           sc[k] = __ldg(p.scales + gi);
+          if (ZF) {
+            float delta;
+            dq::split_zero_point<BITS>(__ldg(p.zeros_f + gi), z[k], delta);
+            cz[k] = -delta * sc[k];
+          } else {
+            z[k] = __ldg(p.zeros + gi);
+          }
         }
       }
       pf_kb += X_GROUPS;
@@ -266,10 +275,10 @@ qdx_pair_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_consta
       }
     };
     uint32_t z[2], zn[2];
-    float sc[2], scn[2];
-    if ((uint32_t)grp < total_it) load_zs(z, sc);
+    float sc[2], scn[2], cz[2], czn[2];
+    if ((uint32_t)grp < total_it) load_zs(z, sc, cz);
     for (uint32_t it = grp; it < total_it; it += X_GROUPS) {
-      if (it + X_GROUPS < total_it) load_zs(zn, scn);
+      if (it + X_GROUPS < total_it) load_zs(zn, scn, czn);
       const int s = it % XSTAGES;
       const int q = it % XQ_SLOTS;
       if (!mbar_wait(smem_u32(&bars->pk_full[q]), (it / XQ_SLOTS) & 1u, abort_flag)) break;
@@ -291,8 +300,13 @@ qdx_pair_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_consta
         }
       }
       uint32_t oa[16], ob[16];
-      dq::unit32_natural<BITS, true>(wa, z[0], sc[0], oa);
-      dq::unit32_natural<BITS, true>(wb, z[1], sc[1], ob);
+      if constexpr (ZF) {
+        dq::unit32_affine<BITS>(wa, z[0], sc[0], cz[0], oa);
+        dq::unit32_affine<BITS>(wb, z[1], sc[1], cz[1], ob);
+      } else {
+        dq::unit32_natural<BITS, true>(wa, z[0], sc[0], oa);
+        dq::unit32_natural<BITS, true>(wb, z[1], sc[1], ob);
+      }
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&bars->pk_empty[q]));   // codes consumed: slot free
       if (!mbar_wait_cluster(smem_u32(&bars->empty[s]), ((it / XSTAGES) & 1u) ^ 1u, abort_flag)) break;
@@ -310,6 +324,7 @@ qdx_pair_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_consta
       if (lane == 0) mbar_arrive_cluster_release(full_w_leader0 + s * 8);
       z[0] = zn[0]; z[1] = zn[1];
       sc[0] = scn[0]; sc[1] = scn[1];
+      cz[0] = czn[0]; cz[1] = czn[1];
     }
   }
 
@@ -330,10 +345,10 @@ qdx_pair_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_consta
   }
 }
 
-template <int BITS>
+template <int BITS, bool ZF>
 int launch_dx_pair_t(const CUtensorMap& ta, const CUtensorMap& tq, const DxParams& p, int pairs,
                      cudaStream_t st) {
-  auto kern = qdx_pair_kernel<BITS>;
+  auto kern = qdx_pair_kernel<BITS, ZF>;
   PEQA_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, X_SMEM_BYTES));
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(2 * pairs, 1, 1);
@@ -358,9 +373,11 @@ bool dx_pair_supported(const peqa_qweight_t* w) {
   return ((size_t)w->in_features * w->bits / 8) % 16 == 0;
 }
 
-int launch_dx_pair(const peqa_qweight_t* w, int g, const void* dY, int T, void* dX, cudaStream_t st) {
+int launch_dx_pair(const peqa_qweight_t* w, const float* zeros_f, int g, const void* dY, int T,
+                   void* dX, cudaStream_t st) {
   DxParams p;
   p.zeros = w->zeros;
+  p.zeros_f = zeros_f;
   p.scales = w->scales;
   p.out = static_cast<__nv_bfloat16*>(dX);
   p.N = w->out_features;
@@ -405,7 +422,11 @@ int launch_dx_pair(const peqa_qweight_t* w, int g, const void* dY, int T, void* 
   const int tiles = p.j_tiles * p.t_tiles;
   const int max_pairs = sms / 2;
   const int pairs = tiles < max_pairs ? tiles : max_pairs;
-  return w->bits == 4 ? launch_dx_pair_t<4>(ta, tq, p, pairs, st) : launch_dx_pair_t<3>(ta, tq, p, pairs, st);
+  if (zeros_f)
+    return w->bits == 4 ? launch_dx_pair_t<4, true>(ta, tq, p, pairs, st)
+                        : launch_dx_pair_t<3, true>(ta, tq, p, pairs, st);
+  return w->bits == 4 ? launch_dx_pair_t<4, false>(ta, tq, p, pairs, st)
+                      : launch_dx_pair_t<3, false>(ta, tq, p, pairs, st);
 }
 
 }  // namespace peqa

@@ -448,3 +448,11 @@ extern "C" int peqa_scale_adamw(float* scales, const float* dS, float* m, float*
   PEQA_CUDA(cudaGetLastError());
   return PEQA_OK;
 }
+
+// App. K's "zero-points only" and "both" modes: the same AdamW step on the real-valued
+// zero-points, driven by dZ.
+extern "C" int peqa_zero_adamw(float* zeros_f, const float* dZ, float* m, float* v, int64_t numel,
+                               float lr, float beta1, float beta2, float eps, float weight_decay,
+                               int64_t step, void* stream) {
+  return peqa_scale_adamw(zeros_f, dZ, m, v, numel, lr, beta1, beta2, eps, weight_decay, step, stream);
+}

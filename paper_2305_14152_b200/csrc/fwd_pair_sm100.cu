@@ -64,6 +64,7 @@ struct PairBarriers {
 
 struct PairParams {
   const uint8_t* zeros;
+  const float* zeros_f;   // real-valued zero-points (App. K) or nullptr; replaces `zeros`
   const float* scales;
   __nv_bfloat16* out;   // Y [T, N]
   int N, K, G, g, g_shift, T;
@@ -76,7 +77,7 @@ __device__ __forceinline__ int pair_group_of(const PairParams& p, int col) {
   return p.g_shift >= 0 ? (col >> p.g_shift) : (col / p.g);
 }
 
-template <int BITS, bool FOLD>
+template <int BITS, bool FOLD, bool ZF>
 __global__ void __launch_bounds__(kPairThreads, 1)
 qfwd_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_q,
                  const PairParams p) {
@@ -273,13 +274,27 @@ qfwd_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     // channel), and one 2-byte / 8-byte load when the groups are 32 columns wide
     const bool one_group = p.G == 1 || (p.g & 63) == 0;
     const bool pair_load = !one_group && p.g == 32 && (p.G & 1) == 0;
-    auto load_zs = [&](uint32_t (&z)[2], float (&sc)[2]) {
+    // cz: the constant term -delta * s of a real-valued zero-point (ZF), else unused
+    auto load_zs = [&](uint32_t (&z)[2], float (&sc)[2], float (&cz)[2]) {
       z[0] = z[1] = 0u;
       sc[0] = sc[1] = 0.0f;
+      cz[0] = cz[1] = 0.0f;
       const int col = pf_kb * PK;
       if (pf_r < p.N && col < p.K) {
         const size_t gi = (size_t)pf_r * p.G + pair_group_of(p, col);
-        if (one_group) {
+        if (ZF) {
+          float delta;
+          sc[0] = __ldg(p.scales + gi);
+          dq::split_zero_point<BITS>(__ldg(p.zeros_f + gi), z[0], delta);
+          cz[0] = -delta * sc[0];
+          z[1] = z[0]; sc[1] = sc[0]; cz[1] = cz[0];
+          if (!one_group && col + 32 < p.K) {
+            const size_t g1 = (size_t)pf_r * p.G + pair_group_of(p, col + 32);
+            sc[1] = __ldg(p.scales + g1);
+            dq::split_zero_point<BITS>(__ldg(p.zeros_f + g1), z[1], delta);
+            cz[1] = -delta * sc[1];
+          }
+        } else if (one_group) {
           z[0] = z[1] = __ldg(p.zeros + gi);
           if (FOLD) sc[0] = sc[1] = __ldg(p.scales + gi);
         } else if (pair_load) {
@@ -309,12 +324,12 @@ qfwd_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
       }
     };
     uint32_t z[2], zn[2];
-    float sc[2], scn[2];
+    float sc[2], scn[2], cz[2], czn[2];
     int cur_kb = pf_kb;
-    if ((uint32_t)grp < total_it) load_zs(z, sc);
+    if ((uint32_t)grp < total_it) load_zs(z, sc, cz);
     for (uint32_t it = grp; it < total_it; it += P_GROUPS) {
       const int next_kb = pf_kb;
-      if (it + P_GROUPS < total_it) load_zs(zn, scn);
+      if (it + P_GROUPS < total_it) load_zs(zn, scn, czn);
       const int s = it % PSTAGES;
       const int q = it % PQ_SLOTS;
       if (!mbar_wait(smem_u32(&bars->pk_full[q]), (it / PQ_SLOTS) & 1u, abort_flag)) break;
@@ -337,8 +352,13 @@ qfwd_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         }
       }
       uint32_t o0[16], o1[16];
-      dq::unit32_natural<BITS, FOLD>(w[0], z[0], sc[0], o0);
-      dq::unit32_natural<BITS, FOLD>(w[1], z[1], sc[1], o1);
+      if constexpr (ZF) {
+        dq::unit32_affine<BITS>(w[0], z[0], sc[0], cz[0], o0);
+        dq::unit32_affine<BITS>(w[1], z[1], sc[1], cz[1], o1);
+      } else {
+        dq::unit32_natural<BITS, FOLD>(w[0], z[0], sc[0], o0);
+        dq::unit32_natural<BITS, FOLD>(w[1], z[1], sc[1], o1);
+      }
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&bars->pk_empty[q]));   // codes consumed: slot free
       if (!mbar_wait_cluster(smem_u32(&bars->empty[s]), ((it / PSTAGES) & 1u) ^ 1u, abort_flag)) break;
@@ -356,6 +376,7 @@ qfwd_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
       if (lane == 0) mbar_arrive_cluster_release(full_w_leader0 + s * 8);
       z[0] = zn[0]; z[1] = zn[1];
       sc[0] = scn[0]; sc[1] = scn[1];
+      cz[0] = czn[0]; cz[1] = czn[1];
       cur_kb = next_kb;
     }
   }
@@ -377,10 +398,10 @@ qfwd_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
   }
 }
 
-template <int BITS, bool FOLD>
+template <int BITS, bool FOLD, bool ZF>
 int launch_pair_t(const CUtensorMap& tx, const CUtensorMap& tq, const PairParams& p, int pairs,
                   cudaStream_t st) {
-  auto kern = qfwd_pair_kernel<BITS, FOLD>;
+  auto kern = qfwd_pair_kernel<BITS, FOLD, ZF>;
   PEQA_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM_BYTES));
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(2 * pairs, 1, 1);
@@ -407,9 +428,11 @@ bool fwd_pair_supported(const peqa_qweight_t* w) {
   return ((size_t)w->in_features * w->bits / 8) % 16 == 0;
 }
 
-int launch_fwd_pair(const peqa_qweight_t* w, int g, const void* X, int T, void* Y, cudaStream_t st) {
+int launch_fwd_pair(const peqa_qweight_t* w, const float* zeros_f, int g, const void* X, int T,
+                    void* Y, cudaStream_t st) {
   PairParams p;
   p.zeros = w->zeros;
+  p.zeros_f = zeros_f;
   p.scales = w->scales;
   p.out = static_cast<__nv_bfloat16*>(Y);
   p.N = w->out_features;
@@ -455,9 +478,14 @@ int launch_fwd_pair(const peqa_qweight_t* w, int g, const void* X, int T, void* 
   const int max_pairs = sms / 2;
   const int pairs = tiles < max_pairs ? tiles : max_pairs;
   const bool fold = p.G > 1;
+  if (zeros_f)   // a real-valued zero-point is folded into the operand whatever the group size
+    return w->bits == 4 ? launch_pair_t<4, true, true>(tx, tq, p, pairs, st)
+                        : launch_pair_t<3, true, true>(tx, tq, p, pairs, st);
   if (w->bits == 4)
-    return fold ? launch_pair_t<4, true>(tx, tq, p, pairs, st) : launch_pair_t<4, false>(tx, tq, p, pairs, st);
-  return fold ? launch_pair_t<3, true>(tx, tq, p, pairs, st) : launch_pair_t<3, false>(tx, tq, p, pairs, st);
+    return fold ? launch_pair_t<4, true, false>(tx, tq, p, pairs, st)
+                : launch_pair_t<4, false, false>(tx, tq, p, pairs, st);
+  return fold ? launch_pair_t<3, true, false>(tx, tq, p, pairs, st)
+              : launch_pair_t<3, false, false>(tx, tq, p, pairs, st);
 }
 
 }  // namespace peqa

@@ -101,6 +101,7 @@ __device__ __forceinline__ void drain_after_abort() {
 struct QGemmParams {
   const uint32_t* qw;
   const uint8_t* zeros;
+  const float* zeros_f;   // real-valued zero-points (App. K) or nullptr; replaces `zeros`
   const float* scales;
   __nv_bfloat16* out;   // [T, R]
   int N, K, G, g, T;
@@ -117,6 +118,7 @@ struct Unit {
   uint32_t w[BITS];
   uint32_t z;
   float s;
+  float c;   // -delta * s of a real-valued zero-point z + delta (App. K), else 0
 };
 
 __device__ __forceinline__ int group_of(const QGemmParams& p, int col) {
@@ -142,29 +144,30 @@ __device__ __forceinline__ Unit<BITS> load_unit(const QGemmParams& p, int i, int
       }
     }
     const size_t gidx = (size_t)i * p.G + group_of(p, col0);
-    u.z = __ldg(p.zeros + gidx);
     u.s = __ldg(p.scales + gidx);
+    u.c = 0.0f;
+    if (p.zeros_f) {
+      float delta;
+      dq::split_zero_point<BITS>(__ldg(p.zeros_f + gidx), u.z, delta);
+      u.c = -delta * u.s;
+    } else {
+      u.z = __ldg(p.zeros + gidx);
+    }
   } else {
     // Outside the matrix: codes equal to the zero-point dequantise to exactly 0.
     u.z = 0u;
     u.s = 0.0f;
+    u.c = 0.0f;
   }
   return u;
 }
 
-// Dequantise one unit and store its 64 bytes (four 16-byte chunks starting at
-// chunk0) into a 128-byte tile row; the chunk index is XORed with (row & 7)
-// as the 128-byte swizzle requires.
+// (q - z) [* bf16(s)] of one unit; with a real-valued zero-point (zf, uniform over the
+// launch, only with FOLD) the affine form (q - zi) * s + c.
 template <int BITS, bool FOLD>
-__device__ __forceinline__ void store_unit(const Unit<BITS>& u, uint8_t* row_ptr, int chunk0,
-                                           int swz) {
-  uint32_t o[16];
-  dq::unit32_natural<BITS, FOLD>(u.w, u.z, u.s, o);
-#pragma unroll
-  for (int q = 0; q < 4; ++q) {
-    *reinterpret_cast<uint4*>(row_ptr + (((chunk0 + q) ^ swz) << 4)) =
-        make_uint4(o[4 * q], o[4 * q + 1], o[4 * q + 2], o[4 * q + 3]);
-  }
+__device__ __forceinline__ void dequant_unit(const Unit<BITS>& u, bool zf, uint32_t (&o)[16]) {
+  if (FOLD && zf) dq::unit32_affine<BITS>(u.w, u.z, u.s, u.c, o);
+  else dq::unit32_natural<BITS, FOLD>(u.w, u.z, u.s, o);
 }
 
 // PKTMA: the packed codes of a stage arrive by TMA in shared memory (needs a
@@ -416,7 +419,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmap_act,
       }
       uint32_t o[UPT][16];
 #pragma unroll
-      for (int k = 0; k < UPT; ++k) dq::unit32_natural<BITS, FOLD>(cur[k].w, cur[k].z, cur[k].s, o[k]);
+      for (int k = 0; k < UPT; ++k) dequant_unit<BITS, FOLD>(cur[k], p.zeros_f != nullptr, o[k]);
       if (PKTMA) {
         // every lane has consumed its codes by now: hand the slot back
         __syncwarp();
@@ -457,6 +460,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmap_act,
 struct DsParams {
   const uint32_t* qw;
   const uint8_t* zeros;
+  const float* zeros_f;   // real-valued zero-points (App. K) or nullptr; only with DZ
   float* out;        // [N, K / piece]: dS itself when piece == g, else partial sums
   float* out_z;      // same shape: dZ (or its partial sums of dW); only read by ds_kernel<.., true>
   const float* scales;
@@ -614,6 +618,7 @@ ds_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_constant__ C
         const bool row_ok = i < p.N;
         uint32_t w[BITS];
         uint32_t z = 0u;
+        float delta = 0.0f;   // real-valued zero-point = z + delta
 #pragma unroll
         for (int q = 0; q < BITS; ++q) w[q] = 0u;
         if (row_ok) {
@@ -624,7 +629,8 @@ ds_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_constant__ C
           } else {
             w[0] = __ldg(src); w[1] = __ldg(src + 1); w[2] = __ldg(src + 2);
           }
-          z = __ldg(p.zeros + (size_t)i * p.G + col0 / p.g);
+          if (DZ && p.zeros_f) dq::split_zero_point<BITS>(__ldg(p.zeros_f + (size_t)i * p.G + col0 / p.g), z, delta);
+          else z = __ldg(p.zeros + (size_t)i * p.G + col0 / p.g);
         }
         uint32_t o[16];
         dq::unit32_natural<BITS, false>(w, z, 0.0f, o);
@@ -637,6 +643,9 @@ ds_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_constant__ C
         }
         if (((cc + 1) % chunks_per_piece) == 0) {
           if (row_ok) {
+            // with a real-valued zero-point, sum (q - z) dW = sum (q - zi) dW - delta * sum dW;
+            // partial pieces are stored raw and corrected after they have been added
+            if (DZ && p.zeros_f && p.piece == p.g) acc = fmaf(-delta, accz, acc);
             p.out[(size_t)i * npieces + col0 / p.piece] = acc;
             if (ADAM) {
               // pieces are whole groups here (the launcher only asks for this then): acc is
@@ -677,6 +686,27 @@ ds_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_constant__ C
     atomicExch(p.status, (int)PEQA_ERR_DEVICE_TIMEOUT);
     p.status[1] = (int)blockIdx.x;
   }
+}
+
+// Real-valued zero-point, groups wider than a piece: dS = sum(pieces) - delta * sum(dW pieces)
+// and dZ = -s * sum(dW pieces), pieces added in index order.
+__global__ void ds_reduce_zf_kernel(const float* __restrict__ partial_s, const float* __restrict__ partial_w,
+                                    float* __restrict__ dS, float* __restrict__ dZ, long long n_out,
+                                    int pieces_per_group, const float* __restrict__ zeros_f,
+                                    const float* __restrict__ scales, int bits) {
+  long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= n_out) return;
+  float acc_s = 0.0f, acc_w = 0.0f;
+  for (int q = 0; q < pieces_per_group; ++q) {
+    acc_s += partial_s[e * pieces_per_group + q];
+    acc_w += partial_w[e * pieces_per_group + q];
+  }
+  uint32_t zi;
+  float delta;
+  if (bits == 3) dq::split_zero_point<3>(zeros_f[e], zi, delta);
+  else dq::split_zero_point<4>(zeros_f[e], zi, delta);
+  dS[e] = fmaf(-delta, acc_w, acc_s);
+  dZ[e] = -scales[e] * acc_w;
 }
 
 // dS[i, gi] = sum of the group's partial pieces, in index order (deterministic); with
@@ -756,11 +786,12 @@ int launch_qgemm_t(const CUtensorMap& tmap, const CUtensorMap& tmap_pk, bool pkt
                : launch_qgemm_k<BITS, TRANS, FOLD, false>(tmap, tmap_pk, p, grid, st);
 }
 
-int launch_qgemm(const peqa_qweight_t* w, int g, const void* act, int T, void* out, bool trans,
-                 cudaStream_t st) {
+int launch_qgemm(const peqa_qweight_t* w, const float* zeros_f, int g, const void* act, int T,
+                 void* out, bool trans, cudaStream_t st) {
   QGemmParams p;
   p.qw = w->qweight;
   p.zeros = w->zeros;
+  p.zeros_f = zeros_f;
   p.scales = w->scales;
   p.out = static_cast<__nv_bfloat16*>(out);
   p.N = w->out_features;
@@ -784,7 +815,7 @@ int launch_qgemm(const peqa_qweight_t* w, int g, const void* act, int T, void* o
   PEQA_TRY(sm_count(&sms));
   const int tiles = p.r_tiles * p.t_tiles;
   const int grid = tiles < sms ? tiles : sms;
-  const bool fold = trans || p.G > 1;
+  const bool fold = trans || p.G > 1 || zeros_f != nullptr;
   // Packed codes by TMA need a 16-byte row pitch: always true for 4-bit, K % 128 == 0 for 3-bit.
   const bool pktma = ((size_t)p.wpr * 4) % 16 == 0;
   CUtensorMap tmap_pk = tmap;
@@ -818,14 +849,16 @@ int ds_piece(int g) { return gcd_int(g, 128); }
 
 }  // namespace
 
-int launch_fwd(const peqa_qweight_t* w, int g, const void* X, int T, void* Y, cudaStream_t st) {
-  if (fwd_pair_supported(w)) return launch_fwd_pair(w, g, X, T, Y, st);
-  return launch_qgemm(w, g, X, T, Y, false, st);
+int launch_fwd(const peqa_qweight_t* w, const float* zeros_f, int g, const void* X, int T, void* Y,
+               cudaStream_t st) {
+  if (fwd_pair_supported(w)) return launch_fwd_pair(w, zeros_f, g, X, T, Y, st);
+  return launch_qgemm(w, zeros_f, g, X, T, Y, false, st);
 }
 
-int launch_dx(const peqa_qweight_t* w, int g, const void* dY, int T, void* dX, cudaStream_t st) {
-  if (dx_pair_supported(w)) return launch_dx_pair(w, g, dY, T, dX, st);
-  return launch_qgemm(w, g, dY, T, dX, true, st);
+int launch_dx(const peqa_qweight_t* w, const float* zeros_f, int g, const void* dY, int T, void* dX,
+              cudaStream_t st) {
+  if (dx_pair_supported(w)) return launch_dx_pair(w, zeros_f, g, dY, T, dX, st);
+  return launch_qgemm(w, zeros_f, g, dY, T, dX, true, st);
 }
 
 size_t ds_workspace_bytes(const peqa_qweight_t* w, int g, int T) {
@@ -840,13 +873,16 @@ size_t dsdz_workspace_bytes(const peqa_qweight_t* w, int g, int T) {
   return 2 * ds_workspace_bytes(w, g, T);
 }
 
-int launch_ds(const peqa_qweight_t* w, int g, const void* X, const void* dY, int T, float* dS,
-              float* dZ, const DsAdam* adam, void* workspace, size_t workspace_bytes, cudaStream_t st) {
+int launch_ds(const peqa_qweight_t* w, const float* zeros_f, int g, const void* X, const void* dY,
+              int T, float* dS, float* dZ, const DsAdam* adam, void* workspace,
+              size_t workspace_bytes, cudaStream_t st) {
   if (adam && dZ) return PEQA_ERR_BAD_SHAPE;   // dZ reads the scales the step would be rewriting
+  if (zeros_f && !dZ) return PEQA_ERR_NULL;    // the correction needs the sums dZ is made of
   (void)workspace_bytes;
   DsParams p;
   p.qw = w->qweight;
   p.zeros = w->zeros;
+  p.zeros_f = zeros_f;
   p.N = w->out_features;
   p.K = w->in_features;
   p.g = g;
@@ -909,6 +945,12 @@ int launch_ds(const peqa_qweight_t* w, int g, const void* X, const void* dY, int
     const long long n_out = (long long)p.N * p.G;
     const int ppg = g / p.piece;
     const int blocks = (int)((n_out + 255) / 256);
+    if (zeros_f) {
+      ds_reduce_zf_kernel<<<blocks, 256, 0, st>>>(p.out, p.out_z, dS, dZ, n_out, ppg, zeros_f, w->scales,
+                                                  w->bits);
+      PEQA_CUDA(cudaGetLastError());
+      return PEQA_OK;
+    }
     ds_reduce_kernel<<<blocks, 256, 0, st>>>(p.out, dS, n_out, ppg, nullptr, p.adam, p.adam_s,
                                              p.adam_m, p.adam_v);
     PEQA_CUDA(cudaGetLastError());

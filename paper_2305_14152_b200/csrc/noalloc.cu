@@ -64,5 +64,5 @@ extern "C" int peqa_qlinear_bwd_ds_static(const peqa_qweight_t* w, const void* X
   if (need > 0) PEQA_TRY(scratch_for_current_device(&scratch));
   // Every partial sum the reduction reads is written by the gradient kernel of
   // the same call first, so nothing in the array has to start at zero.
-  return launch_ds(w, g, X, dY, T, dS, nullptr, nullptr, scratch, need, as_stream(stream));
+  return launch_ds(w, nullptr, g, X, dY, T, dS, nullptr, nullptr, scratch, need, as_stream(stream));
 }
