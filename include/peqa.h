@@ -319,23 +319,29 @@ size_t peqa_bwd_ds_static_capacity_bytes(void);
  * quantization and is shared by every task (Sec. 3.3), so a server may keep it
  * in the order the small-batch kernel streams best.  The canonical packed
  * layout above stays the interchange format; the prepared buffer holds exactly
- * the same bits, rearranged:
- *   rg = row / 8, r = row % 8, u = column / 128 (U = K / 128), C = bits;
- *   the 4*bits words of a row's 128-column unit are cut into C chunks of 16
- *   bytes, and chunk c of unit (row, u) is stored at 16-byte index
- *   ((rg*C + c)*U + u)*8 + r;
- *   inside every 32-column run the code of column 2k is stored at code position
- *   lo(k) and the code of column 2k+1 at position hi(k), k = 0..15, where for
- *   bits = 4: lo(k) = 8*(k/4) + k%4, hi(k) = lo(k) + 4, and for bits = 3:
+ * the same codes, rearranged (zero codes fill columns K .. 512*T - 1 and the row
+ * group that completes an odd count of row groups):
+ *   rg = row / 8, r = row % 8, step t = column / 512, T = ceil(K / 512), C = bits;
+ *   block (rg, t) is C*512 bytes at byte offset (((rg/2)*T + t)*2 + rg%2)*C*512
+ *   and consists of C chunks of 32 lanes of 16 bytes, chunk-major: word wo of
+ *   chunk c of lane l is the lane's word wi = 4*c + wo;
+ *   lane l = 4*r + c4 holds, of row 8*rg + r, columns 8*c4 .. 8*c4 + 7 of each of
+ *   the step's sixteen 32-column runs; its 4*C words are four strings of C words
+ *   (string s = words s*C .. s*C + C - 1 = runs 4s .. 4s + 3 of the step);
+ *   a string is a little-endian bit string of 32 code positions (position p =
+ *   bits [bits*p, bits*p + bits)); the code of string column
+ *   cs = 8*(run % 4) + column % 8 is stored at position lo(cs/2) when cs is even
+ *   and hi(cs/2) when cs is odd, where for bits = 4: lo(k) = 8*(k/4) + k%4,
+ *   hi(k) = lo(k) + 4, and for bits = 3:
  *   lo = {1,0,3,2,4,9,12,11,15,14,18,21,24,23,26,25},
- *   hi = {5,6,7,8,10,13,16,17,19,20,22,27,28,29,30,31}
- *   (code position p = bits [bits*p, bits*p + bits) of the run's bit string).
+ *   hi = {5,6,7,8,10,13,16,17,19,20,22,27,28,29,30,31}.
  * peqa_decode_unprepare(peqa_decode_prepare(Q)) == Q bit for bit.
  * Requires K % 128 == 0 and N % 8 == 0; the prepared buffer has
- * peqa_decode_prepared_bytes(w) = N*K*bits/8 bytes (0 for an unsupported shape)
- * and must be 16-byte aligned.  Only bits, out_features, in_features and
- * group_size of *w are read by prepared_bytes and unprepare; prepare also reads
- * w->qweight.
+ * peqa_decode_prepared_bytes(w) = 2*ceil(N/16) * T * bits * 512 bytes (N*K*bits/8
+ * when K % 512 == 0 and N % 16 == 0; 0 for an unsupported shape) and must be
+ * 16-byte aligned.  Only
+ * bits, out_features, in_features and group_size of *w are read by
+ * prepared_bytes and unprepare; prepare also reads w->qweight.
  */
 size_t peqa_decode_prepared_bytes(const peqa_qweight_t* w);
 int peqa_decode_prepare(const peqa_qweight_t* w, uint32_t* prepared, void* stream);
@@ -343,18 +349,20 @@ int peqa_decode_unprepare(const peqa_qweight_t* w, const uint32_t* prepared, uin
                           void* stream);
 
 /*
- * Small-batch forward (Sec. 3.1 / 3.3) reading the prepared weights, for layers
- * with one scale per channel (group_size 0 or K; else PEQA_ERR_BAD_SHAPE):
- *   Y[m,i] = s_m[i] * sum_j X[m,j] * (Q[i,j] - z[i]),   1 <= M <= 16
- * where s_m = w->scales, or, when task_ids is not NULL, row
- * clamp(task_ids[m], 0, n_tasks-1) of scale_table (fp32 [n_tasks, N]): token m is
- * served with the scales of its own task (Sec. 3.3).  w->qweight is not read.
+ * Small-batch forward (Sec. 3.1 / 3.3) reading the prepared weights:
+ *   Y[m,i] = sum_g s_m[i,g] * sum_{j in g} X[m,j] * (Q[i,j] - z[i,g]),   1 <= M <= 16
+ * for one scale per channel (group_size 0 or K), groups of 64, 128 or 256
+ * columns, and groups that are multiples of 512 columns (Sec. 4.2; other group
+ * sizes: PEQA_ERR_BAD_SHAPE, use peqa_qlinear_decode).  s_m = w->scales, or,
+ * when task_ids is not NULL, entry clamp(task_ids[m], 0, n_tasks-1) of
+ * scale_table (fp32 [n_tasks, N, G]): token m is served with the scales of its
+ * own task (Sec. 3.3).  w->qweight is not read.
  *   X  in  bf16 [M, K]    Y  out  bf16 [M, N]    task_ids  in  int32 [M] (device)
  * No workspace.  The kernel is launched so that it may begin while earlier work
- * on `stream` is still draining: it reads `prepared`, w->zeros and the scales
- * before that work is known to be complete (X is read and Y written only after
- * it has completed).  These tensors must therefore be final when the call is made
- * -- synchronise once after peqa_decode_prepare or after loading a scale table.
+ * on `stream` is still draining: it starts to read `prepared` before that work
+ * is known to be complete (X, the zero-points and the scales are read and Y is
+ * written only after it has completed).  `prepared` must therefore be final when
+ * the call is made -- synchronise once after peqa_decode_prepare.
  */
 int peqa_qlinear_decode_prepared(const peqa_qweight_t* w, const uint32_t* prepared,
                                  const void* X_bf16, int M, void* Y_bf16,

@@ -168,18 +168,19 @@ def bwd_ds(X_bits, dY_bits, qweight, zeros, bits: int, group_size: int = 0,
     return dS
 
 
-def fwd_multitask(X_bits, qweight, zeros, scale_table, task_ids, bits: int) -> np.ndarray:
-    """Per-channel forward in which token m uses the scales of task task_ids[m] (Sec. 3.3: Q and
-    z are shared by all tasks, s is task-specific).  scale_table is [n_tasks, N]."""
+def fwd_multitask(X_bits, qweight, zeros, scale_table, task_ids, bits: int, group_size: int = 0) -> np.ndarray:
+    """Forward in which token m uses the scales of task task_ids[m] (Sec. 3.3: Q and z are shared
+    by all tasks, s is task-specific).  scale_table is [n_tasks, N] for one scale per channel or
+    [n_tasks, N, G] for grouped scales (Sec. 4.2)."""
     X_bits = _c(X_bits, np.uint16)
     scale_table = _c(scale_table, np.float32)
     task_ids = np.asarray(task_ids, dtype=np.int64)
-    n_tasks, N = scale_table.shape
+    n_tasks, N = scale_table.shape[:2]
     Y = np.empty((X_bits.shape[0], N), np.float64)
     for task in range(n_tasks):
         rows = np.nonzero(task_ids == task)[0]
         if rows.size:
-            Y[rows] = fwd(X_bits[rows], qweight, zeros, scale_table[task].reshape(N, 1), bits, 0)
+            Y[rows] = fwd(X_bits[rows], qweight, zeros, scale_table[task].reshape(N, -1), bits, group_size)
     return Y
 
 

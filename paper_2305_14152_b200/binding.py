@@ -386,10 +386,12 @@ def decode_prepare(w: QWeight) -> torch.Tensor:
     return out
 
 
-def decode_unprepare(w: QWeight, prepared: torch.Tensor) -> torch.Tensor:
+def decode_unprepare(w: QWeight, prepared: torch.Tensor, out=None) -> torch.Tensor:
     """Canonical packed matrix rebuilt from a prepared buffer."""
     _dev(prepared, torch.int32, "prepared")
-    out = torch.empty((w.N, w.K * w.bits // 32), dtype=torch.int32, device=prepared.device)
+    if out is None:
+        out = torch.empty((w.N, w.K * w.bits // 32), dtype=torch.int32, device=prepared.device)
+    _dev(out, torch.int32, "out")
     cs = w.c_struct()
     _check(lib().peqa_decode_unprepare(ctypes.byref(cs), prepared.data_ptr(), out.data_ptr(), _stream()),
            "peqa_decode_unprepare")
@@ -398,7 +400,7 @@ def decode_unprepare(w: QWeight, prepared: torch.Tensor) -> torch.Tensor:
 
 def qlinear_decode_prepared(w: QWeight, prepared: torch.Tensor, X: torch.Tensor, Y=None,
                             scale_table=None, task_ids=None):
-    """Decode from the prepared weights; with scale_table [n_tasks, N] and task_ids [M] every
+    """Decode from the prepared weights; with scale_table [n_tasks, N, G] and task_ids [M] every
     token uses the scales of its own task."""
     _dev(prepared, torch.int32, "prepared")
     _dev(X, torch.bfloat16, "X")

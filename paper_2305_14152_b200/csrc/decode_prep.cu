@@ -1,46 +1,57 @@
 // Small-batch forward (token generation) from a prepared copy of the frozen
-// weights:  Y[m,i] = s[i] * sum_j X[m,j] * (Q[i,j] - z[i])   (Eq. 2, M <= 16 tokens,
-// one scale per channel; Sec. 3.1 / 3.3: the memory-bound matrix-vector regime).
+// weights:  Y[m,i] = sum_g s[i,g] * sum_{j in g} X[m,j] * (Q[i,j] - z[i,g])   (Eq. 2 with
+// M <= 16 tokens; Sec. 3.1 / 3.3: the memory-bound matrix-vector regime).
 //
 // The frozen matrix never changes after quantization (Sec. 3.3), so a server
 // can keep it in whatever order suits the kernel.  The prepared layout stores the
 // same bits as the canonical packed matrix, rearranged so that
-//   * the 16-byte piece every lane of a warp needs next lies in one contiguous
-//     512-byte run (no shared-memory staging of the weights: they go from HBM
-//     straight to registers, several 16-byte loads per lane in flight), and
-//   * inside every 32-column run, the two codes one logic operation extracts as
-//     a bf16 pair are the codes of two ADJACENT columns, so the activations are
-//     used in their natural order.
+//   * everything one warp needs for one step (8 rows x 512 columns) is one
+//     contiguous block that a single bulk copy moves into shared memory, in the
+//     order the lanes read it (16 bytes per lane and read, no bank conflicts);
+//   * the sixteen contraction slots of one warp-level MMA are sixteen columns of
+//     one 32-column run, so they share a quantization group and the scale and
+//     zero-point can be applied per group to the accumulator;
+//   * the two codes one logic operation extracts as a bf16 pair are the codes of
+//     two ADJACENT columns, so the activations are used in their natural order.
 //
-// Layout.  rg = row / 8, r = row % 8, unit u = column / 128 (U = K / 128 units),
-// C = bits (16-byte chunks per unit of one row: 48 or 64 bytes).  Chunk c of the
-// unit (row, u) is stored at 16-byte index ((rg * C + c) * U + u) * 8 + r.  The
-// 4*bits words of a unit are its four 32-column runs in order; within a run, the
-// code of column 2k sits at bit position bits*stream_lo(k) and the code of column
-// 2k+1 at bits*stream_hi(k) (k = 0..15; dequant.cuh).
+// Layout.  rg = row / 8, r = row % 8, step t = column / 512 (T = ceil(K / 512)
+// steps; columns beyond K hold zero codes), C = bits.  Block (rg, t) is C*512
+// bytes at byte offset (((rg/2)*T + t)*2 + rg%2)*C*512, so the two row groups of a
+// pair alternate step by step and a pair's consecutive steps are contiguous
+// (an odd count of row groups is padded with a group of zero codes): chunk c
+// (0..C-1), lane l (0..31), 16 bytes each, chunk-major.  Lane l = 4*r + c4 owns, of row 8*rg + r, columns
+// 8*c4 .. 8*c4+7 of each of the step's sixteen 32-column runs.  Its 4*C words are
+// four strings of C words; string s holds runs 4s .. 4s+3, its string column
+// cs = 8*(run % 4) + (column % 8); string column 2k sits at code position
+// stream_lo(k) and 2k+1 at stream_hi(k) (dequant.cuh), code position p being bits
+// [bits*p, bits*p + bits) of the string read as a little-endian bit string.
 //
 // Work split.  One CTA per SM owns a contiguous range of 8-row groups and all
-// of K for them, so no sum crosses a CTA: no workspace, no atomics.  Two row
-// groups form a "pair", the 16 rows of a warp-level mma.m16n8k16 whose 8-wide
-// side are the tokens.  Lane (r, c) = (lane / 4, lane % 4) holds, for rows r of
-// both groups, one unit of 128 columns; a warp step is four units.  The sixteen
-// warps are arranged as PG pairs x S splits of the unit range, chosen on the
-// host so that all warps have the same number of steps.  Codes reach the tensor
-// core as the biased integers (bias + q) they are after one logic operation;
-// the zero-point and bias terms come off the sum at the end:
-//   y = s * (acc - z * sum_j x_j - sum_j bias_j x_j).
-// Warps' partial sums meet in shared memory after each round and are added in
-// warp order, so results do not depend on timing.
+// of K for them, so no sum crosses a CTA: no workspace, no atomics.  Row
+// groups 2P and 2P+1 form a "pair", the 16 rows of a warp-level mma.m16n8k16
+// whose 8-wide side are the tokens (a range that starts or ends inside a pair
+// runs that group as a half pair).  The CTA's (pair, step) list, pair-major, is cut into sixteen
+// contiguous ranges of equal cost, one per warp.  A warp streams its range
+// through a private ring in shared memory: lane 0 issues one bulk copy per slot
+// (one or two steps of a pair: 3 to 8 KiB of contiguous memory; streaming reads
+// on this part want few, large copies and well over 100 KiB in flight per SM)
+// and all lanes wait on the slot's mbarrier.  Codes reach the tensor core as the biased integers
+// (bias + q) they are after one logic operation; the zero-point and bias terms
+// come off the sum when a group (or the row) is complete:
+//   y += s * (acc - z * sum_j x_j - sum_j bias_j x_j).
+// When a warp's range crosses into the next pair it parks its sums in shared
+// memory; at the end the parked sums of each pair are added in warp order, so
+// results do not depend on timing.
 //
 // Activations are staged in shared memory, all of K when they fit, otherwise in
-// chunks of units with the per-output sums carried in shared memory.
+// chunks of steps with the per-output sums carried in shared memory.
 //
 // Launch overlap.  The kernel is launched with programmatic stream
 // serialization: it lets the next kernel in the stream start as soon as SMs
 // free up, requests its own first weights at once, and only then waits for the
-// preceding kernel before it touches X or Y.  The prepared weights, zero-points
-// and scales are therefore read before earlier work in the stream is known to be
-// complete: they must be final when the call is made.
+// preceding kernel before it touches X or Y.  The prepared weights are
+// therefore read before earlier work in the stream is known to be complete:
+// they must be final when the call is made.
 #include <cuda_bf16.h>
 
 #include "common.cuh"
@@ -51,30 +62,39 @@ namespace peqa {
 
 namespace {
 
-constexpr int kPWarps = 16;
+using namespace ptx;
+
+#ifndef PEQA_PREP_WARPS
+#define PEQA_PREP_WARPS 16
+#endif
+constexpr int kPWarps = PEQA_PREP_WARPS;
 constexpr int kPThreads = kPWarps * 32;
-constexpr int kPUnitPitch = 272;                   // 128 activations (256 B) + 16 B bank skew
 constexpr int kPSmemLimit = 227 * 1024;
+constexpr int kPMaxSlots = 4;
+constexpr int kStepCols = 512;
+constexpr int kPBarBytes = kPWarps * kPMaxSlots * 8;              // the warps' mbarriers
+constexpr int kPHeadBytes = kPBarBytes + 128;                     // + abort flag and wait limit
 
 struct PrepParams {
-  const uint4* P;           // prepared weights
-  const uint8_t* zeros;     // [N]
-  const float* scales;      // [N] or table [n_tasks, N]
+  const uint8_t* P;         // prepared weights
+  const uint8_t* zeros;     // [N, G]
+  const float* scales;      // [N, G] or table [n_tasks, N, G]
   const __nv_bfloat16* X;   // [M, K]
   __nv_bfloat16* Y;         // [M, N]
   const int32_t* task_ids;  // nullptr: one task
   int n_tasks;
-  int N, K, U, M;
+  int N, K, G, M;
   int rgs;                  // row groups in the matrix (N / 8)
   int rg_per_cta;
-  int S, PG;                // splits of a pair's unit range, pairs per round (S * PG = 16)
-  int rounds;               // ceil(pairs per CTA / PG)
-  int chunk_units;          // units of K staged at a time
+  int T;                    // steps of 512 columns per row group
+  int spc;                  // steps per staged chunk of activations
   int nchunks;
-  int ups;                  // units per split within a full chunk (multiple of 4)
-  int spr;                  // steps per split and round (ups / 4)
+  int slots;                // ring slots per warp
+  int sps;                  // steps per slot (1 or 2)
+  int maxseg;               // parked partial sums per warp and chunk
   int x_pitch;              // bytes between staged token rows
   int pairs_per_cta;
+  int* status;
 };
 
 __device__ __forceinline__ void pmma_16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0,
@@ -86,35 +106,49 @@ __device__ __forceinline__ void pmma_16816(float (&d)[4], const uint32_t (&a)[4]
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
-__device__ __forceinline__ uint4 ldg_stream(const uint4* p) {
+// Contiguous bulk copy global -> shared memory; its bytes are credited to `bar`.  Both
+// addresses 16-byte aligned, bytes a multiple of 16.
+__device__ __forceinline__ void bulk_load(uint32_t dst_smem, const void* src, uint32_t bytes,
+                                          uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+      ::"r"(dst_smem), "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(bar)
+      : "memory");
+}
+
+// 16 bytes of a ring slot.  Volatile at both compiler levels: the read must be issued before
+// the bulk copy that refills the slot, and neither the compiler nor the assembler can see
+// that the copy writes this memory, so an ordinary load could be moved behind it.
+__device__ __forceinline__ uint4 ring_load(uint32_t addr) {
   uint4 v;
-  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+  asm volatile("ld.volatile.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
                : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-               : "l"(p));
+               : "r"(addr)
+               : "memory");
   return v;
 }
 
-// One lane's weights of one step: rows r of the pair's two groups, one unit each.
+// One lane's weights of one step: row r of the pair's two groups.
 template <int BITS>
 struct StepRegs {
   uint4 a[BITS];
   uint4 b[BITS];
 };
 
-// MMAs 2*MM and 2*MM + 1 of a 32-column run: the run's pairs 4*MM .. 4*MM + 3, i.e. its
-// columns 8*MM .. 8*MM + 7, whose activations are one 16-byte word per token.
-template <int BITS, int NT, int MM>
+// MMAs 2*MM and 2*MM + 1 of string S: run 4*S + MM of the step, whose eight columns of this
+// lane are one 16-byte word of activations per token.
+template <int BITS, int NT, bool HAS_B, int MM>
 __device__ __forceinline__ void run_mma2(const uint32_t (&wa)[BITS], const uint32_t (&wb)[BITS],
-                                         bool has_b, const uint8_t* x0, const uint8_t* x1,
+                                         const uint8_t* x0, const uint8_t* x1,
                                          float (&acc)[NT][4]) {
-  const uint4 xa = *reinterpret_cast<const uint4*>(x0 + MM * 16);
+  const uint4 xa = *reinterpret_cast<const uint4*>(x0 + MM * 64);
   uint4 xb = make_uint4(0u, 0u, 0u, 0u);
-  if (NT == 2) xb = *reinterpret_cast<const uint4*>(x1 + MM * 16);
+  if (NT == 2) xb = *reinterpret_cast<const uint4*>(x1 + MM * 64);
   uint32_t f0[4], f1[4];
   dq::mma_pairs_stream<BITS, 2 * MM>(wa, f0[0], f0[2]);
   dq::mma_pairs_stream<BITS, 2 * MM + 1>(wa, f1[0], f1[2]);
   f0[1] = f0[3] = f1[1] = f1[3] = 0u;
-  if (has_b) {
+  if (HAS_B) {
     dq::mma_pairs_stream<BITS, 2 * MM>(wb, f0[1], f0[3]);
     dq::mma_pairs_stream<BITS, 2 * MM + 1>(wb, f1[1], f1[3]);
   }
@@ -126,342 +160,601 @@ __device__ __forceinline__ void run_mma2(const uint32_t (&wa)[BITS], const uint3
   }
 }
 
-template <int BITS, int NT>
-__device__ __forceinline__ void step_compute(const StepRegs<BITS>& w, bool has_b, const uint8_t* x0,
-                                             const uint8_t* x1, float (&acc)[NT][4]) {
-  const uint32_t* fa = reinterpret_cast<const uint32_t*>(w.a);
-  const uint32_t* fb = reinterpret_cast<const uint32_t*>(w.b);
-#pragma unroll
-  for (int s = 0; s < 4; ++s) {
-    uint32_t wa[BITS], wb[BITS];
-#pragma unroll
-    for (int e = 0; e < BITS; ++e) {
-      wa[e] = fa[s * BITS + e];
-      wb[e] = fb[s * BITS + e];
-    }
-    run_mma2<BITS, NT, 0>(wa, wb, has_b, x0 + s * 64, x1 + s * 64, acc);
-    run_mma2<BITS, NT, 1>(wa, wb, has_b, x0 + s * 64, x1 + s * 64, acc);
-    run_mma2<BITS, NT, 2>(wa, wb, has_b, x0 + s * 64, x1 + s * 64, acc);
-    run_mma2<BITS, NT, 3>(wa, wb, has_b, x0 + s * 64, x1 + s * 64, acc);
-  }
-}
-
-// Bias the code of column j (0..31) of a run carries when it reaches the tensor core.
+// Bias the code of string column cs (0..31) carries when it reaches the tensor core.
 template <int BITS>
-__host__ __device__ constexpr float column_bias(int j) {
+__host__ __device__ constexpr float column_bias(int cs) {
   if (BITS == 4) return 128.0f;
-  return dq::stream_alt(3, j >> 1) ? ((j & 1) ? 16.0f : 64.0f) : ((j & 1) ? 128.0f : 8.0f);
+  return dq::stream_alt(3, cs >> 1) ? ((cs & 1) ? 16.0f : 64.0f) : ((cs & 1) ? 128.0f : 8.0f);
 }
 
-template <int BITS, int NT>
+// GSH: quantization groups of 32 << GSH columns (1: 64, 2: 128, 3: 256), or 0: one group
+// per row or groups that are multiples of 512 columns (the sums of a whole staged chunk of
+// steps are taken off at once, which needs the chunk to lie inside one group).
+template <int BITS, int NT, int GSH>
 __global__ void __launch_bounds__(kPThreads, 1)
 decode_prep_kernel(const PrepParams p) {
-  constexpr int C = BITS;                            // 16-byte chunks per unit of one row
+  constexpr int C = BITS;                            // 16-byte chunks per lane, step and group
+  constexpr int BLK = C * 512;                       // bytes of one block (rg, t)
   constexpr int TOKP = 8 * NT;
+  constexpr bool GROUPED = GSH != 0;
+  constexpr int RUNS_PER_GROUP = GROUPED ? (1 << GSH) : 16;
+  constexpr int GPS = 16 / RUNS_PER_GROUP;           // groups per step (GROUPED)
   extern __shared__ uint8_t prep_smem_raw[];
   uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(prep_smem_raw) + 127) &
                                              ~static_cast<uintptr_t>(127));
-  float* partial = reinterpret_cast<float*>(base);                 // [2][16 warps][16 rows][TOKP]
-  float* yacc = partial + 2 * kPWarps * 16 * TOKP;                  // [pairs][16][TOKP]
-  float* xtot = yacc + (size_t)p.pairs_per_cta * 16 * TOKP;         // [TOKP][2]: sum x, sum bias*x
-  uint8_t* xzero = reinterpret_cast<uint8_t*>(xtot + TOKP * 2);     // 256 B of zeros
-  uint8_t* xs = xzero + 256;                                        // [M][x_pitch]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(base);                        // [warps][kPMaxSlots]
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(base + kPBarBytes);   // [0] flag, [1] limit
+  const int toks = (p.M + 1) & ~1;                                           // tokens kept of a tile
+  float* part = reinterpret_cast<float*>(base + kPHeadBytes);                // [warps][maxseg][16][toks]
+  float* yacc = part + (size_t)kPWarps * p.maxseg * 16 * toks;               // [pairs][16][toks]
+  float* sums = yacc + (p.nchunks > 1 ? (size_t)p.pairs_per_cta * 16 * toks : 0);
+  // sums, GROUPED: [groups of the chunk][TOKP][2] = (sum x, sum bias*x) per group and token;
+  // else [16 warps][TOKP][2]: every warp's share of the chunk's sums, added in warp order
+  const int sum_rows = GROUPED ? p.spc * GPS : kPWarps;
+  uint8_t* xs = reinterpret_cast<uint8_t*>(
+      (reinterpret_cast<uintptr_t>(sums + (size_t)sum_rows * TOKP * 2) + 127) & ~static_cast<uintptr_t>(127));
+  uint8_t* ring = xs + (((size_t)p.M * p.x_pitch + 127) & ~static_cast<size_t>(127));
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int r8 = lane >> 2, c4 = lane & 3;
   const int rg0 = blockIdx.x * p.rg_per_cta;
   const int rg_end = min(p.rgs, rg0 + p.rg_per_cta);
-  const int split = warp % p.S, pr = warp / p.S;
+  // pairs are (2P, 2P+1) for the whole matrix; a range that starts (ends) at an odd row group
+  // has a half pair in front (at the end)
+  const int P0 = rg0 >> 1;
+  const int lead = rg0 & 1;
+  const int rest = rg_end - rg0 - lead;
+  const int trail = rest & 1;
+  const int F = rest >> 1;                           // full pairs
+  const int npairs = lead + F + trail;
+  const int slot_bytes = 2 * BLK * p.sps;
 
   // the next kernel of the stream may be scheduled as SMs free up
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
-  // ---- weight stream of this warp: step i = (chunk, round, st)
-  const int steps_per_chunk = p.rounds * p.spr;
-  const int total = p.nchunks * steps_per_chunk;
-  auto step_unit = [&](int i, int& chunk, int& round, bool& active) -> int {
-    chunk = i / steps_per_chunk;
-    const int rem = i - chunk * steps_per_chunk;
-    round = rem / p.spr;
-    const int st = rem - round * p.spr;
-    const int cu0 = chunk * p.chunk_units;
-    const int cend = min(p.U, cu0 + p.chunk_units);
-    const int u = cu0 + split * p.ups + 4 * st + c4;
-    active = u < min(cend, cu0 + (split + 1) * p.ups);
-    return u;
-  };
-  auto load_step = [&](int i, StepRegs<BITS>& w) {
-#pragma unroll
-    for (int c = 0; c < C; ++c) {
-      w.a[c] = make_uint4(0u, 0u, 0u, 0u);
-      w.b[c] = make_uint4(0u, 0u, 0u, 0u);
-    }
-    if (i >= total) return;
-    int chunk, round;
-    bool active;
-    const int u = step_unit(i, chunk, round, active);
-    const int rga = rg0 + 2 * (round * p.PG + pr);
-    if (!active || rga >= rg_end) return;
-    const size_t plane = (size_t)p.U * 8;                         // 16-byte pieces per (rg, c)
-    const uint4* pa = p.P + (size_t)rga * C * plane + (size_t)u * 8 + r8;
-#pragma unroll
-    for (int c = 0; c < C; ++c) w.a[c] = ldg_stream(pa + c * plane);
-    if (rga + 1 < rg_end) {
-      const uint4* pb = pa + C * plane;
-#pragma unroll
-      for (int c = 0; c < C; ++c) w.b[c] = ldg_stream(pb + c * plane);
-    }
-  };
+  if (threadIdx.x == 0) {
+    abort_flag[0] = 0;
+    abort_flag[1] = p.status[4];
+  }
+  if (lane == 0) {
+    for (int s = 0; s < p.slots; ++s) mbar_init(smem_u32(&bars[warp * kPMaxSlots + s]), 1);
+    fence_mbar_init();
+  }
+  __syncwarp();
 
-  StepRegs<BITS> w0, w1;
-  load_step(0, w0);
-  load_step(1, w1);
-
-  for (int i = threadIdx.x; i < 64 + TOKP * 2; i += kPThreads) {
-    if (i < 64) reinterpret_cast<uint32_t*>(xzero)[i] = 0u;
-    else xtot[i - 64] = 0.0f;
+  // ---- this warp's steps of a chunk: [bound(w), bound(w+1)) of the pair-major list, cut so
+  // that the warps' costs are equal (a step of a full pair costs 2, of a half pair 1)
+  auto spc_of = [&](int ch) { return min(p.spc, p.T - ch * p.spc); };
+  auto bound = [&](int w, int spc_c) {
+    const int tot = (lead + 2 * F + trail) * spc_c;
+    int b = (int)(((long long)w * tot) / kPWarps);
+    int at = 0;
+    if (lead) {
+      if (b <= spc_c) return b;
+      b -= spc_c;
+      at = spc_c;
+    }
+    return b <= 2 * F * spc_c ? at + ((b + 1) >> 1) : at + F * spc_c + (b - 2 * F * spc_c);
+  };
+  auto pair_full = [&](int lp) { return lp >= lead && lp < lead + F; };
+  // first row group of local pair lp (the only one of a half pair)
+  auto pair_rg = [&](int lp) { return lp == 0 ? rg0 : 2 * (P0 + lp); };
+  // ---- ring: issue cursor (only lane 0 uses it)
+  const uint32_t ring_w = smem_u32(ring) + (uint32_t)warp * (uint32_t)(p.slots * slot_bytes);
+  const uint32_t bar_w = smem_u32(&bars[warp * kPMaxSlots]);
+  int i_ch = 0, i_lin = 0, i_hi = 0, i_spc = 1;
+  int i_lp = 0, i_tl = 0, i_slot = 0;               // pair and step of i_lin; slot of the next copy
+  auto issue_seek = [&]() {       // moves to the first chunk (from i_ch on) where this warp has steps
+    while (i_ch < p.nchunks) {
+      i_spc = spc_of(i_ch);
+      i_lin = bound(warp, i_spc);
+      i_hi = bound(warp + 1, i_spc);
+      i_lp = i_lin / i_spc;
+      i_tl = i_lin - i_lp * i_spc;
+      if (i_lin < i_hi) return;
+      ++i_ch;
+    }
+  };
+  auto issue_next = [&]() {
+    if (i_ch >= p.nchunks) return;
+    const int lp = i_lp, tl = i_tl;
+    const int t = i_ch * p.spc + tl;
+    const int n = (p.sps == 2 && i_lin + 1 < i_hi && tl + 1 < i_spc) ? 2 : 1;
+    const int rg = pair_rg(lp);
+    const int slot = i_slot;
+    const uint32_t bar = bar_w + slot * 8;
+    const uint32_t dst = ring_w + slot * slot_bytes;
+    // block (rg, t) lies at (((rg >> 1) * T + t) * 2 + (rg & 1)) * BLK
+    const uint8_t* src = p.P + ((((size_t)(rg >> 1) * p.T + t) * 2 + (rg & 1)) * BLK);
+    if (pair_full(lp)) {
+      mbar_arrive_expect_tx(bar, n * 2 * BLK);
+      bulk_load(dst, src, n * 2 * BLK, bar);                       // steps t .. t+n-1 are contiguous
+    } else {
+      mbar_arrive_expect_tx(bar, n * BLK);
+      bulk_load(dst, src, BLK, bar);
+      if (n == 2) bulk_load(dst + 2 * BLK, src + 2 * BLK, BLK, bar);
+    }
+    i_slot = i_slot + 1 == p.slots ? 0 : i_slot + 1;
+    i_lin += n;
+    i_tl += n;
+    if (i_tl >= i_spc) {
+      i_tl = 0;
+      ++i_lp;
+    }
+    if (i_lin >= i_hi) {
+      ++i_ch;
+      issue_seek();
+    }
+  };
+  if (lane == 0) {
+    issue_seek();
+    for (int s = 0; s < p.slots; ++s) issue_next();
   }
 
   // everything below reads X or writes Y: the preceding kernel must have completed
   asm volatile("griddepcontrol.wait;" ::: "memory");
 
-  // bias of the eight columns of a 16-byte piece of X: piece q = (piece index) % 4 of its run
-  float bias8[8];
-  {
-    const int q = lane & 3;
-#pragma unroll
-    for (int e = 0; e < 8; ++e) {
-      float b = column_bias<BITS>(e);
-      if (q == 1) b = column_bias<BITS>(8 + e);
-      if (q == 2) b = column_bias<BITS>(16 + e);
-      if (q == 3) b = column_bias<BITS>(24 + e);
-      bias8[e] = b;
-    }
-  }
+  int c_slot = 0;
+  uint32_t c_phase = 0;                              // parity of the ring's current round
+  bool ok = true;
 
-  int i = 0;
-  for (int chunk = 0; chunk < p.nchunks; ++chunk) {
-    const int cu0 = chunk * p.chunk_units;
-    const int cun = min(p.U, cu0 + p.chunk_units) - cu0;           // units in this chunk
-    if (chunk > 0) __syncthreads();                                // the previous chunk is no longer read
-    // ---- stage X[:, chunk]: 16 pieces of 16 bytes per unit and token
-    for (int idx = threadIdx.x; idx < p.M * cun * 16; idx += kPThreads) {
-      const int m = idx / (cun * 16);
-      const int rem = idx - m * cun * 16;
-      const int uu = rem >> 4, piece = rem & 15;
-      ptx::cp_async_16(ptx::smem_u32(xs + (size_t)m * p.x_pitch + uu * kPUnitPitch + piece * 16),
-                       p.X + (size_t)m * p.K + (size_t)(cu0 + uu) * 128 + piece * 8);
+  for (int ch = 0; ch < p.nchunks; ++ch) {
+    const int spc_c = spc_of(ch);
+    const int col0 = ch * p.spc * kStepCols;                       // first column of the chunk
+    const int ccols = min(p.K - col0, spc_c * kStepCols);          // real columns in it
+    if (ch > 0) __syncthreads();                                   // the previous chunk is no longer read
+    // ---- stage X[:, chunk] (columns beyond K read as zero)
+    const int pieces = spc_c * (kStepCols / 8);                    // 16-byte pieces per token
+    for (int idx = threadIdx.x; idx < p.M * pieces; idx += kPThreads) {
+      const int m = idx / pieces, pc = idx - m * pieces;
+      uint8_t* dst = xs + (size_t)m * p.x_pitch + pc * 16;
+      if (pc * 8 < ccols) cp_async_16(smem_u32(dst), p.X + (size_t)m * p.K + col0 + pc * 8);
+      else *reinterpret_cast<uint4*>(dst) = make_uint4(0u, 0u, 0u, 0u);
     }
     asm volatile("cp.async.wait_all;" ::: "memory");
     __syncthreads();
-    // ---- per token: sum of x and sum of bias * x over the chunk, added to the running totals
-    if (warp < p.M) {
-      float sx = 0.0f, sb = 0.0f;
-      const uint8_t* row = xs + (size_t)warp * p.x_pitch;
-      for (int pc = lane; pc < cun * 16; pc += 32) {               // pc % 4 == lane % 4
-        const uint4 v = *reinterpret_cast<const uint4*>(row + (pc >> 4) * kPUnitPitch + (pc & 15) * 16);
+    // ---- sum of x and sum of bias * x: per token and group, or per token and warp
+    {
+      // bias of the two columns in word e of a piece whose run in the step is run % 4 == rq
+      auto piece_sums = [&](const uint8_t* ptr, int rq, float& sx, float& sb) {
+        const uint4 v = *reinterpret_cast<const uint4*>(ptr);
         const uint32_t wv[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
           const float lo = __uint_as_float(wv[e] << 16), hi = __uint_as_float(wv[e] & 0xFFFF0000u);
           sx += lo + hi;
-          sb = fmaf(bias8[2 * e], lo, sb);
-          sb = fmaf(bias8[2 * e + 1], hi, sb);
+          float b0 = 128.0f, b1 = 128.0f;
+          if (BITS == 3) {
+            const bool alt = (dq::stream_alt_mask3() >> (4 * rq + e)) & 1u;
+            b0 = alt ? 64.0f : 8.0f;
+            b1 = alt ? 16.0f : 128.0f;
+          }
+          sb = fmaf(b0, lo, sb);
+          sb = fmaf(b1, hi, sb);
         }
-      }
+      };
+      if (GROUPED) {
+        const int ngr = spc_c * GPS;
+        constexpr int gpieces = RUNS_PER_GROUP * 4;                // 16-byte pieces per group
+        for (int idx = threadIdx.x; idx < ngr * p.M; idx += kPThreads) {
+          const int gi = idx / p.M, m = idx - gi * p.M;
+          const uint8_t* row = xs + (size_t)m * p.x_pitch + (size_t)gi * gpieces * 16;
+          float sx = 0.0f, sb = 0.0f;
+          for (int pc = 0; pc < gpieces; ++pc)
+            piece_sums(row + pc * 16, (gi * RUNS_PER_GROUP + (pc >> 2)) & 3, sx, sb);
+          sums[((size_t)gi * TOKP + m) * 2] = sx;
+          sums[((size_t)gi * TOKP + m) * 2 + 1] = sb;
+        }
+        __syncthreads();
+      } else {
+        // piece pc of a token goes to thread pc % 512: its run % 4 is the same for all of them
+        for (int m = 0; m < p.M; ++m) {
+          float sx = 0.0f, sb = 0.0f;
+          const uint8_t* row = xs + (size_t)m * p.x_pitch;
+          for (int pc = threadIdx.x; pc < pieces; pc += kPThreads)
+            piece_sums(row + pc * 16, (threadIdx.x >> 2) & 3, sx, sb);
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        sx += __shfl_xor_sync(0xffffffffu, sx, o);
-        sb += __shfl_xor_sync(0xffffffffu, sb, o);
-      }
-      if (lane == 0) {
-        xtot[warp * 2] += sx;
-        xtot[warp * 2 + 1] += sb;
+          for (int o = 16; o > 0; o >>= 1) {
+            sx += __shfl_xor_sync(0xffffffffu, sx, o);
+            sb += __shfl_xor_sync(0xffffffffu, sb, o);
+          }
+          if (lane == 0) {
+            sums[(warp * TOKP + m) * 2] = sx;
+            sums[(warp * TOKP + m) * 2 + 1] = sb;
+          }
+        }
+        // read after the barrier that follows the main loop
       }
     }
 
-    for (int round = 0; round < p.rounds; ++round) {
-      const int pair = round * p.PG + pr;
-      const int rga = rg0 + 2 * pair;
-      const bool has_b = rga + 1 < rg_end;
-      float acc[NT][4];
+    // ---- this warp's steps of the chunk
+    const int lo = bound(warp, spc_c), hi = bound(warp + 1, spc_c);
+    int seg = 0, cur_pair = -1;
+    float acc[NT][4], yv[NT][4];
 #pragma unroll
-      for (int nt = 0; nt < NT; ++nt)
+    for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-        for (int e = 0; e < 4; ++e) acc[nt][e] = 0.0f;
-
-      for (int st = 0; st < p.spr; ++st, ++i) {
-        int ch2, rd2;
-        bool active;
-        const int u = step_unit(i, ch2, rd2, active);
-        active = active && rga < rg_end;
-        const uint8_t* x0 = xzero;
-        const uint8_t* x1 = xzero;
-        if (active) {
-          const uint8_t* xu = xs + (u - cu0) * kPUnitPitch;
-          x0 = xu + (size_t)(r8 < p.M ? r8 : 0) * p.x_pitch;
-          x1 = xu + (size_t)(r8 + 8 < p.M ? r8 + 8 : 0) * p.x_pitch;
-        }
-        step_compute<BITS, NT>(w0, has_b, x0, x1, acc);
-        w0 = w1;
-        load_step(i + 2, w1);
-      }
-
-      // ---- this warp's partial sums: [16 rows][TOKP]
-      const int buf = (chunk * p.rounds + round) & 1;
-      float* mine = partial + (size_t)((buf * kPWarps + warp) * 16) * TOKP;
+      for (int e = 0; e < 4; ++e) acc[nt][e] = yv[nt][e] = 0.0f;
+    auto park = [&]() {
+      float* mine = part + ((size_t)(warp * p.maxseg + seg) * 16) * toks;
 #pragma unroll
       for (int nt = 0; nt < NT; ++nt) {
         const int tk = nt * 8 + c4 * 2;
-        *reinterpret_cast<float2*>(mine + r8 * TOKP + tk) = make_float2(acc[nt][0], acc[nt][1]);
-        *reinterpret_cast<float2*>(mine + (r8 + 8) * TOKP + tk) = make_float2(acc[nt][2], acc[nt][3]);
+        const float* v = GROUPED ? yv[nt] : acc[nt];
+        if (seg < p.maxseg && tk < toks) {
+          *reinterpret_cast<float2*>(mine + r8 * toks + tk) = make_float2(v[0], v[1]);
+          *reinterpret_cast<float2*>(mine + (r8 + 8) * toks + tk) = make_float2(v[2], v[3]);
+        }
+#pragma unroll
+        for (int e = 0; e < 4; ++e) acc[nt][e] = yv[nt][e] = 0.0f;
       }
-      __syncthreads();
-      // ---- add the splits of every pair of this round in warp order
-      const float* bufp = partial + (size_t)(buf * kPWarps * 16) * TOKP;
-      for (int idx = threadIdx.x; idx < p.PG * 16 * p.M; idx += kPThreads) {
-        const int q = idx / (16 * p.M);
-        const int rem = idx - q * 16 * p.M;
-        const int m = rem >> 4, lr = rem & 15;
-        const int pr2 = round * p.PG + q;
-        const int rg = rg0 + 2 * pr2 + (lr >> 3);
-        if (rg >= rg_end) continue;
-        float sum = 0.0f;
-        for (int sp = 0; sp < p.S; ++sp) sum += bufp[((q * p.S + sp) * 16 + lr) * TOKP + m];
-        if (p.nchunks > 1) {
-          float* ya = yacc + ((size_t)pr2 * 16 + lr) * TOKP + m;
-          if (chunk > 0) sum += *ya;
-          if (chunk + 1 < p.nchunks) {
-            *ya = sum;
-            continue;
+      ++seg;
+    };
+    const uint8_t* xl = xs + (size_t)(r8 < p.M ? r8 : 0) * p.x_pitch + c4 * 16;
+    const uint8_t* xh = xs + (size_t)(r8 + 8 < p.M ? r8 + 8 : 0) * p.x_pitch + c4 * 16;
+
+    int lin = lo;
+    int lp = lo / spc_c, tl = lo - lp * spc_c;
+    while (ok && lin < hi) {
+      const int nsteps = (p.sps == 2 && lin + 1 < hi && tl + 1 < spc_c) ? 2 : 1;
+      const int slot = c_slot;
+      if (!mbar_wait(bar_w + slot * 8, c_phase, abort_flag)) { ok = false; break; }
+      if (++c_slot == p.slots) {
+        c_slot = 0;
+        c_phase ^= 1u;
+      }
+      for (int j = 0; j < nsteps; ++j) {
+        if (lp != cur_pair) {
+          if (cur_pair >= 0) park();
+          cur_pair = lp;
+        }
+        const bool has_b = pair_full(lp);
+        StepRegs<BITS> w;
+        {
+          const uint32_t sp = ring_w + (uint32_t)(slot * slot_bytes + j * 2 * BLK + lane * 16);
+#pragma unroll
+          for (int c = 0; c < C; ++c) w.a[c] = ring_load(sp + c * 512);
+          if (has_b) {
+#pragma unroll
+            for (int c = 0; c < C; ++c) w.b[c] = ring_load(sp + (C + c) * 512);
+          } else {
+#pragma unroll
+            for (int c = 0; c < C; ++c) w.b[c] = make_uint4(0u, 0u, 0u, 0u);
           }
         }
-        const int row = rg * 8 + (lr & 7);
-        const float z = (float)__ldg(p.zeros + row);
-        const float* sc = p.scales;
-        if (p.task_ids) {
-          const int task = min(max(__ldg(p.task_ids + m), 0), p.n_tasks - 1);
-          sc += (size_t)task * p.N;
+        if (j + 1 == nsteps) {
+          // every lane has issued its reads of the slot: it can be refilled
+          __syncwarp();
+          if (lane == 0) issue_next();
         }
-        sum = (sum - fmaf(z, xtot[m * 2], xtot[m * 2 + 1])) * __ldg(sc + row);
-        p.Y[(size_t)m * p.N + row] = __float2bfloat16_rn(sum);
+
+        // scale and zero-point of this lane's rows for the groups of the step (GROUPED)
+        const int rowa = pair_rg(lp) * 8 + r8, rowb = rowa + 8;
+        float gs_a = 0.0f, gs_b = 0.0f, gz_a = 0.0f, gz_b = 0.0f;
+        float gs2_a = 0.0f, gs2_b = 0.0f, gz2_a = 0.0f, gz2_b = 0.0f;
+        const int gstep0 = ((ch * p.spc + tl) * GPS);              // first group of the step
+        if (GROUPED && !p.task_ids) {
+          // lane c4 fetches group c4 % GPS (and, with eight groups a step, group c4 + 4)
+          const int gl = c4 % GPS;
+          if (gstep0 + gl < p.G) {
+            gs_a = __ldg(p.scales + (size_t)rowa * p.G + gstep0 + gl);
+            gz_a = (float)__ldg(p.zeros + (size_t)rowa * p.G + gstep0 + gl);
+            if (has_b) {
+              gs_b = __ldg(p.scales + (size_t)rowb * p.G + gstep0 + gl);
+              gz_b = (float)__ldg(p.zeros + (size_t)rowb * p.G + gstep0 + gl);
+            }
+          }
+          if (GPS == 8 && gstep0 + gl + 4 < p.G) {
+            gs2_a = __ldg(p.scales + (size_t)rowa * p.G + gstep0 + gl + 4);
+            gz2_a = (float)__ldg(p.zeros + (size_t)rowa * p.G + gstep0 + gl + 4);
+            if (has_b) {
+              gs2_b = __ldg(p.scales + (size_t)rowb * p.G + gstep0 + gl + 4);
+              gz2_b = (float)__ldg(p.zeros + (size_t)rowb * p.G + gstep0 + gl + 4);
+            }
+          }
+        }
+        // group gi of the step is complete: take z * sum x + sum bias * x off and scale
+        auto flush = [&](int gi) {
+          const int gg = gstep0 + gi;                              // group index in the row
+          const float* sm = sums + ((size_t)(tl * GPS + gi) * TOKP) * 2;
+          if (!p.task_ids) {
+            const int src = (lane & ~3) | (gi & 3 & (GPS - 1));
+            const float sa = __shfl_sync(0xffffffffu, gi >= 4 ? gs2_a : gs_a, src);
+            const float sb = __shfl_sync(0xffffffffu, gi >= 4 ? gs2_b : gs_b, src);
+            const float za = __shfl_sync(0xffffffffu, gi >= 4 ? gz2_a : gz_a, src);
+            const float zb = __shfl_sync(0xffffffffu, gi >= 4 ? gz2_b : gz_b, src);
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+              const float4 sv = *reinterpret_cast<const float4*>(sm + (nt * 8 + c4 * 2) * 2);
+              yv[nt][0] = fmaf(sa, acc[nt][0] - fmaf(za, sv.x, sv.y), yv[nt][0]);
+              yv[nt][1] = fmaf(sa, acc[nt][1] - fmaf(za, sv.z, sv.w), yv[nt][1]);
+              yv[nt][2] = fmaf(sb, acc[nt][2] - fmaf(zb, sv.x, sv.y), yv[nt][2]);
+              yv[nt][3] = fmaf(sb, acc[nt][3] - fmaf(zb, sv.z, sv.w), yv[nt][3]);
+            }
+          } else if (gg < p.G) {
+            // every token has the scales of its own task (Sec. 3.3)
+            const float za = (float)__ldg(p.zeros + (size_t)rowa * p.G + gg);
+            const float zb = has_b ? (float)__ldg(p.zeros + (size_t)rowb * p.G + gg) : 0.0f;
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+              const float4 sv = *reinterpret_cast<const float4*>(sm + (nt * 8 + c4 * 2) * 2);
+#pragma unroll
+              for (int e = 0; e < 2; ++e) {
+                const int tok = nt * 8 + c4 * 2 + e;
+                const int task = tok < p.M ? min(max(__ldg(p.task_ids + tok), 0), p.n_tasks - 1) : 0;
+                const float* tab = p.scales + (size_t)task * p.N * p.G;
+                const float sa = __ldg(tab + (size_t)rowa * p.G + gg);
+                const float sb = has_b ? __ldg(tab + (size_t)rowb * p.G + gg) : 0.0f;
+                const float sx = e ? sv.z : sv.x, sbx = e ? sv.w : sv.y;
+                yv[nt][e] = fmaf(sa, acc[nt][e] - fmaf(za, sx, sbx), yv[nt][e]);
+                yv[nt][2 + e] = fmaf(sb, acc[nt][2 + e] - fmaf(zb, sx, sbx), yv[nt][2 + e]);
+              }
+            }
+          }
+#pragma unroll
+          for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) acc[nt][e] = 0.0f;
+        };
+
+        const uint32_t* fa = reinterpret_cast<const uint32_t*>(w.a);
+        const uint32_t* fb = reinterpret_cast<const uint32_t*>(w.b);
+        const uint8_t* x0 = xl + (size_t)tl * (kStepCols * 2);
+        const uint8_t* x1 = xh + (size_t)tl * (kStepCols * 2);
+#pragma unroll
+        for (int s = 0; s < 4; ++s) {
+          uint32_t wa[BITS], wb[BITS];
+#pragma unroll
+          for (int e = 0; e < BITS; ++e) {
+            wa[e] = fa[s * BITS + e];
+            wb[e] = fb[s * BITS + e];
+          }
+          const uint8_t* xs0 = x0 + s * 256;
+          const uint8_t* xs1 = x1 + s * 256;
+          if (has_b) {
+            run_mma2<BITS, NT, true, 0>(wa, wb, xs0, xs1, acc);
+            run_mma2<BITS, NT, true, 1>(wa, wb, xs0, xs1, acc);
+            if (GROUPED && RUNS_PER_GROUP == 2) flush(2 * s);
+            run_mma2<BITS, NT, true, 2>(wa, wb, xs0, xs1, acc);
+            run_mma2<BITS, NT, true, 3>(wa, wb, xs0, xs1, acc);
+          } else {
+            run_mma2<BITS, NT, false, 0>(wa, wb, xs0, xs1, acc);
+            run_mma2<BITS, NT, false, 1>(wa, wb, xs0, xs1, acc);
+            if (GROUPED && RUNS_PER_GROUP == 2) flush(2 * s);
+            run_mma2<BITS, NT, false, 2>(wa, wb, xs0, xs1, acc);
+            run_mma2<BITS, NT, false, 3>(wa, wb, xs0, xs1, acc);
+          }
+          if (GROUPED && RUNS_PER_GROUP == 2) flush(2 * s + 1);
+          if (GROUPED && RUNS_PER_GROUP == 4) flush(s);
+          if (GROUPED && RUNS_PER_GROUP == 8 && (s & 1)) flush(s >> 1);
+        }
+        ++lin;
+        if (++tl == spc_c) {
+          tl = 0;
+          ++lp;
+        }
       }
+    }
+    if (cur_pair >= 0) park();
+    __syncthreads();
+
+    // ---- add the parked sums of every pair in warp order
+    const bool last = ch + 1 == p.nchunks;
+    for (int idx = threadIdx.x; idx < npairs * 16 * p.M; idx += kPThreads) {
+      const int lp = idx / (16 * p.M);
+      const int rem = idx - lp * 16 * p.M;
+      const int m = rem >> 4, lr = rem & 15;
+      if (!pair_full(lp) && lr >= 8) continue;                     // a half pair has eight rows
+      float sum = 0.0f;
+      for (int w = 0; w < kPWarps; ++w) {
+        const int wl = bound(w, spc_c), wh = bound(w + 1, spc_c);
+        if (wl >= wh) continue;
+        const int sg = lp - wl / spc_c;
+        if (sg < 0 || sg >= p.maxseg || lp > (wh - 1) / spc_c) continue;
+        sum += part[((size_t)(w * p.maxseg + sg) * 16 + lr) * toks + m];
+      }
+      const int row = pair_rg(lp) * 8 + lr;
+      if (!GROUPED) {
+        // the chunk lies inside one group: take its zero-point and bias terms off, then scale
+        float sx = 0.0f, sb = 0.0f;
+        for (int w = 0; w < kPWarps; ++w) {
+          sx += sums[(w * TOKP + m) * 2];
+          sb += sums[(w * TOKP + m) * 2 + 1];
+        }
+        const int gg = p.G == 1 ? 0 : col0 / (p.K / p.G);
+        const float z = (float)__ldg(p.zeros + (size_t)row * p.G + gg);
+        sum -= fmaf(z, sx, sb);
+        const float* tab = p.scales;
+        if (p.task_ids) tab += (size_t)min(max(__ldg(p.task_ids + m), 0), p.n_tasks - 1) * p.N * p.G;
+        sum *= __ldg(tab + (size_t)row * p.G + gg);
+      }
+      if (p.nchunks > 1) {
+        float* ya = yacc + ((size_t)lp * 16 + lr) * toks + m;
+        if (ch > 0) sum += *ya;
+        if (!last) {
+          *ya = sum;
+          continue;
+        }
+      }
+      p.Y[(size_t)m * p.N + row] = __float2bfloat16_rn(sum);
+    }
+  }
+
+  if (!ok || abort_flag[0]) {
+    // let copies already in flight land before shared memory is released
+    for (int i = 0; i < 64; ++i) __nanosleep(1000);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      atomicExch(p.status, (int)PEQA_ERR_DEVICE_TIMEOUT);
+      p.status[1] = (int)blockIdx.x;
     }
   }
 }
 
 // ------------------------------------------------------------- prepare / unprepare
-// One thread per (row, 32-column run): moves the run's words between the two layouts and
-// permutes the codes inside it.  TO_PREPARED: canonical -> prepared, else the inverse.
+// One thread per (row group, step, lane, string): moves the string's 32 codes between the
+// two layouts.  TO_PREPARED: canonical -> prepared, else the inverse.
 template <int BITS, bool TO_PREPARED>
 __global__ void prep_layout_kernel(const uint32_t* __restrict__ src, uint32_t* __restrict__ dst,
-                                   int N, int K) {
-  const int runs = K / 32, U = K / 128;
+                                   int N, int K, int T) {
   const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (idx >= (size_t)N * runs) return;
-  const int row = (int)(idx / runs), run = (int)(idx - (size_t)row * runs);
-  const int u = run >> 2, s = run & 3;
-  const int rg = row >> 3, r = row & 7;
-  const uint32_t* canon = (TO_PREPARED ? src : dst) + (size_t)row * (K * BITS / 32) + (size_t)run * BITS;
-  uint32_t* canon_w = const_cast<uint32_t*>(canon);
+  const int rgs = N / 8, rgs2 = (rgs + 1) & ~1;      // the buffer holds whole pairs of row groups
+  const size_t total = (size_t)rgs2 * T * 128;
+  if (idx >= total) return;
+  const int s = (int)(idx & 3), lane = (int)((idx >> 2) & 31);
+  const size_t rt = idx >> 7;
+  const int t = (int)(rt % T), rg = (int)(rt / T);
+  const size_t blk = ((size_t)(rg >> 1) * T + t) * 2 + (rg & 1);
+  const int r8 = lane >> 2, c4 = lane & 3;
+  const int row = rg * 8 + r8;
+  // word e of string s of this lane: word index wi = s*BITS + e of the lane's 4*BITS words
   auto prep_word = [&](int e) -> size_t {
     const int wi = s * BITS + e;
     const int c = wi >> 2, wo = wi & 3;
-    return ((((size_t)rg * BITS + c) * U + u) * 8 + r) * 4 + wo;
+    return ((blk * BITS + c) * 32 + lane) * 4 + wo;
   };
-  uint32_t in[BITS], out[BITS];
+  if (rg >= rgs) {                                   // the missing half of the last pair
+    if (TO_PREPARED) {
 #pragma unroll
-  for (int e = 0; e < BITS; ++e) {
-    in[e] = TO_PREPARED ? canon[e] : src[prep_word(e)];
-    out[e] = 0u;
+      for (int e = 0; e < BITS; ++e) dst[prep_word(e)] = 0u;
+    }
+    return;
   }
-  auto get = [&](int pos) -> uint32_t {
-    const int bit = pos * BITS;
-    uint32_t v = in[bit >> 5] >> (bit & 31);
-    if ((bit & 31) + BITS > 32) v |= in[(bit >> 5) + 1] << (32 - (bit & 31));
+  const int wpr = K * BITS / 32;
+  const uint32_t* canon_r = (TO_PREPARED ? src : dst) + (size_t)row * wpr;
+  uint32_t* canon_w = dst + (size_t)row * wpr;
+  // code of column j of a canonical row
+  auto canon_get = [&](int j) -> uint32_t {
+    const int bit = j * BITS;
+    uint32_t v = canon_r[bit >> 5] >> (bit & 31);
+    if ((bit & 31) + BITS > 32) v |= canon_r[(bit >> 5) + 1] << (32 - (bit & 31));
     return v & ((1u << BITS) - 1u);
   };
-  auto put = [&](int pos, uint32_t code) {
+  uint32_t str[BITS];
+#pragma unroll
+  for (int e = 0; e < BITS; ++e) str[e] = TO_PREPARED ? 0u : src[prep_word(e)];
+  auto str_get = [&](int pos) -> uint32_t {
     const int bit = pos * BITS;
-    out[bit >> 5] |= code << (bit & 31);
-    if ((bit & 31) + BITS > 32) out[(bit >> 5) + 1] |= code >> (32 - (bit & 31));
+    uint32_t v = str[bit >> 5] >> (bit & 31);
+    if ((bit & 31) + BITS > 32) v |= str[(bit >> 5) + 1] << (32 - (bit & 31));
+    return v & ((1u << BITS) - 1u);
   };
+  auto str_put = [&](int pos, uint32_t code) {
+    const int bit = pos * BITS;
+    str[bit >> 5] |= code << (bit & 31);
+    if ((bit & 31) + BITS > 32) str[(bit >> 5) + 1] |= code >> (32 - (bit & 31));
+  };
+  if (TO_PREPARED) {
 #pragma unroll
-  for (int k = 0; k < 16; ++k) {
-    const int lo = dq::stream_lo(BITS, k), hi = dq::stream_hi(BITS, k);
-    if (TO_PREPARED) {
-      put(lo, get(2 * k));
-      put(hi, get(2 * k + 1));
-    } else {
-      put(2 * k, get(lo));
-      put(2 * k + 1, get(hi));
+    for (int k = 0; k < 16; ++k) {
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const int cs = 2 * k + h;
+        const int col = t * kStepCols + 32 * (4 * s + (cs >> 3)) + 8 * c4 + (cs & 7);
+        const uint32_t code = col < K ? canon_get(col) : 0u;
+        str_put(h ? dq::stream_hi(BITS, k) : dq::stream_lo(BITS, k), code);
+      }
     }
-  }
 #pragma unroll
-  for (int e = 0; e < BITS; ++e) {
-    if (TO_PREPARED) dst[prep_word(e)] = out[e];
-    else canon_w[e] = out[e];
+    for (int e = 0; e < BITS; ++e) dst[prep_word(e)] = str[e];
+  } else {
+    // the eight columns of a run this lane owns are BITS whole bytes of the canonical row
+    uint8_t* rowb = reinterpret_cast<uint8_t*>(canon_w);
+#pragma unroll
+    for (int rr = 0; rr < 4; ++rr) {
+      const int col = t * kStepCols + 32 * (4 * s + rr) + 8 * c4;
+      if (col >= K) continue;
+      uint32_t bits8 = 0u;
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        const int cs = 8 * rr + e, k = cs >> 1;
+        const uint32_t code = str_get((cs & 1) ? dq::stream_hi(BITS, k) : dq::stream_lo(BITS, k));
+        bits8 |= code << (BITS * e);
+      }
+      uint8_t* o = rowb + (size_t)col * BITS / 8;
+#pragma unroll
+      for (int b = 0; b < BITS; ++b) o[b] = (uint8_t)(bits8 >> (8 * b));
+    }
   }
 }
 
 struct PrepPlan {
-  int rg_per_cta, grid, S, PG, rounds, chunk_units, nchunks, ups, spr, x_pitch, pairs;
+  int rg_per_cta, grid, T, spc, nchunks, slots, sps, maxseg, x_pitch, pairs;
   size_t smem;
 };
 
-int x_pitch_for(int units) {
-  const int raw = units * kPUnitPitch;
-  return raw + ((64 - raw % 128) % 128 + 128) % 128;              // pitch % 128 == 64
+int x_pitch_for(int steps) {
+  const int raw = steps * kStepCols * 2;
+  return raw + 64;                                                // pitch % 128 == 64
 }
 
-// Chooses the split of the sixteen warps (PG pairs x S splits) and the units of K staged at a
-// time so that the warps' step counts are equal and as small as possible.
-int plan_prep(int N, int K, int M, PrepPlan* plan) {
-  int sms = 0, dev = 0;
-  PEQA_CUDA(cudaGetDevice(&dev));
-  PEQA_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-  const int rgs = N / 8, U = K / 128;
+// Chooses how many steps of activations are staged at a time and the shape of the warps'
+// rings.  gcols: columns of one quantization group.
+int plan_prep(int N, int K, int M, int bits, int gcols, PrepPlan* plan) {
+  const int sms = sm_count_or(148);
+  const int rgs = N / 8;
   const int NT = M <= 8 ? 1 : 2, TOKP = 8 * NT;
+  const int toks = (M + 1) & ~1;
+  const int step_bytes = 2 * bits * 512;
+  plan->T = (K + kStepCols - 1) / kStepCols;
   plan->rg_per_cta = (rgs + sms - 1) / sms;
   plan->grid = (rgs + plan->rg_per_cta - 1) / plan->rg_per_cta;
-  plan->pairs = (plan->rg_per_cta + 1) / 2;
-  const size_t fixed = 128 + (size_t)2 * kPWarps * 16 * TOKP * 4 + (size_t)plan->pairs * 16 * TOKP * 4 +
-                       (size_t)TOKP * 2 * 4 + 256 + 64;
-  long long best = -1;
-  for (int S = 1; S <= kPWarps; S *= 2) {
-    const int PG = kPWarps / S;
-    const int rounds = (plan->pairs + PG - 1) / PG;
-    // largest chunk that fits, a multiple of 4 * S units unless all of K fits
-    int cu = U;
-    while (cu > 0 && fixed + (size_t)M * x_pitch_for(cu) > (size_t)kPSmemLimit) --cu;
-    if (cu <= 0) continue;
-    if (cu < U) cu -= cu % (4 * S);
-    if (cu <= 0) continue;
-    long long cost = 0;
-    const int nchunks = (U + cu - 1) / cu;
-    for (int c = 0; c < nchunks; ++c) {
-      const int ups = (((cu + S - 1) / S + 3) / 4) * 4;
-      cost += (long long)rounds * (ups / 4) * 8 + rounds + 6;      // steps (x8), barriers, staging
-    }
-    if (best < 0 || cost < best) {
-      best = cost;
-      plan->S = S;
-      plan->PG = PG;
-      plan->rounds = rounds;
-      plan->chunk_units = cu;
-      plan->nchunks = nchunks;
-      plan->ups = (((cu + S - 1) / S + 3) / 4) * 4;
-      plan->spr = plan->ups / 4;
-      plan->x_pitch = x_pitch_for(cu);
-      plan->smem = fixed + (size_t)M * plan->x_pitch;
+  plan->pairs = plan->rg_per_cta / 2 + 2;                         // incl. a half pair at either end
+  const bool grouped = gcols < kStepCols;
+  const int gps = grouped ? kStepCols / gcols : 0;
+  auto need = [&](int spc, int slots, int sps, int* maxseg) -> size_t {
+    const int nch = (plan->T + spc - 1) / spc;
+    // a warp's share of a chunk is at most `cost` units (a full pair-step costs 2): it touches
+    // at most ceil(cost / (2 * spc)) + 1 full pairs and the half pairs at the ends
+    const int cost = (2 * plan->pairs * spc + kPWarps - 1) / kPWarps + 1;
+    *maxseg = (cost + 2 * spc - 1) / (2 * spc) + 3;
+    if (*maxseg > plan->pairs) *maxseg = plan->pairs;
+    size_t b = 128 + kPHeadBytes;
+    b += (size_t)kPWarps * (*maxseg) * 16 * toks * 4;
+    if (nch > 1) b += (size_t)plan->pairs * 16 * toks * 4;
+    b += (size_t)(grouped ? spc * gps : kPWarps) * TOKP * 2 * 4 + 128;
+    b += (((size_t)M * x_pitch_for(spc)) + 127) / 128 * 128;
+    b += (size_t)kPWarps * slots * sps * step_bytes;
+    return b;
+  };
+  // a chunk must lie inside one quantization group unless the groups are applied per step
+  const int steps_per_group = grouped ? 1 : gcols / kStepCols;     // one group per row: >= T
+  const bool one_group = gcols >= K;
+  // ring shapes in order of preference: bytes in flight first, larger copies on a tie
+  const int shapes[5][2] = {{2, 2}, {4, 1}, {3, 1}, {2, 1}, {1, 1}};   // {slots, steps per slot}
+  int seg = 0;
+  plan->spc = 0;
+  // all of K staged at once, with the best ring that fits ...
+  if (grouped || one_group) {
+    for (int i = 0; i < 4 && plan->spc == 0; ++i)
+      if (need(plan->T, shapes[i][0], shapes[i][1], &seg) <= (size_t)kPSmemLimit) {
+        plan->spc = plan->T;
+        plan->slots = shapes[i][0];
+        plan->sps = shapes[i][1];
+      }
+  }
+  // ... else the largest chunk of steps beside a ring of two single steps
+  if (plan->spc == 0) {
+    for (int spc = plan->T; spc >= 1 && plan->spc == 0; --spc) {
+      if (!grouped && !one_group && (steps_per_group % spc) != 0) continue;
+      if (need(spc, 2, 1, &seg) <= (size_t)kPSmemLimit) {
+        plan->spc = spc;
+        plan->slots = 2;
+        plan->sps = 1;
+      }
     }
   }
-  return best < 0 ? PEQA_ERR_TOO_LARGE : PEQA_OK;
+  if (plan->spc == 0) return PEQA_ERR_TOO_LARGE;
+  plan->nchunks = (plan->T + plan->spc - 1) / plan->spc;
+  plan->x_pitch = x_pitch_for(plan->spc);
+  plan->smem = need(plan->spc, plan->slots, plan->sps, &seg);
+  plan->maxseg = seg;
+  return PEQA_OK;
 }
 
-template <int BITS, int NT>
+template <int BITS, int NT, int GSH>
 int launch_prep_t(const PrepParams& p, int grid, size_t smem, cudaStream_t st) {
-  auto kern = decode_prep_kernel<BITS, NT>;
+  auto kern = decode_prep_kernel<BITS, NT, GSH>;
   PEQA_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(grid, 1, 1);
@@ -477,11 +770,27 @@ int launch_prep_t(const PrepParams& p, int grid, size_t smem, cudaStream_t st) {
   return PEQA_OK;
 }
 
+template <int BITS, int NT>
+int launch_prep_g(const PrepParams& p, int gsh, int grid, size_t smem, cudaStream_t st) {
+  switch (gsh) {
+    case 1: return launch_prep_t<BITS, NT, 1>(p, grid, smem, st);
+    case 2: return launch_prep_t<BITS, NT, 2>(p, grid, smem, st);
+    case 3: return launch_prep_t<BITS, NT, 3>(p, grid, smem, st);
+    default: return launch_prep_t<BITS, NT, 0>(p, grid, smem, st);
+  }
+}
+
 int check_prep_layer(const peqa_qweight_t* w) {
   if (!w) return PEQA_ERR_NULL;
   PEQA_TRY(check_bits_shape(w->out_features, w->in_features, w->bits, w->group_size));
   if (w->in_features % 128 != 0 || w->out_features % 8 != 0) return PEQA_ERR_BAD_SHAPE;
   return PEQA_OK;
+}
+
+// Group sizes the prepared kernel serves: one group per row, groups that are multiples of
+// 512 columns, and groups of 64, 128 or 256 columns.
+bool prep_group_supported(int K, int g) {
+  return g == K || g % kStepCols == 0 || g == 64 || g == 128 || g == 256;
 }
 
 }  // namespace
@@ -492,7 +801,9 @@ using namespace peqa;
 
 extern "C" size_t peqa_decode_prepared_bytes(const peqa_qweight_t* w) {
   if (check_prep_layer(w) != PEQA_OK) return 0;
-  return (size_t)w->out_features * w->in_features * w->bits / 8;
+  const size_t T = ((size_t)w->in_features + kStepCols - 1) / kStepCols;
+  const size_t rgs2 = ((size_t)w->out_features / 8 + 1) & ~(size_t)1;   // whole pairs of row groups
+  return rgs2 * T * w->bits * 512;
 }
 
 static int run_layout(const peqa_qweight_t* w, const uint32_t* src, uint32_t* dst, bool to_prepared,
@@ -500,16 +811,18 @@ static int run_layout(const peqa_qweight_t* w, const uint32_t* src, uint32_t* ds
   PEQA_TRY(check_prep_layer(w));
   if (!src || !dst) return PEQA_ERR_NULL;
   if (!aligned16(src) || !aligned16(dst)) return PEQA_ERR_ALIGNMENT;
-  const size_t n = (size_t)w->out_features * (w->in_features / 32);
+  const int T = (w->in_features + kStepCols - 1) / kStepCols;
+  const size_t n = (size_t)((w->out_features / 8 + 1) & ~1) * T * 128;
   const int threads = 256;
   const unsigned blocks = (unsigned)((n + threads - 1) / threads);
   cudaStream_t st = as_stream(stream);
+  const int N = w->out_features, K = w->in_features;
   if (w->bits == 3) {
-    if (to_prepared) prep_layout_kernel<3, true><<<blocks, threads, 0, st>>>(src, dst, w->out_features, w->in_features);
-    else prep_layout_kernel<3, false><<<blocks, threads, 0, st>>>(src, dst, w->out_features, w->in_features);
+    if (to_prepared) prep_layout_kernel<3, true><<<blocks, threads, 0, st>>>(src, dst, N, K, T);
+    else prep_layout_kernel<3, false><<<blocks, threads, 0, st>>>(src, dst, N, K, T);
   } else {
-    if (to_prepared) prep_layout_kernel<4, true><<<blocks, threads, 0, st>>>(src, dst, w->out_features, w->in_features);
-    else prep_layout_kernel<4, false><<<blocks, threads, 0, st>>>(src, dst, w->out_features, w->in_features);
+    if (to_prepared) prep_layout_kernel<4, true><<<blocks, threads, 0, st>>>(src, dst, N, K, T);
+    else prep_layout_kernel<4, false><<<blocks, threads, 0, st>>>(src, dst, N, K, T);
   }
   PEQA_CUDA(cudaGetLastError());
   return PEQA_OK;
@@ -531,7 +844,8 @@ extern "C" int peqa_qlinear_decode_prepared(const peqa_qweight_t* w, const uint3
                                             const int32_t* task_ids, void* stream) {
   PEQA_TRY(check_prep_layer(w));
   if (!prepared || !X || !Y || !w->zeros) return PEQA_ERR_NULL;
-  if (effective_group(w->in_features, w->group_size) != w->in_features) return PEQA_ERR_BAD_SHAPE;
+  const int g = effective_group(w->in_features, w->group_size);
+  if (!prep_group_supported(w->in_features, g)) return PEQA_ERR_BAD_SHAPE;
   if (M < 1 || M > 16) return PEQA_ERR_BAD_SHAPE;
   if (task_ids) {
     if (!scale_table) return PEQA_ERR_NULL;
@@ -542,9 +856,9 @@ extern "C" int peqa_qlinear_decode_prepared(const peqa_qweight_t* w, const uint3
   if (!aligned16(prepared) || !aligned16(X) || !aligned16(Y)) return PEQA_ERR_ALIGNMENT;
   PEQA_TRY(check_arch());
   PrepPlan plan;
-  PEQA_TRY(plan_prep(w->out_features, w->in_features, M, &plan));
+  PEQA_TRY(plan_prep(w->out_features, w->in_features, M, w->bits, g, &plan));
   PrepParams p;
-  p.P = reinterpret_cast<const uint4*>(prepared);
+  p.P = reinterpret_cast<const uint8_t*>(prepared);
   p.zeros = w->zeros;
   p.scales = task_ids ? scale_table : w->scales;
   p.X = static_cast<const __nv_bfloat16*>(X);
@@ -553,22 +867,25 @@ extern "C" int peqa_qlinear_decode_prepared(const peqa_qweight_t* w, const uint3
   p.n_tasks = n_tasks;
   p.N = w->out_features;
   p.K = w->in_features;
-  p.U = p.K / 128;
+  p.G = p.K / g;
   p.M = M;
   p.rgs = p.N / 8;
   p.rg_per_cta = plan.rg_per_cta;
-  p.S = plan.S;
-  p.PG = plan.PG;
-  p.rounds = plan.rounds;
-  p.chunk_units = plan.chunk_units;
+  p.T = plan.T;
+  p.spc = plan.spc;
   p.nchunks = plan.nchunks;
-  p.ups = plan.ups;
-  p.spr = plan.spr;
+  p.slots = plan.slots;
+  p.sps = plan.sps;
+  p.maxseg = plan.maxseg;
   p.x_pitch = plan.x_pitch;
   p.pairs_per_cta = plan.pairs;
   cudaStream_t st = as_stream(stream);
+  PEQA_TRY(status_word(st, &p.status));
+  const int gsh = g == 64 ? 1 : g == 128 ? 2 : g == 256 ? 3 : 0;
   const int NT = M <= 8 ? 1 : 2;
   if (w->bits == 3)
-    return NT == 1 ? launch_prep_t<3, 1>(p, plan.grid, plan.smem, st) : launch_prep_t<3, 2>(p, plan.grid, plan.smem, st);
-  return NT == 1 ? launch_prep_t<4, 1>(p, plan.grid, plan.smem, st) : launch_prep_t<4, 2>(p, plan.grid, plan.smem, st);
+    return NT == 1 ? launch_prep_g<3, 1>(p, gsh, plan.grid, plan.smem, st)
+                   : launch_prep_g<3, 2>(p, gsh, plan.grid, plan.smem, st);
+  return NT == 1 ? launch_prep_g<4, 1>(p, gsh, plan.grid, plan.smem, st)
+                 : launch_prep_g<4, 2>(p, gsh, plan.grid, plan.smem, st);
 }

@@ -268,3 +268,19 @@ def test_multitask_forward_rows_are_single_task_forwards():
         assert np.allclose(Y[m], table[ids[m]].astype(np.float64) * u[m], rtol=1e-12, atol=1e-12)
     same = oracle.fwd_multitask(d["X"], qw, zeros, table, np.zeros(T, int), 4)
     assert np.array_equal(same, oracle.fwd(d["X"], qw, zeros, scales, 4, 0))
+
+
+def test_multitask_forward_with_grouped_scales():
+    """Grouped task tables [n_tasks, N, G]: row m is the explicit fp64 product with the weight
+    s_task[i, g(j)] * (Q[i, j] - z[i, g(j)]) of its own task."""
+    T, N, K, g = 5, 6, 128, 32
+    d, codes, zeros, scales, qw = _case(43, N, K, T, 3, g)
+    rng = np.random.default_rng(5)
+    table = (scales[None] * rng.uniform(0.5, 2.0, size=(3, N, K // g))).astype(np.float32)
+    ids = np.array([1, 2, 0, 1, 1])
+    Y = oracle.fwd_multitask(d["X"], qw, zeros, table, ids, 3, g)
+    X = _f(d["X"])
+    centred = codes.astype(np.float64) - np.repeat(zeros.astype(np.float64), g, axis=1)
+    for m in range(T):
+        W_hat = np.repeat(table[ids[m]].astype(np.float64), g, axis=1) * centred
+        assert np.allclose(Y[m], W_hat @ X[m], rtol=1e-12, atol=1e-12)
