@@ -269,6 +269,8 @@ class Linear:
         self.v = torch.zeros((self.N, self.G), dtype=torch.float32, device=dev)
         self.dS = torch.empty((self.N, self.G), dtype=torch.float32, device=dev)
         self.Yd = torch.empty((1, self.N), dtype=torch.bfloat16, device=dev)
+        # Q is frozen (Sec. 3.3): the copy the decode kernel streams is prepared once, here
+        self.prep = binding.decode_prepare(self.qw) if binding.decode_prepared_supported(self.qw) else None
         self.ws = binding.alloc_workspace(binding.OP_BWD, self.T, self.qw)
 
 
@@ -292,6 +294,8 @@ def run_stage(binding, L, k, Y, dX, step_no):
     elif k == 3:
         binding.qlinear_bwd_ds_adamw(L.qw, L.X, L.dY, L.m, L.v, LR, BETA1, BETA2, EPS, WD, step_no,
                                      dS=L.dS, workspace=L.ws)
+    elif L.prep is not None:
+        binding.qlinear_decode_prepared(L.qw, L.prep, L.X[:1], L.Yd)
     else:
         binding.qlinear_decode(L.qw, L.X[:1], L.Yd)
 
@@ -582,18 +586,30 @@ def bench_decode(torch, binding, dev, peaks, reps=30, shapes=None):
                             "frac_measured_hbm": wbytes / (us * 1e-6) / 1e9 / peaks["hbm_gbs"], "clocks": clk}
         preps = [binding.decode_prepare(qw) for qw in qws]
         torch.cuda.synchronize()
-        for M in (1, 4, 16):
+
+        def time_both(qws_, M, G, into, prefix):
             X = torch.randn((M, K), device=dev, generator=gen).to(torch.bfloat16)
             Y = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
-            ws = binding.alloc_workspace(binding.OP_DECODE, M, qws[0])
-            nbytes = wbytes + N * 5 + M * K * 2 + M * N * 2
-            for key, fn in (("prepared", lambda i: binding.qlinear_decode_prepared(qws[i], preps[i], X, Y)),
-                            ("canonical", lambda i: binding.qlinear_decode(qws[i], X, Y, workspace=ws))):
+            ws = binding.alloc_workspace(binding.OP_DECODE, M, qws_[0])
+            nbytes = wbytes + N * G * 5 + M * K * 2 + M * N * 2
+            for key, fn in (("prepared", lambda i: binding.qlinear_decode_prepared(qws_[i], preps[i], X, Y)),
+                            ("canonical", lambda i: binding.qlinear_decode(qws_[i], X, Y, workspace=ws))):
                 us, clk = timed(fn)
                 gbs = nbytes / (us * 1e-6) / 1e9
-                rec[f"M{M}_{key}"] = {"us": us, "GB/s": gbs, "frac_measured_hbm": gbs / peaks["hbm_gbs"],
-                                      "frac_nominal_8000": gbs / NOMINAL_HBM_GBS, "bytes": nbytes,
-                                      "frac_of_bare_read_time": rec["bare_read"]["us"] / us, "clocks": clk}
+                into[f"{prefix}M{M}_{key}"] = {"us": us, "GB/s": gbs, "frac_measured_hbm": gbs / peaks["hbm_gbs"],
+                                               "frac_nominal_8000": gbs / NOMINAL_HBM_GBS, "bytes": nbytes,
+                                               "frac_of_bare_read_time": rec["bare_read"]["us"] / us, "clocks": clk}
+
+        for M in (1, 4, 16):
+            time_both(qws, M, 1, rec, "")
+        # the same matrices with scales in groups of 64 columns (the LLaMA-65B layer workload's setting)
+        G64 = K // 64
+        z64 = torch.full((N, G64), 3, dtype=torch.uint8, device=dev)
+        s64 = torch.full((N, G64), 0.01, dtype=torch.float32, device=dev)
+        qws64 = [binding.QWeight(3, N, K, 64, q, z64, s64) for q in qs]
+        for M in (1, 4):
+            time_both(qws64, M, G64, rec, "g64_")
+        del qws64, z64, s64
         del preps
         binding.check_status()
         res[name] = rec
@@ -679,9 +695,11 @@ def render_md(path):
         for name, rec in doc["decode"].items():
             b = rec["bare_read"]
             for key, v in rec.items():
-                if not key.startswith("M"):
+                if not (key.startswith("M") or key.startswith("g64_M")):
                     continue
-                o.append(f"| {name} {key.split('_')[1]} | {b['us']:.1f} ({b['GB/s']:.0f}) | {key[1:].split('_')[0]} | {v['us']:.1f} | "
+                grp = "g64 " if key.startswith("g64_") else ""
+                key = key[4:] if key.startswith("g64_") else key
+                o.append(f"| {name} {grp}{key.split('_')[1]} | {b['us']:.1f} ({b['GB/s']:.0f}) | {key[1:].split('_')[0]} | {v['us']:.1f} | "
                          f"{v['GB/s']:.0f} | {v['frac_measured_hbm']:.2f} | {v['frac_nominal_8000']:.2f} | "
                          f"{v['frac_of_bare_read_time']:.2f} |")
     if doc.get("cpu_baseline"):

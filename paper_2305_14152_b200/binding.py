@@ -375,6 +375,13 @@ def decode_prepared_bytes(w: QWeight) -> int:
     return int(lib().peqa_decode_prepared_bytes(ctypes.byref(cs)))
 
 
+def decode_prepared_supported(w: QWeight) -> bool:
+    """True when qlinear_decode_prepared serves this layer: K % 128 == 0, N % 8 == 0 and one scale
+    per channel, groups of 64, 128 or 256 columns, or groups that are multiples of 512 columns."""
+    g = w.group_size or w.K
+    return decode_prepared_bytes(w) > 0 and (g == w.K or g % 512 == 0 or g in (64, 128, 256))
+
+
 def decode_prepare(w: QWeight) -> torch.Tensor:
     """Prepared copy of w.qweight for qlinear_decode_prepared (int32 bit patterns, flat)."""
     n = decode_prepared_bytes(w)

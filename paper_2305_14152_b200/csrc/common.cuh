@@ -105,6 +105,51 @@ __device__ __forceinline__ void adamw_update(float& s, float gr, float& m, float
 }
 #endif
 
+// Work items of the CTA-pair kernels (forward, dX).  A tile is 512 tokens x 256 outputs held as
+// two accumulators of 256 tokens.  Tiles are dealt round-robin to the pairs; when the last round
+// would keep at most half of the pairs busy, its tiles are cut into two items of 256 tokens each,
+// so that round takes about half as long.  Items [0, full_items) are whole tiles, the rest are
+// halves: item full_items + 2*i + h is half h of tile full_items + i.
+struct PairItems {
+  int o_tiles;       // 256-wide tiles along the output dimension
+  int full_items;    // items that are whole tiles
+  int total_items;
+};
+inline PairItems make_pair_items(int o_tiles, int t_tiles, int T, int pairs) {
+  PairItems it;
+  const int tiles = o_tiles * t_tiles;
+  it.o_tiles = o_tiles;
+  it.full_items = tiles;
+  it.total_items = tiles;
+  const int rem = pairs > 0 ? tiles % pairs : 0;
+  if (T % 512 == 0 && tiles > pairs && rem > 0 && 2 * rem <= pairs) {
+    it.full_items = tiles - rem;
+    it.total_items = tiles + rem;
+  }
+  return it;
+}
+#ifdef __CUDACC__
+// Output tile, first token and token blocks (1 or 2) of an item.
+__device__ __forceinline__ void pair_item(const PairItems& it, int item, int T, int& o_tile, int& tt0,
+                                          int& blocks) {
+  int tile = item, half = -1;
+  if (item >= it.full_items) {
+    const int h = item - it.full_items;
+    tile = it.full_items + (h >> 1);
+    half = h & 1;
+  }
+  const int t_tile = tile / it.o_tiles;
+  o_tile = tile - t_tile * it.o_tiles;
+  tt0 = t_tile * 512;
+  if (half >= 0) {
+    tt0 += half * 256;
+    blocks = 1;
+  } else {
+    blocks = tt0 + 256 < T ? 2 : 1;
+  }
+}
+#endif
+
 // Entry points implemented in the individual translation units.
 // zeros_f != nullptr: real-valued zero-points [N, G] (App. K) replace w->zeros
 int launch_fwd(const peqa_qweight_t* w, const float* zeros_f, int g, const void* X, int T, void* Y,

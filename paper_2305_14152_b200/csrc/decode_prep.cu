@@ -73,7 +73,8 @@ constexpr int kPSmemLimit = 227 * 1024;
 constexpr int kPMaxSlots = 4;
 constexpr int kStepCols = 512;
 constexpr int kPBarBytes = kPWarps * kPMaxSlots * 8;              // the warps' mbarriers
-constexpr int kPHeadBytes = kPBarBytes + 128;                     // + abort flag and wait limit
+// + abort flag, wait limit and, per warp, the bounds of its steps and its first and last pair
+constexpr int kPHeadBytes = (kPBarBytes + 32 + 3 * (kPWarps + 1) * 4 + 127) / 128 * 128;
 
 struct PrepParams {
   const uint8_t* P;         // prepared weights
@@ -184,6 +185,9 @@ decode_prep_kernel(const PrepParams p) {
                                              ~static_cast<uintptr_t>(127));
   uint64_t* bars = reinterpret_cast<uint64_t*>(base);                        // [warps][kPMaxSlots]
   volatile int* abort_flag = reinterpret_cast<volatile int*>(base + kPBarBytes);   // [0] flag, [1] limit
+  int* wbound = const_cast<int*>(abort_flag) + 8;                            // [warps + 1] bounds of the chunk
+  int* wfirst = wbound + kPWarps + 1;                                        // [warps] first pair of the range
+  int* wlast = wfirst + kPWarps + 1;                                         // [warps] last pair, -1: no steps
   const int toks = (p.M + 1) & ~1;                                           // tokens kept of a tile
   float* part = reinterpret_cast<float*>(base + kPHeadBytes);                // [warps][maxseg][16][toks]
   float* yacc = part + (size_t)kPWarps * p.maxseg * 16 * toks;               // [pairs][16][toks]
@@ -303,72 +307,85 @@ decode_prep_kernel(const PrepParams p) {
     const int col0 = ch * p.spc * kStepCols;                       // first column of the chunk
     const int ccols = min(p.K - col0, spc_c * kStepCols);          // real columns in it
     if (ch > 0) __syncthreads();                                   // the previous chunk is no longer read
-    // ---- stage X[:, chunk] (columns beyond K read as zero)
+    // ---- stage X[:, chunk] (columns beyond K read as zero) and take, per token, the sum of x
+    // and the sum of bias * x: per group (a thread stages and sums whole groups), or over the
+    // pieces this thread staged itself, added up per warp (the warps' shares are added in
+    // warp order when the rows are finished)
     const int pieces = spc_c * (kStepCols / 8);                    // 16-byte pieces per token
-    for (int idx = threadIdx.x; idx < p.M * pieces; idx += kPThreads) {
-      const int m = idx / pieces, pc = idx - m * pieces;
+    if (threadIdx.x <= kPWarps) {
+      const int wl = bound(threadIdx.x, spc_c);
+      wbound[threadIdx.x] = wl;
+      if (threadIdx.x < kPWarps) {
+        const int wh = bound(threadIdx.x + 1, spc_c);
+        wfirst[threadIdx.x] = wl / spc_c;
+        wlast[threadIdx.x] = wh > wl ? (wh - 1) / spc_c : -1;
+      }
+    }
+    // bias of the two columns in word e of a piece whose run in the step is run % 4 == rq
+    auto piece_sums = [&](const uint8_t* ptr, int rq, float& sx, float& sb) {
+      const uint4 v = *reinterpret_cast<const uint4*>(ptr);
+      const uint32_t wv[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float lo = __uint_as_float(wv[e] << 16), hi = __uint_as_float(wv[e] & 0xFFFF0000u);
+        sx += lo + hi;
+        float b0 = 128.0f, b1 = 128.0f;
+        if (BITS == 3) {
+          const bool alt = (dq::stream_alt_mask3() >> (4 * rq + e)) & 1u;
+          b0 = alt ? 64.0f : 8.0f;
+          b1 = alt ? 16.0f : 128.0f;
+        }
+        sb = fmaf(b0, lo, sb);
+        sb = fmaf(b1, hi, sb);
+      }
+    };
+    auto stage_piece = [&](int m, int pc) {
       uint8_t* dst = xs + (size_t)m * p.x_pitch + pc * 16;
       if (pc * 8 < ccols) cp_async_16(smem_u32(dst), p.X + (size_t)m * p.K + col0 + pc * 8);
       else *reinterpret_cast<uint4*>(dst) = make_uint4(0u, 0u, 0u, 0u);
-    }
-    asm volatile("cp.async.wait_all;" ::: "memory");
-    __syncthreads();
-    // ---- sum of x and sum of bias * x: per token and group, or per token and warp
-    {
-      // bias of the two columns in word e of a piece whose run in the step is run % 4 == rq
-      auto piece_sums = [&](const uint8_t* ptr, int rq, float& sx, float& sb) {
-        const uint4 v = *reinterpret_cast<const uint4*>(ptr);
-        const uint32_t wv[4] = {v.x, v.y, v.z, v.w};
+    };
+    if (GROUPED) {
+      const int ngr = spc_c * GPS;
+      constexpr int gpieces = RUNS_PER_GROUP * 4;                  // 16-byte pieces per group
+      for (int idx = threadIdx.x; idx < ngr * p.M; idx += kPThreads) {
+        const int gi = idx / p.M, m = idx - gi * p.M;
+        for (int pc = 0; pc < gpieces; ++pc) stage_piece(m, gi * gpieces + pc);
+      }
+      asm volatile("cp.async.wait_all;" ::: "memory");
+      for (int idx = threadIdx.x; idx < ngr * p.M; idx += kPThreads) {
+        const int gi = idx / p.M, m = idx - gi * p.M;
+        const uint8_t* row = xs + (size_t)m * p.x_pitch + (size_t)gi * gpieces * 16;
+        float sx = 0.0f, sb = 0.0f;
+        for (int pc = 0; pc < gpieces; ++pc)
+          piece_sums(row + pc * 16, (gi * RUNS_PER_GROUP + (pc >> 2)) & 3, sx, sb);
+        sums[((size_t)gi * TOKP + m) * 2] = sx;
+        sums[((size_t)gi * TOKP + m) * 2 + 1] = sb;
+      }
+    } else {
+      // piece pc of a token goes to thread pc % 512: its run % 4 is the same for all of them
+      for (int m = 0; m < p.M; ++m)
+        for (int pc = threadIdx.x; pc < pieces; pc += kPThreads) stage_piece(m, pc);
+      asm volatile("cp.async.wait_all;" ::: "memory");
+      for (int m = 0; m < p.M; ++m) {
+        float sx = 0.0f, sb = 0.0f;
+        const uint8_t* row = xs + (size_t)m * p.x_pitch;
+        for (int pc = threadIdx.x; pc < pieces; pc += kPThreads)
+          piece_sums(row + pc * 16, (threadIdx.x >> 2) & 3, sx, sb);
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const float lo = __uint_as_float(wv[e] << 16), hi = __uint_as_float(wv[e] & 0xFFFF0000u);
-          sx += lo + hi;
-          float b0 = 128.0f, b1 = 128.0f;
-          if (BITS == 3) {
-            const bool alt = (dq::stream_alt_mask3() >> (4 * rq + e)) & 1u;
-            b0 = alt ? 64.0f : 8.0f;
-            b1 = alt ? 16.0f : 128.0f;
-          }
-          sb = fmaf(b0, lo, sb);
-          sb = fmaf(b1, hi, sb);
+        for (int o = 16; o > 0; o >>= 1) {
+          sx += __shfl_xor_sync(0xffffffffu, sx, o);
+          sb += __shfl_xor_sync(0xffffffffu, sb, o);
         }
-      };
-      if (GROUPED) {
-        const int ngr = spc_c * GPS;
-        constexpr int gpieces = RUNS_PER_GROUP * 4;                // 16-byte pieces per group
-        for (int idx = threadIdx.x; idx < ngr * p.M; idx += kPThreads) {
-          const int gi = idx / p.M, m = idx - gi * p.M;
-          const uint8_t* row = xs + (size_t)m * p.x_pitch + (size_t)gi * gpieces * 16;
-          float sx = 0.0f, sb = 0.0f;
-          for (int pc = 0; pc < gpieces; ++pc)
-            piece_sums(row + pc * 16, (gi * RUNS_PER_GROUP + (pc >> 2)) & 3, sx, sb);
-          sums[((size_t)gi * TOKP + m) * 2] = sx;
-          sums[((size_t)gi * TOKP + m) * 2 + 1] = sb;
+        if (lane == 0) {
+          sums[(warp * TOKP + m) * 2] = sx;
+          sums[(warp * TOKP + m) * 2 + 1] = sb;
         }
-        __syncthreads();
-      } else {
-        // piece pc of a token goes to thread pc % 512: its run % 4 is the same for all of them
-        for (int m = 0; m < p.M; ++m) {
-          float sx = 0.0f, sb = 0.0f;
-          const uint8_t* row = xs + (size_t)m * p.x_pitch;
-          for (int pc = threadIdx.x; pc < pieces; pc += kPThreads)
-            piece_sums(row + pc * 16, (threadIdx.x >> 2) & 3, sx, sb);
-#pragma unroll
-          for (int o = 16; o > 0; o >>= 1) {
-            sx += __shfl_xor_sync(0xffffffffu, sx, o);
-            sb += __shfl_xor_sync(0xffffffffu, sb, o);
-          }
-          if (lane == 0) {
-            sums[(warp * TOKP + m) * 2] = sx;
-            sums[(warp * TOKP + m) * 2 + 1] = sb;
-          }
-        }
-        // read after the barrier that follows the main loop
       }
     }
+    __syncthreads();
 
     // ---- this warp's steps of the chunk
-    const int lo = bound(warp, spc_c), hi = bound(warp + 1, spc_c);
+    const int lo = wbound[warp], hi = wbound[warp + 1];
     int seg = 0, cur_pair = -1;
     float acc[NT][4], yv[NT][4];
 #pragma unroll
@@ -547,10 +564,8 @@ decode_prep_kernel(const PrepParams p) {
       if (!pair_full(lp) && lr >= 8) continue;                     // a half pair has eight rows
       float sum = 0.0f;
       for (int w = 0; w < kPWarps; ++w) {
-        const int wl = bound(w, spc_c), wh = bound(w + 1, spc_c);
-        if (wl >= wh) continue;
-        const int sg = lp - wl / spc_c;
-        if (sg < 0 || sg >= p.maxseg || lp > (wh - 1) / spc_c) continue;
+        const int sg = lp - wfirst[w];
+        if (sg < 0 || sg >= p.maxseg || lp > wlast[w]) continue;
         sum += part[((size_t)(w * p.maxseg + sg) * 16 + lr) * toks + m];
       }
       const int row = pair_rg(lp) * 8 + lr;

@@ -66,6 +66,7 @@ struct DxParams {
   __nv_bfloat16* out;   // dX [T, K]
   int N, K, G, g, g_shift, T;
   int j_tiles, t_tiles, k_blocks;   // 256-column tiles, 512-token tiles, 64-row stages over N
+  PairItems items;
   int* status;
 };
 
@@ -115,7 +116,7 @@ qdx_pair_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_consta
   cluster_sync_all();
   tc_fence_after();
   const uint32_t tmem_base = bars->tmem_base;
-  const int total_tiles = p.j_tiles * p.t_tiles;
+  const int total_tiles = p.items.total_items;      // work items: whole tiles, then halves
   const int pair = blockIdx.x >> 1;
   const int n_pairs = gridDim.x >> 1;
   const int my_tiles = (total_tiles - pair + n_pairs - 1) / n_pairs;
@@ -126,8 +127,8 @@ qdx_pair_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_consta
       uint32_t it = 0;
       bool ok = true;
       for (int tile = pair; ok && tile < total_tiles; tile += n_pairs) {
-        const int tt0 = (tile / p.j_tiles) * 512;
-        const int blocks = tt0 + 256 < p.T ? 2 : 1;
+        int j_tile, tt0, blocks;
+        pair_item(p.items, tile, p.T, j_tile, tt0, blocks);
         const int t0 = tt0 + (int)rank * 128;
         for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
           const int s = it % XSTAGES;
@@ -147,7 +148,9 @@ qdx_pair_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_consta
       uint32_t it = 0;
       bool ok = true;
       for (int tile = pair; ok && tile < total_tiles; tile += n_pairs) {
-        const int w0 = (tile % p.j_tiles) * 256 + (int)rank * 128;   // first column of this CTA
+        int j_tile, tt0, blocks;
+        pair_item(p.items, tile, p.T, j_tile, tt0, blocks);
+        const int w0 = j_tile * 256 + (int)rank * 128;   // first column of this CTA
         for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
           const int q = it % XQ_SLOTS;
           const uint32_t ph = (it / XQ_SLOTS) & 1u;
@@ -166,7 +169,8 @@ qdx_pair_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_consta
       int local = 0;
       bool ok = true;
       for (int tile = pair; ok && tile < total_tiles; tile += n_pairs, ++local) {
-        const int blocks = (tile / p.j_tiles) * 512 + 256 < p.T ? 2 : 1;
+        int j_tile, tt0, blocks;
+        pair_item(p.items, tile, p.T, j_tile, tt0, blocks);
         if (!mbar_wait_cluster(smem_u32(&bars->acc_empty), (uint32_t)(local & 1) ^ 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
         for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
@@ -198,9 +202,9 @@ qdx_pair_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_consta
     int local = 0;
     bool ok = true;
     for (int tile = pair; ok && tile < total_tiles; tile += n_pairs, ++local) {
-      const int j0 = (tile % p.j_tiles) * 256;
-      const int tt0 = (tile / p.j_tiles) * 512;
-      const int blocks = tt0 + 256 < p.T ? 2 : 1;
+      int j_tile, tt0, blocks;
+      pair_item(p.items, tile, p.T, j_tile, tt0, blocks);
+      const int j0 = j_tile * 256;
       const int t = tt0 + m * 256 + (int)rank * 128 + quarter * 32 + lane;
       if (!mbar_wait_cluster(smem_u32(&bars->acc_full), (uint32_t)(local & 1), abort_flag)) { ok = false; break; }
       tc_fence_after();
@@ -246,7 +250,12 @@ qdx_pair_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_consta
     const uint32_t total_it = (uint32_t)my_tiles * (uint32_t)p.k_blocks;
     int pf_tile = pair, pf_kb = grp;
     while (pf_kb >= p.k_blocks) { pf_kb -= p.k_blocks; pf_tile += n_pairs; }
-    int pf_col = (pf_tile % p.j_tiles) * 256 + (int)rank * 128 + 32 * u4;
+    auto item_col = [&](int item) {
+      int j_tile, tt0, blocks;
+      pair_item(p.items, item, p.T, j_tile, tt0, blocks);
+      return j_tile * 256 + (int)rank * 128 + 32 * u4;
+    };
+    int pf_col = item_col(pf_tile);
     // cz: the constant term -delta * s of a real-valued zero-point (ZF), else unused
     auto load_zs = [&](uint32_t (&z)[2], float (&sc)[2], float (&cz)[2]) {
 #pragma unroll
@@ -271,7 +280,7 @@ qdx_pair_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_consta
       while (pf_kb >= p.k_blocks) {
         pf_kb -= p.k_blocks;
         pf_tile += n_pairs;
-        pf_col = (pf_tile % p.j_tiles) * 256 + (int)rank * 128 + 32 * u4;
+        pf_col = item_col(pf_tile);
       }
     };
     uint32_t z[2], zn[2];
@@ -422,6 +431,7 @@ int launch_dx_pair(const peqa_qweight_t* w, const float* zeros_f, int g, const v
   const int tiles = p.j_tiles * p.t_tiles;
   const int max_pairs = sms / 2;
   const int pairs = tiles < max_pairs ? tiles : max_pairs;
+  p.items = make_pair_items(p.j_tiles, p.t_tiles, T, pairs);
   if (zeros_f)
     return w->bits == 4 ? launch_dx_pair_t<4, true>(ta, tq, p, pairs, st)
                         : launch_dx_pair_t<3, true>(ta, tq, p, pairs, st);

@@ -69,6 +69,7 @@ struct PairParams {
   __nv_bfloat16* out;   // Y [T, N]
   int N, K, G, g, g_shift, T;
   int n_tiles, t_tiles, k_blocks;   // 256-channel tiles, 512-token tiles, 64-deep stages
+  PairItems items;
   int* status;
 };
 
@@ -118,7 +119,7 @@ qfwd_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
   cluster_sync_all();
   tc_fence_after();
   const uint32_t tmem_base = bars->tmem_base;
-  const int total_tiles = p.n_tiles * p.t_tiles;
+  const int total_tiles = p.items.total_items;      // work items: whole tiles, then halves
   const int pair = blockIdx.x >> 1;
   const int n_pairs = gridDim.x >> 1;
   const int my_tiles = (total_tiles - pair + n_pairs - 1) / n_pairs;
@@ -132,8 +133,8 @@ qfwd_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
       // that the stage never fills and the bounded waits have to end the kernel
       const uint32_t starve = p.status[5] != 0 ? 1u : 0u;
       for (int tile = pair; ok && tile < total_tiles; tile += n_pairs) {
-        const int tt0 = (tile / p.n_tiles) * 512;
-        const int blocks = tt0 + 256 < p.T ? 2 : 1;
+        int n_tile, tt0, blocks;
+        pair_item(p.items, tile, p.T, n_tile, tt0, blocks);
         const int t0 = tt0 + (int)rank * 128;
         for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
           const int s = it % PSTAGES;
@@ -156,7 +157,9 @@ qfwd_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
       uint32_t it = 0;
       bool ok = true;
       for (int tile = pair; ok && tile < total_tiles; tile += n_pairs) {
-        const int r0 = (tile % p.n_tiles) * 256 + (int)rank * 128;
+        int n_tile, tt0, blocks;
+        pair_item(p.items, tile, p.T, n_tile, tt0, blocks);
+        const int r0 = n_tile * 256 + (int)rank * 128;
         for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
           const int q = it % PQ_SLOTS;
           const uint32_t ph = (it / PQ_SLOTS) & 1u;
@@ -176,7 +179,8 @@ qfwd_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
       int local = 0;
       bool ok = true;
       for (int tile = pair; ok && tile < total_tiles; tile += n_pairs, ++local) {
-        const int blocks = (tile / p.n_tiles) * 512 + 256 < p.T ? 2 : 1;
+        int n_tile, tt0, blocks;
+        pair_item(p.items, tile, p.T, n_tile, tt0, blocks);
         if (!mbar_wait_cluster(smem_u32(&bars->acc_empty), (uint32_t)(local & 1) ^ 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
         for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
@@ -209,9 +213,9 @@ qfwd_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     int local = 0;
     bool ok = true;
     for (int tile = pair; ok && tile < total_tiles; tile += n_pairs, ++local) {
-      const int n0 = (tile % p.n_tiles) * 256;
-      const int tt0 = (tile / p.n_tiles) * 512;
-      const int blocks = tt0 + 256 < p.T ? 2 : 1;
+      int n_tile, tt0, blocks;
+      pair_item(p.items, tile, p.T, n_tile, tt0, blocks);
+      const int n0 = n_tile * 256;
       const int t = tt0 + m * 256 + (int)rank * 128 + quarter * 32 + lane;
       if (!mbar_wait_cluster(smem_u32(&bars->acc_full), (uint32_t)(local & 1), abort_flag)) { ok = false; break; }
       tc_fence_after();
@@ -268,7 +272,12 @@ qfwd_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     // cursor of the stage whose (s, z) is being prefetched, walked without divisions
     int pf_tile = pair, pf_kb = grp;
     while (pf_kb >= p.k_blocks) { pf_kb -= p.k_blocks; pf_tile += n_pairs; }
-    int pf_r = (pf_tile % p.n_tiles) * 256 + (int)rank * 128 + row;
+    auto item_row = [&](int item) {
+      int n_tile, tt0, blocks;
+      pair_item(p.items, item, p.T, n_tile, tt0, blocks);
+      return n_tile * 256 + (int)rank * 128 + row;
+    };
+    int pf_r = item_row(pf_tile);
     // every lane reads another row, so each load of a warp touches 32 sectors: the two
     // units of a stage share one load when they share a group (g >= 64, or one scale per
     // channel), and one 2-byte / 8-byte load when the groups are 32 columns wide
@@ -320,7 +329,7 @@ qfwd_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
       while (pf_kb >= p.k_blocks) {
         pf_kb -= p.k_blocks;
         pf_tile += n_pairs;
-        pf_r = (pf_tile % p.n_tiles) * 256 + (int)rank * 128 + row;
+        pf_r = item_row(pf_tile);
       }
     };
     uint32_t z[2], zn[2];
@@ -477,6 +486,7 @@ int launch_fwd_pair(const peqa_qweight_t* w, const float* zeros_f, int g, const 
   const int tiles = p.n_tiles * p.t_tiles;
   const int max_pairs = sms / 2;
   const int pairs = tiles < max_pairs ? tiles : max_pairs;
+  p.items = make_pair_items(p.n_tiles, p.t_tiles, T, pairs);
   const bool fold = p.G > 1;
   if (zeros_f)   // a real-valued zero-point is folded into the operand whatever the group size
     return w->bits == 4 ? launch_pair_t<4, true, true>(tx, tq, p, pairs, st)

@@ -154,3 +154,12 @@ def test_c2_llama7b_attention_projection_full():
     d = next(synth.generate("c2"))
     res = _run_all(d, 3, 128)
     print("c2 errors (rel-L2, max-abs):", res)
+
+
+@pytest.mark.parametrize("bits,g,N,K", [(3, 128, 2560, 256), (4, 0, 256, 2560)])
+def test_last_round_of_tiles_cut_in_halves(bits, g, N, K):
+    """4096 tokens give 8 token tiles; with 10 tiles along the output (N = 2560 for the forward,
+    K = 2560 for dX) that is 80 tiles for the 74 CTA pairs of a 148-SM part, so the six tiles of
+    the last round run as twelve items of 256 tokens.  Every output element is checked."""
+    d = synth.custom(17 + bits, N, K, 4096, bits, g, outliers=True, sigma_dy=1e-2)
+    _run_all(d, bits, g, check=("Y", "dX"))
