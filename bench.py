@@ -413,6 +413,10 @@ def run_cuda(args):
         "value_frac_of_nominal_2250": value / world / NOMINAL_BF16_TFLOPS,
     }
 
+    # ---- the same fwd + dX + dS/AdamW of the seven linears as ONE library call per step
+    if not args.only_step:
+        out["layer_call"] = bench_layer_call(args, binding, torch, layers, peaks, warmup)
+
     # ---- end to end through the host-buffer entry point (pinned host memory both ways)
     out["e2e"] = None
     if not args.only_step:
@@ -434,6 +438,31 @@ def run_cuda(args):
         print(json.dumps(out), flush=True)
     if dist is not None:
         dist.destroy_process_group()
+
+
+def bench_layer_call(args, binding, torch, layers, peaks, warmup):
+    """peqa_layer_train_step: forward, dX and dS with the AdamW step for all linears of the layer,
+    enqueued by one call (no quantize or decode stage, no events between the kernels)."""
+    dev = layers[0].X.device
+    items = [binding.LayerLinear(w=L.qw, X=L.X, dY=L.dY,
+                                 Y=torch.empty((L.T, L.N), dtype=torch.bfloat16, device=dev),
+                                 dX=torch.empty((L.T, L.K), dtype=torch.bfloat16, device=dev),
+                                 dS=L.dS, m=L.m, v=L.v, workspace=L.ws) for L in layers]
+    for i in range(2):
+        binding.layer_train_step(items, LR, BETA1, BETA2, EPS, WD, step=warmup + 1000 + i)
+    binding.check_status()
+    steps = args.steps
+    with Timed(torch) as tm:
+        for i in range(steps):
+            binding.layer_train_step(items, LR, BETA1, BETA2, EPS, WD, step=warmup + 2000 + i)
+    binding.check_status()
+    ms = tm.ms / steps
+    flop = 3.0 * sum(L.flop for L in layers)
+    tf = flop / (ms * 1e-3) / 1e12
+    peak, which = peak_for_clock(peaks, tm.clocks)
+    return {"what": "peqa_layer_train_step: fwd, dX, dS+AdamW of the seven linears per call", "steps": steps,
+            "ms_per_step": ms, "value": tf, "unit": "TFLOP/s", "clocks": tm.clocks, "peak": peak,
+            "peak_kind": which, "frac_of_peak": tf / peak, "frac_of_nominal_2250": tf / NOMINAL_BF16_TFLOPS}
 
 
 def bench_e2e(args, binding, torch, layers, Y, dX, dist, dev, world, flop_step):
@@ -683,6 +712,12 @@ def render_md(path):
                      f"{p['qlinear_fwd_ms']:.4f} | {p['qlinear_bwd_dx_ms']:.4f} | {p['qlinear_bwd_ds_ms']:.4f} | "
                      f"{p['quantize_rtn_ms']:.4f} | {p['qlinear_decode_ms']:.4f} | {p['fwd_dx_ds_tflops']:.0f} | "
                      f"{p['frac_of_nominal_2250']:.2f} |")
+    if doc.get("layer_call"):
+        lc = doc["layer_call"]
+        o.append("")
+        o.append(f"One call per layer ({lc['what']}): {lc['value']:.0f} TFLOP/s, {lc['ms_per_step']:.3f} ms per step; "
+                 f"clock {lc['clocks']['sm_mhz']} MHz, {lc['frac_of_peak']:.2f} of the measured {lc['peak_kind']} "
+                 f"peak, {lc['frac_of_nominal_2250']:.2f} of nominal.")
     if doc.get("e2e"):
         e = doc["e2e"]
         o.append("")

@@ -168,6 +168,43 @@ int peqa_qlinear_bwd_ds_adamw(const peqa_qweight_t* w, const void* X_bf16, const
                               void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * One training step of several PEQA linears in one call: for each linear, in the
+ * order given, the forward of Eq. 2, then dX and dS by the chain rule on it and,
+ * when apply_adamw is non-zero, App. A's AdamW step on its scales where dS becomes
+ * final (the calls peqa_qlinear_fwd, peqa_qlinear_bwd (dX only) and
+ * peqa_qlinear_bwd_ds_adamw would make, enqueued back to back with every
+ * argument of every linear checked before the first launch).  A transformer
+ * layer's quantized projections -- q, k, v, o, gate, up, down -- are such a list.
+ * Each linear has its own activations X [T, K_i], upstream gradient dY [T, N_i]
+ * and outputs Y [T, N_i], dX [T, K_i], dS [N_i, G_i] (overwritten); composing the
+ * layer (attention, residuals, summing the dX of projections that share an
+ * input) stays with the caller.  With apply_adamw == 0 the scales are left as
+ * they are and m, v may be NULL: a data-parallel caller sums dS over its ranks
+ * first and then calls peqa_scale_adamw.
+ *   workspace: peqa_workspace_bytes(PEQA_OP_BWD, T, &w) bytes per linear, 256-byte
+ *   aligned (may be NULL when that is 0); the linears may share one workspace,
+ *   since their kernels run in stream order.
+ * 1 <= n_linears <= PEQA_LAYER_MAX_LINEARS.  Shape rules and return codes as for
+ * the single calls; nothing is enqueued when a check fails.
+ */
+#define PEQA_LAYER_MAX_LINEARS 16
+typedef struct {
+  peqa_qweight_t w;       /* w.scales must be writable when apply_adamw != 0 */
+  const void* X_bf16;     /* [T, K] */
+  const void* dY_bf16;    /* [T, N] */
+  void* Y_bf16;           /* [T, N] out */
+  void* dX_bf16;          /* [T, K] out */
+  float* dS;              /* [N, G] out */
+  float* m;               /* [N, G] in/out, AdamW first moment */
+  float* v;               /* [N, G] in/out, AdamW second moment */
+  void* workspace;
+  size_t workspace_bytes;
+} peqa_layer_linear_t;
+int peqa_layer_train_step(const peqa_layer_linear_t* linears, int n_linears, int T, int apply_adamw,
+                          float lr, float beta1, float beta2, float eps, float weight_decay,
+                          int64_t step, void* stream);
+
+/*
  * Scale gradient and zero-point gradient together (App. K trains z as well as
  * s).  By the chain rule on Eq. 2, with dW = dY^T X never leaving the chip,
  *   dS[i,gi] = sum_{j in group gi} (Q[i,j] - z[i,gi]) * dW[i,j]     (as peqa_qlinear_bwd)

@@ -42,6 +42,12 @@ class _QWeight(ctypes.Structure):
                 ("scales", ctypes.c_void_p)]
 
 
+class _LayerLinear(ctypes.Structure):
+    _fields_ = [("w", _QWeight), ("X", ctypes.c_void_p), ("dY", ctypes.c_void_p), ("Y", ctypes.c_void_p),
+                ("dX", ctypes.c_void_p), ("dS", ctypes.c_void_p), ("m", ctypes.c_void_p),
+                ("v", ctypes.c_void_p), ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t)]
+
+
 def lib() -> ctypes.CDLL:
     """Load the shared library (built by paper_2305_14152_b200.build); never falls back."""
     global _lib
@@ -96,6 +102,9 @@ def lib() -> ctypes.CDLL:
         L.peqa_zero_adamw.restype = ctypes.c_int
         L.peqa_selftest_configure.argtypes = [i32, i32]
         L.peqa_selftest_configure.restype = ctypes.c_int
+        L.peqa_layer_train_step.argtypes = [ctypes.POINTER(_LayerLinear), i32, i32, i32, f32, f32, f32, f32, f32,
+                                            i64, vp]
+        L.peqa_layer_train_step.restype = ctypes.c_int
         L.peqa_probe_read.argtypes = [vp, sz, vp, sz, vp]
         L.peqa_probe_read.restype = ctypes.c_int
         for name in ("peqa_quantize_rtn", "peqa_pack", "peqa_unpack", "peqa_qlinear_fwd",
@@ -315,6 +324,45 @@ def qlinear_bwd_ds_adamw(w: QWeight, X: torch.Tensor, dY: torch.Tensor, m: torch
                                            beta2, eps, weight_decay, step, wp, wb, _stream()),
            "peqa_qlinear_bwd_ds_adamw")
     return dS
+
+
+@dataclass
+class LayerLinear:
+    """Buffers of one linear of a layer step (all device tensors; m, v may be None when the
+    optimizer step is not applied; workspace may be None when the layer needs none)."""
+    w: QWeight
+    X: torch.Tensor          # bf16 [T, K]
+    dY: torch.Tensor         # bf16 [T, N]
+    Y: torch.Tensor          # bf16 [T, N] out
+    dX: torch.Tensor         # bf16 [T, K] out
+    dS: torch.Tensor         # fp32 [N, G] out
+    m: torch.Tensor | None = None
+    v: torch.Tensor | None = None
+    workspace: torch.Tensor | None = None
+
+
+def layer_train_step(linears, lr: float = 0.0, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.0, step=1,
+                     apply_adamw=True) -> None:
+    """Forward, dX and dS (and, with apply_adamw, the AdamW step on the scales) of every linear of
+    `linears` in one library call."""
+    arr = (_LayerLinear * len(linears))()
+    T = linears[0].dY.shape[0]
+    for a, L in zip(arr, linears):
+        _dev(L.X, torch.bfloat16, "X")
+        _dev(L.dY, torch.bfloat16, "dY")
+        _dev(L.Y, torch.bfloat16, "Y")
+        _dev(L.dX, torch.bfloat16, "dX")
+        _dev(L.dS, torch.float32, "dS")
+        if L.dY.shape[0] != T or L.X.shape[0] != T:
+            raise ValueError("all linears of a layer step take the same number of tokens")
+        wp, wb = _ws(L.workspace)
+        a.w = L.w.c_struct()
+        a.X, a.dY, a.Y, a.dX, a.dS = (L.X.data_ptr(), L.dY.data_ptr(), L.Y.data_ptr(), L.dX.data_ptr(),
+                                      L.dS.data_ptr())
+        a.m, a.v = _ptr(L.m), _ptr(L.v)
+        a.workspace, a.workspace_bytes = wp, wb
+    _check(lib().peqa_layer_train_step(arr, len(linears), T, 1 if apply_adamw else 0, lr, beta1, beta2, eps,
+                                       weight_decay, step, _stream()), "peqa_layer_train_step")
 
 
 def qlinear_bwd_dsdz(w: QWeight, X: torch.Tensor, dY: torch.Tensor, dS=None, dZ=None, workspace=None):

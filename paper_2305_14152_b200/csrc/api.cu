@@ -219,6 +219,49 @@ extern "C" int peqa_qlinear_bwd_ds_adamw(const peqa_qweight_t* w, const void* X,
   return launch_ds(w, nullptr, g, X, dY, T, dS, nullptr, &adam, workspace, workspace_bytes, as_stream(stream));
 }
 
+// Checks of one linear of a layer step; fills the workspace need of its dS pass.
+static int check_layer_linear(const peqa_layer_linear_t* L, int T, int apply_adamw, int* g_out) {
+  int g = 0, G = 0;
+  PEQA_TRY(check_qweight(&L->w, &g, &G));
+  if (!L->X_bf16 || !L->dY_bf16 || !L->Y_bf16 || !L->dX_bf16 || !L->dS) return PEQA_ERR_NULL;
+  if (apply_adamw && (!L->m || !L->v)) return PEQA_ERR_NULL;
+  PEQA_TRY(check_gemm_shape(&L->w, T));
+  if (!aligned16(L->X_bf16) || !aligned16(L->dY_bf16) || !aligned16(L->Y_bf16) || !aligned16(L->dX_bf16) || !aligned16(L->dS))
+    return PEQA_ERR_ALIGNMENT;
+  const size_t need = ds_workspace_bytes(&L->w, g, T);
+  if (need > 0) {
+    if (!L->workspace || L->workspace_bytes < need) return PEQA_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(L->workspace) & 255u) return PEQA_ERR_ALIGNMENT;
+  }
+  *g_out = g;
+  return PEQA_OK;
+}
+
+extern "C" int peqa_layer_train_step(const peqa_layer_linear_t* linears, int n_linears, int T,
+                                     int apply_adamw, float lr, float beta1, float beta2, float eps,
+                                     float weight_decay, int64_t step, void* stream) {
+  if (!linears) return PEQA_ERR_NULL;
+  if (n_linears < 1 || n_linears > PEQA_LAYER_MAX_LINEARS) return PEQA_ERR_BAD_SHAPE;
+  if (apply_adamw && step < 1) return PEQA_ERR_BAD_SHAPE;
+  int g[PEQA_LAYER_MAX_LINEARS];
+  for (int i = 0; i < n_linears; ++i) PEQA_TRY(check_layer_linear(&linears[i], T, apply_adamw, &g[i]));
+  PEQA_TRY(check_arch());
+  cudaStream_t st = as_stream(stream);
+  DsAdam adam;
+  adam.c = adamw_consts(lr, beta1, beta2, eps, weight_decay, (long long)(apply_adamw ? step : 1));
+  for (int i = 0; i < n_linears; ++i) {
+    const peqa_layer_linear_t* L = &linears[i];
+    PEQA_TRY(launch_fwd(&L->w, nullptr, g[i], L->X_bf16, T, L->Y_bf16, st));
+    PEQA_TRY(launch_dx(&L->w, nullptr, g[i], L->dY_bf16, T, L->dX_bf16, st));
+    adam.scales = const_cast<float*>(L->w.scales);
+    adam.m = L->m;
+    adam.v = L->v;
+    PEQA_TRY(launch_ds(&L->w, nullptr, g[i], L->X_bf16, L->dY_bf16, T, L->dS, nullptr, apply_adamw ? &adam : nullptr,
+                       L->workspace, L->workspace_bytes, st));
+  }
+  return PEQA_OK;
+}
+
 extern "C" int peqa_qlinear_bwd_dsdz(const peqa_qweight_t* w, const void* X, const void* dY, int T,
                                      float* dS, float* dZ, void* workspace,
                                      size_t workspace_bytes, void* stream) {
