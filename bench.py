@@ -57,28 +57,31 @@ def load_peaks():
         return dict(FALLBACK_PEAKS), "fallback"
 
 
-def device_sources_sha256():
+SHARED_DEVICE_HEADERS = ("common.cuh", "dequant.cuh", "sm100_ptx.cuh", "tensor_map.cuh")
+
+
+def device_sources_sha256(files):
+    """Hash of the kernel sources a stage's counters depend on (its .cu file and the shared headers)."""
     import hashlib
     h = hashlib.sha256()
     csrc = os.path.join(ROOT, "paper_2305_14152_b200", "csrc")
-    for name in sorted(os.listdir(csrc)):
+    for name in sorted(set(files) | set(SHARED_DEVICE_HEADERS)):
         with open(os.path.join(csrc, name), "rb") as f:
-            text = f.read()
-        if name.endswith(".cuh") or b"__global__" in text:      # device code only
-            h.update(text)
+            h.update(f.read())
     return h.hexdigest()
 
 
 def measured_traffic(stage_name):
     """DRAM bytes per launch of the dominant kernel from the committed ncu capture (scaled to the
-    mean launch of the headline step as that file states), or None when the kernel sources have
+    mean launch of the headline step as that file states), or None when the kernel's sources have
     changed since the counters were taken."""
     try:
         with open(os.path.join(ROOT, "profiles", "dram_traffic_c5.json")) as f:
             doc = json.load(f)
-        if device_sources_sha256() != doc["kernel_sources_sha256"] or doc.get("workload") != WORKLOAD:
+        k = doc["kernels"][stage_name]
+        if doc.get("workload") != WORKLOAD or device_sources_sha256(k["sources"]) != k["sources_sha256"]:
             return None
-        return doc["kernels"][stage_name]["traffic_bytes_mean_launch"]
+        return k["traffic_bytes_mean_launch"]
     except Exception:
         return None
 

@@ -473,8 +473,28 @@ struct DsParams {
   int wpr;
   int piece;         // columns per output piece: 32, 64 or 128; divides g
   int i_tiles, j_tiles, k_blocks;
+  int band, band_rows;   // tile order: tiles per band and which dimension is banded (see ds_tile)
   int* status;
 };
+
+// Tile order of the dS kernel.  One of the two tile dimensions is taken in bands of `band`
+// tiles (row tiles of dY^T when band_rows, else column tiles of X); within a band the other
+// dimension moves slowest.  The pairs that run at the same time then share a band of operand
+// rows (band x 2 MiB at T = 4096) that stays in L2 while the other operand is swept once per
+// band; with the plain order (all row tiles for one column tile) dY was re-read from HBM for
+// every few column tiles: 4x the algorithmic bytes on the 8192 x 8192 layer.
+__device__ __forceinline__ void ds_tile(const DsParams& p, int tile, int& it, int& jt) {
+  const int banded = p.band_rows ? p.i_tiles : p.j_tiles;   // tiles along the banded dimension
+  const int other = p.band_rows ? p.j_tiles : p.i_tiles;
+  const int per_band = p.band * other;
+  const int b = tile / per_band;
+  const int r = tile - b * per_band;
+  const int width = min(p.band, banded - b * p.band);
+  const int o = r / width;
+  const int w = b * p.band + (r - o * width);
+  it = p.band_rows ? w : o;
+  jt = p.band_rows ? o : w;
+}
 
 // A CTA pair (cta_group::2) owns a 256 x 256 tile of dW: CTA `rank` holds rows
 // [i0 + 128*rank, +128) of dY^T as its A operand and accumulator, and loads the
@@ -541,8 +561,10 @@ ds_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_constant__ C
       uint32_t it = 0;
       bool ok = true;
       for (int tile = pair; ok && tile < total_tiles; tile += n_pairs) {
-        const int i0 = (tile % p.i_tiles) * (2 * BM) + (int)rank * BM;
-        const int j0 = (tile / p.i_tiles) * BN + (int)rank * (BN / 2);
+        int ti, tj;
+        ds_tile(p, tile, ti, tj);
+        const int i0 = ti * (2 * BM) + (int)rank * BM;
+        const int j0 = tj * BN + (int)rank * (BN / 2);
         for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
           const int s = it % DS_STAGES;
           const uint32_t ph = (it / DS_STAGES) & 1u;
@@ -601,8 +623,10 @@ ds_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_constant__ C
     int local = 0;
     bool ok = true;
     for (int tile = pair; ok && tile < total_tiles; tile += n_pairs, ++local) {
-      const int i0 = (tile % p.i_tiles) * (2 * BM) + (int)rank * BM;
-      const int j0 = (tile / p.i_tiles) * BN;
+      int ti, tj;
+      ds_tile(p, tile, ti, tj);
+      const int i0 = ti * (2 * BM) + (int)rank * BM;
+      const int j0 = tj * BN;
       const int buf = local & 1;
       const uint32_t acc_ph = (local >> 1) & 1u;
       if (!mbar_wait_cluster(smem_u32(&bars->acc_full[buf]), acc_ph, abort_flag)) { ok = false; break; }
@@ -903,6 +927,17 @@ int launch_ds(const peqa_qweight_t* w, const float* zeros_f, int g, const void* 
   p.i_tiles = (p.N + 2 * BM - 1) / (2 * BM);   // 256-row pair tiles
   p.j_tiles = (p.K + BN - 1) / BN;
   p.k_blocks = (T + BK - 1) / BK;
+  {
+    // a band of about 32 MiB of one operand; band the dimension that gives less HBM traffic:
+    // rows: dY once + X once per band of rows; columns: X once + dY once per band of columns
+    int band = (int)((32u << 20) / ((size_t)512 * (size_t)T));
+    band = band < 1 ? 1 : band;
+    const double by_rows = (double)p.N + (double)p.K * ((p.i_tiles + band - 1) / band);
+    const double by_cols = (double)p.K + (double)p.N * ((p.j_tiles + band - 1) / band);
+    p.band_rows = by_rows <= by_cols ? 1 : 0;
+    const int dim = p.band_rows ? p.i_tiles : p.j_tiles;
+    p.band = band < dim ? band : dim;
+  }
   PEQA_TRY(status_word(st, &p.status));
   CUtensorMap tmap_dy, tmap_x;
   PEQA_TRY(make_tmap_bf16(&tmap_dy, dY, (uint64_t)p.N, (uint64_t)T, BK));
