@@ -39,10 +39,11 @@ constexpr int XBLK_BYTES = 128 * XK * 2;     // one block of 128 tokens of dY: 1
 constexpr int XA_BYTES = 2 * XBLK_BYTES;     // this CTA's two token blocks
 constexpr int XB_BYTES = XK * 128 * 2;       // this CTA's 128 weight columns: 16 KiB
 constexpr int XSTAGE_BYTES = XA_BYTES + XB_BYTES;
-constexpr int XQ_SLOTS = 8;
+constexpr int XQ_SLOTS = 4;
+constexpr int XE_BYTES = 32 * 64;            // one epilogue warp's staging tile: 32 tokens x 32 columns
 constexpr int XQ_BYTES = 4096;               // 64 rows x up to 64 B of codes
 constexpr int X_TMEM_COLS = 512;
-constexpr int X_SMEM_BYTES = XSTAGES * XSTAGE_BYTES + XQ_SLOTS * XQ_BYTES + 1024 + 512;
+constexpr int X_SMEM_BYTES = XSTAGES * XSTAGE_BYTES + XQ_SLOTS * XQ_BYTES + 8 * XE_BYTES + 1024 + 512;
 constexpr int X_GROUPS = 4;
 constexpr int kDxThreads = 896;  // warps: 0 act TMA, 1 MMA, 2 TMEM alloc, 3 code TMA, 4-11 epilogue, 12-27 dequant
 
@@ -78,12 +79,14 @@ __device__ __forceinline__ int dx_group_of(const DxParams& p, int col) {
 template <int BITS, bool ZF>
 __global__ void __launch_bounds__(kDxThreads, 1)
 qdx_pair_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_constant__ CUtensorMap tmap_q,
+                const __grid_constant__ CUtensorMap tmap_out,
                 const DxParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                              ~static_cast<uintptr_t>(1023));
   uint8_t* sm_q = base + XSTAGES * XSTAGE_BYTES;
-  DxBarriers* bars = reinterpret_cast<DxBarriers*>(sm_q + XQ_SLOTS * XQ_BYTES);
+  uint8_t* sm_e = sm_q + XQ_SLOTS * XQ_BYTES;             // 8 epilogue warps x 2 KiB, 64-byte swizzle
+  DxBarriers* bars = reinterpret_cast<DxBarriers*>(sm_e + 8 * XE_BYTES);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();
   const bool leader = rank == 0;
@@ -106,6 +109,7 @@ qdx_pair_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_consta
     fence_mbar_init();
     prefetch_tmap(&tmap_dy);
     prefetch_tmap(&tmap_q);
+    prefetch_tmap(&tmap_out);
   }
   if (warp == 2) {
     tmem_alloc_pair(smem_u32(&bars->tmem_base), X_TMEM_COLS);
@@ -196,43 +200,66 @@ qdx_pair_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_consta
     }
   } else if (warp >= 4 && warp < 12) {
     // ------------------------------------------ epilogue: thread = token, 256 columns
+    // A warp drains 32 tokens x 32 columns at a time through its 2 KiB staging tile (64-byte
+    // swizzle of the output tensor map: 16-byte chunk c of row r at c ^ ((r >> 1) & 3)) and one
+    // tiled bulk store, so the copy engine writes whole sectors of dX; the accumulators are
+    // released as soon as the last chunk has left tensor memory.
     const int quarter = warp & 3;
     const int m = (warp - 4) >> 2;                 // token block = accumulator
     const uint32_t acc_empty_leader = mapa_shared(smem_u32(&bars->acc_empty), 0);
+    uint8_t* stage = sm_e + (warp - 4) * XE_BYTES;
+    uint8_t* srow = stage + lane * 64;
+    const int sw = (lane >> 1) & 3;
     int local = 0;
     bool ok = true;
     for (int tile = pair; ok && tile < total_tiles; tile += n_pairs, ++local) {
       int j_tile, tt0, blocks;
       pair_item(p.items, tile, p.T, j_tile, tt0, blocks);
       const int j0 = j_tile * 256;
-      const int t = tt0 + m * 256 + (int)rank * 128 + quarter * 32 + lane;
+      const int row0 = tt0 + m * 256 + (int)rank * 128 + quarter * 32;   // first token of this warp
       if (!mbar_wait_cluster(smem_u32(&bars->acc_full), (uint32_t)(local & 1), abort_flag)) { ok = false; break; }
       tc_fence_after();
+      int chunks = m < blocks ? (p.K - j0 + 31) / 32 : 0;                // K is a multiple of 32
+      chunks = chunks > 8 ? 8 : chunks;
 #pragma unroll 1
-      for (int cc = 0; cc < 8; ++cc) {
+      for (int cc = 0; cc < chunks; ++cc) {
         const int c0 = j0 + cc * 32;
-        if (c0 >= p.K || m >= blocks) break;
         uint32_t v[32];
         tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + m * 256 + cc * 32, v);
         tmem_ld_wait();
-        if (t < p.T) {
-          __nv_bfloat16* dst = p.out + (size_t)t * p.K + c0;
+        if (cc + 1 == chunks) {
+          // nothing of this tile is left in tensor memory for this warp
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive_cluster(acc_empty_leader);
+        }
+        // the previous store must have finished reading the staging tile
+        if (lane == 0) bulk_wait_group_read0();
+        __syncwarp();
 #pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            uint4 o;
-            __nv_bfloat162 h;
-            h = __floats2bfloat162_rn(__uint_as_float(v[8 * q + 0]), __uint_as_float(v[8 * q + 1])); o.x = *reinterpret_cast<uint32_t*>(&h);
-            h = __floats2bfloat162_rn(__uint_as_float(v[8 * q + 2]), __uint_as_float(v[8 * q + 3])); o.y = *reinterpret_cast<uint32_t*>(&h);
-            h = __floats2bfloat162_rn(__uint_as_float(v[8 * q + 4]), __uint_as_float(v[8 * q + 5])); o.z = *reinterpret_cast<uint32_t*>(&h);
-            h = __floats2bfloat162_rn(__uint_as_float(v[8 * q + 6]), __uint_as_float(v[8 * q + 7])); o.w = *reinterpret_cast<uint32_t*>(&h);
-            *reinterpret_cast<uint4*>(dst + 8 * q) = o;   // K is a multiple of 32: the 32 columns are all valid
-          }
+        for (int q = 0; q < 4; ++q) {
+          uint4 o;
+          __nv_bfloat162 h;
+          h = __floats2bfloat162_rn(__uint_as_float(v[8 * q + 0]), __uint_as_float(v[8 * q + 1])); o.x = *reinterpret_cast<uint32_t*>(&h);
+          h = __floats2bfloat162_rn(__uint_as_float(v[8 * q + 2]), __uint_as_float(v[8 * q + 3])); o.y = *reinterpret_cast<uint32_t*>(&h);
+          h = __floats2bfloat162_rn(__uint_as_float(v[8 * q + 4]), __uint_as_float(v[8 * q + 5])); o.z = *reinterpret_cast<uint32_t*>(&h);
+          h = __floats2bfloat162_rn(__uint_as_float(v[8 * q + 6]), __uint_as_float(v[8 * q + 7])); o.w = *reinterpret_cast<uint32_t*>(&h);
+          *reinterpret_cast<uint4*>(srow + ((q ^ sw) << 4)) = o;
+        }
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0 && row0 < p.T) {
+          tma_store_2d(&tmap_out, smem_u32(stage), c0, row0);
+          bulk_commit_group();
         }
       }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive_cluster(acc_empty_leader);
+      if (chunks == 0) {
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(acc_empty_leader);
+      }
     }
+    if (lane == 0) bulk_wait_group0();             // every store has left shared memory and landed
   } else if (warp >= 12) {
     // ------------------------------------------ weight dequant (this CTA's 128 columns)
     // Group g (four warps) serves the stages with it % 4 == g.  A stage is 64 weight rows x
@@ -355,7 +382,7 @@ qdx_pair_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_consta
 }
 
 template <int BITS, bool ZF>
-int launch_dx_pair_t(const CUtensorMap& ta, const CUtensorMap& tq, const DxParams& p, int pairs,
+int launch_dx_pair_t(const CUtensorMap& ta, const CUtensorMap& tq, const CUtensorMap& to, const DxParams& p, int pairs,
                      cudaStream_t st) {
   auto kern = qdx_pair_kernel<BITS, ZF>;
   PEQA_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, X_SMEM_BYTES));
@@ -371,7 +398,7 @@ int launch_dx_pair_t(const CUtensorMap& ta, const CUtensorMap& tq, const DxParam
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  PEQA_CUDA(cudaLaunchKernelEx(&cfg, kern, ta, tq, p));
+  PEQA_CUDA(cudaLaunchKernelEx(&cfg, kern, ta, tq, to, p));
   return PEQA_OK;
 }
 
@@ -403,7 +430,18 @@ int launch_dx_pair(const peqa_qweight_t* w, const float* zeros_f, int g, const v
   PEQA_TRY(status_word(st, &p.status));
   EncodeTiledFn enc = nullptr;
   PEQA_TRY(tensor_map_encoder(&enc));
-  CUtensorMap ta, tq;
+  CUtensorMap ta, tq, to;
+  {
+    // output dX [T, K]: boxes of 32 columns x 32 tokens, 64-byte swizzle (the epilogue's staging tile)
+    cuuint64_t dims[2] = {(cuuint64_t)p.K, (cuuint64_t)T};
+    cuuint64_t strides[1] = {(cuuint64_t)p.K * 2};
+    cuuint32_t box[2] = {32, 32};
+    cuuint32_t estr[2] = {1, 1};
+    if (enc(&to, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, dX, dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B,
+            CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return cuda_fail(cudaErrorInvalidValue);
+  }
   {
     cuuint64_t dims[2] = {(cuuint64_t)p.N, (cuuint64_t)T};
     cuuint64_t strides[1] = {(cuuint64_t)p.N * 2};
@@ -433,10 +471,10 @@ int launch_dx_pair(const peqa_qweight_t* w, const float* zeros_f, int g, const v
   const int pairs = tiles < max_pairs ? tiles : max_pairs;
   p.items = make_pair_items(p.j_tiles, p.t_tiles, T, pairs);
   if (zeros_f)
-    return w->bits == 4 ? launch_dx_pair_t<4, true>(ta, tq, p, pairs, st)
-                        : launch_dx_pair_t<3, true>(ta, tq, p, pairs, st);
-  return w->bits == 4 ? launch_dx_pair_t<4, false>(ta, tq, p, pairs, st)
-                      : launch_dx_pair_t<3, false>(ta, tq, p, pairs, st);
+    return w->bits == 4 ? launch_dx_pair_t<4, true>(ta, tq, to, p, pairs, st)
+                        : launch_dx_pair_t<3, true>(ta, tq, to, p, pairs, st);
+  return w->bits == 4 ? launch_dx_pair_t<4, false>(ta, tq, to, p, pairs, st)
+                      : launch_dx_pair_t<3, false>(ta, tq, to, p, pairs, st);
 }
 
 }  // namespace peqa

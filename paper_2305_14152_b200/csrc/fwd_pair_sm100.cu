@@ -42,10 +42,11 @@ constexpr int PBLK_BYTES = 128 * PK * 2;     // one block of 128 tokens of X: 16
 constexpr int PA_BYTES = 2 * PBLK_BYTES;     // this CTA's two token blocks
 constexpr int PB_BYTES = 128 * PK * 2;       // this CTA's 128 channels: 16 KiB
 constexpr int PSTAGE_BYTES = PA_BYTES + PB_BYTES;
-constexpr int PQ_SLOTS = 8;
+constexpr int PQ_SLOTS = 4;
+constexpr int PE_BYTES = 32 * 64;            // one epilogue warp's staging tile: 32 tokens x 32 channels
 constexpr int PQ_BYTES = 128 * 32;           // packed codes of one stage: 128 rows x 8 words
 constexpr int P_TMEM_COLS = 512;
-constexpr int P_SMEM_BYTES = PSTAGES * PSTAGE_BYTES + PQ_SLOTS * PQ_BYTES + 1024 + 512;
+constexpr int P_SMEM_BYTES = PSTAGES * PSTAGE_BYTES + PQ_SLOTS * PQ_BYTES + 8 * PE_BYTES + 1024 + 512;
 constexpr int P_GROUPS = 4;        // dequant groups (four warps each)
 constexpr int kPairThreads = 896;  // warps: 0 act TMA, 1 MMA, 2 TMEM alloc, 3 code TMA, 4-11 epilogue, 12-27 dequant
 
@@ -81,12 +82,13 @@ __device__ __forceinline__ int pair_group_of(const PairParams& p, int col) {
 template <int BITS, bool FOLD, bool ZF>
 __global__ void __launch_bounds__(kPairThreads, 1)
 qfwd_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_q,
-                 const PairParams p) {
+                 const __grid_constant__ CUtensorMap tmap_y, const PairParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                              ~static_cast<uintptr_t>(1023));
   uint8_t* sm_q = base + PSTAGES * PSTAGE_BYTES;          // PQ_SLOTS x 4 KiB, plain 32-byte rows
-  PairBarriers* bars = reinterpret_cast<PairBarriers*>(sm_q + PQ_SLOTS * PQ_BYTES);
+  uint8_t* sm_e = sm_q + PQ_SLOTS * PQ_BYTES;             // 8 epilogue warps x 2 KiB, 64-byte swizzle
+  PairBarriers* bars = reinterpret_cast<PairBarriers*>(sm_e + 8 * PE_BYTES);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();
   const bool leader = rank == 0;
@@ -109,6 +111,7 @@ qfwd_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     fence_mbar_init();
     prefetch_tmap(&tmap_x);
     prefetch_tmap(&tmap_q);
+    prefetch_tmap(&tmap_y);
   }
   if (warp == 2) {
     tmem_alloc_pair(smem_u32(&bars->tmem_base), P_TMEM_COLS);
@@ -206,26 +209,42 @@ qfwd_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     }
   } else if (warp >= 4 && warp < 12) {
     // ------------------------------------------ epilogue: thread = token, 256 channels
+    // A warp drains 32 tokens x 32 channels at a time: tensor memory -> registers -> bf16 ->
+    // its 2 KiB staging tile (rows of 64 bytes, 16-byte chunk c of row r at c ^ ((r >> 1) & 3):
+    // the 64-byte swizzle of the output tensor map, which also keeps the stores free of bank
+    // conflicts) -> one tiled bulk store.  The copy engine writes whole sectors of Y; a
+    // thread-per-row store by the warp itself cost 32 half-filled sectors per instruction and
+    // made the drain take ~11,000 cycles a tile.  The accumulators are released as soon as the
+    // last chunk has left tensor memory.
     const int quarter = warp & 3;
     const int m = (warp - 4) >> 2;                 // token block = accumulator
     const uint32_t acc_empty_leader = mapa_shared(smem_u32(&bars->acc_empty), 0);
-    const bool vec_ok = (p.N & 7) == 0;
+    uint8_t* stage = sm_e + (warp - 4) * PE_BYTES;
+    uint8_t* srow = stage + lane * 64;
+    const int sw = (lane >> 1) & 3;
     int local = 0;
     bool ok = true;
     for (int tile = pair; ok && tile < total_tiles; tile += n_pairs, ++local) {
       int n_tile, tt0, blocks;
       pair_item(p.items, tile, p.T, n_tile, tt0, blocks);
       const int n0 = n_tile * 256;
-      const int t = tt0 + m * 256 + (int)rank * 128 + quarter * 32 + lane;
+      const int row0 = tt0 + m * 256 + (int)rank * 128 + quarter * 32;   // first token of this warp
       if (!mbar_wait_cluster(smem_u32(&bars->acc_full), (uint32_t)(local & 1), abort_flag)) { ok = false; break; }
       tc_fence_after();
+      int chunks = m < blocks ? (p.N - n0 + 31) / 32 : 0;
+      chunks = chunks > 8 ? 8 : chunks;
 #pragma unroll 1
-      for (int cc = 0; cc < 8; ++cc) {
+      for (int cc = 0; cc < chunks; ++cc) {
         const int c0 = n0 + cc * 32;
-        if (c0 >= p.N || m >= blocks) break;
         uint32_t v[32];
         tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + m * 256 + cc * 32, v);
         tmem_ld_wait();
+        if (cc + 1 == chunks) {
+          // nothing of this tile is left in tensor memory for this warp
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive_cluster(acc_empty_leader);
+        }
         if (!FOLD) {
           // one scale per channel: every lane reads the same 32 scales (broadcast loads)
 #pragma unroll
@@ -234,30 +253,33 @@ qfwd_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             v[j] = __float_as_uint(__uint_as_float(v[j]) * sc);
           }
         }
-        if (t < p.T) {
-          __nv_bfloat16* dst = p.out + (size_t)t * p.N + c0;
-          if (vec_ok && c0 + 32 <= p.N) {
+        // the previous store must have finished reading the staging tile
+        if (lane == 0) bulk_wait_group_read0();
+        __syncwarp();
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-              uint4 o;
-              __nv_bfloat162 h;
-              h = __floats2bfloat162_rn(__uint_as_float(v[8 * q + 0]), __uint_as_float(v[8 * q + 1])); o.x = *reinterpret_cast<uint32_t*>(&h);
-              h = __floats2bfloat162_rn(__uint_as_float(v[8 * q + 2]), __uint_as_float(v[8 * q + 3])); o.y = *reinterpret_cast<uint32_t*>(&h);
-              h = __floats2bfloat162_rn(__uint_as_float(v[8 * q + 4]), __uint_as_float(v[8 * q + 5])); o.z = *reinterpret_cast<uint32_t*>(&h);
-              h = __floats2bfloat162_rn(__uint_as_float(v[8 * q + 6]), __uint_as_float(v[8 * q + 7])); o.w = *reinterpret_cast<uint32_t*>(&h);
-              *reinterpret_cast<uint4*>(dst + 8 * q) = o;
-            }
-          } else {
-#pragma unroll
-            for (int j = 0; j < 32; ++j)
-              if (c0 + j < p.N) dst[j] = __float2bfloat16_rn(__uint_as_float(v[j]));
-          }
+        for (int q = 0; q < 4; ++q) {
+          uint4 o;
+          __nv_bfloat162 h;
+          h = __floats2bfloat162_rn(__uint_as_float(v[8 * q + 0]), __uint_as_float(v[8 * q + 1])); o.x = *reinterpret_cast<uint32_t*>(&h);
+          h = __floats2bfloat162_rn(__uint_as_float(v[8 * q + 2]), __uint_as_float(v[8 * q + 3])); o.y = *reinterpret_cast<uint32_t*>(&h);
+          h = __floats2bfloat162_rn(__uint_as_float(v[8 * q + 4]), __uint_as_float(v[8 * q + 5])); o.z = *reinterpret_cast<uint32_t*>(&h);
+          h = __floats2bfloat162_rn(__uint_as_float(v[8 * q + 6]), __uint_as_float(v[8 * q + 7])); o.w = *reinterpret_cast<uint32_t*>(&h);
+          *reinterpret_cast<uint4*>(srow + ((q ^ sw) << 4)) = o;
+        }
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0 && row0 < p.T) {
+          tma_store_2d(&tmap_y, smem_u32(stage), c0, row0);
+          bulk_commit_group();
         }
       }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive_cluster(acc_empty_leader);
+      if (chunks == 0) {
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(acc_empty_leader);
+      }
     }
+    if (lane == 0) bulk_wait_group0();             // every store has left shared memory and landed
   } else if (warp >= 12) {
     // ------------------------------------------ weight dequant (this CTA's 128 channels)
     // Group g (four warps) serves the stages with it % 4 == g.  A thread is one channel:
@@ -408,8 +430,8 @@ qfwd_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
 }
 
 template <int BITS, bool FOLD, bool ZF>
-int launch_pair_t(const CUtensorMap& tx, const CUtensorMap& tq, const PairParams& p, int pairs,
-                  cudaStream_t st) {
+int launch_pair_t(const CUtensorMap& tx, const CUtensorMap& tq, const CUtensorMap& ty, const PairParams& p,
+                  int pairs, cudaStream_t st) {
   auto kern = qfwd_pair_kernel<BITS, FOLD, ZF>;
   PEQA_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM_BYTES));
   cudaLaunchConfig_t cfg = {};
@@ -424,7 +446,7 @@ int launch_pair_t(const CUtensorMap& tx, const CUtensorMap& tq, const PairParams
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  PEQA_CUDA(cudaLaunchKernelEx(&cfg, kern, tx, tq, p));
+  PEQA_CUDA(cudaLaunchKernelEx(&cfg, kern, tx, tq, ty, p));
   return PEQA_OK;
 }
 
@@ -458,7 +480,18 @@ int launch_fwd_pair(const peqa_qweight_t* w, const float* zeros_f, int g, const 
   PEQA_TRY(status_word(st, &p.status));
   EncodeTiledFn enc = nullptr;
   PEQA_TRY(tensor_map_encoder(&enc));
-  CUtensorMap tx, tq;
+  CUtensorMap tx, tq, ty;
+  {
+    // output Y [T, N]: boxes of 32 channels x 32 tokens, 64-byte swizzle (the epilogue's staging tile)
+    cuuint64_t dims[2] = {(cuuint64_t)p.N, (cuuint64_t)T};
+    cuuint64_t strides[1] = {(cuuint64_t)p.N * 2};
+    cuuint32_t box[2] = {32, 32};
+    cuuint32_t estr[2] = {1, 1};
+    if (enc(&ty, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Y, dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B,
+            CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return cuda_fail(cudaErrorInvalidValue);
+  }
   {
     cuuint64_t dims[2] = {(cuuint64_t)p.K, (cuuint64_t)T};
     cuuint64_t strides[1] = {(cuuint64_t)p.K * 2};
@@ -489,13 +522,13 @@ int launch_fwd_pair(const peqa_qweight_t* w, const float* zeros_f, int g, const 
   p.items = make_pair_items(p.n_tiles, p.t_tiles, T, pairs);
   const bool fold = p.G > 1;
   if (zeros_f)   // a real-valued zero-point is folded into the operand whatever the group size
-    return w->bits == 4 ? launch_pair_t<4, true, true>(tx, tq, p, pairs, st)
-                        : launch_pair_t<3, true, true>(tx, tq, p, pairs, st);
+    return w->bits == 4 ? launch_pair_t<4, true, true>(tx, tq, ty, p, pairs, st)
+                        : launch_pair_t<3, true, true>(tx, tq, ty, p, pairs, st);
   if (w->bits == 4)
-    return fold ? launch_pair_t<4, true, false>(tx, tq, p, pairs, st)
-                : launch_pair_t<4, false, false>(tx, tq, p, pairs, st);
-  return fold ? launch_pair_t<3, true, false>(tx, tq, p, pairs, st)
-              : launch_pair_t<3, false, false>(tx, tq, p, pairs, st);
+    return fold ? launch_pair_t<4, true, false>(tx, tq, ty, p, pairs, st)
+                : launch_pair_t<4, false, false>(tx, tq, ty, p, pairs, st);
+  return fold ? launch_pair_t<3, true, false>(tx, tq, ty, p, pairs, st)
+              : launch_pair_t<3, false, false>(tx, tq, ty, p, pairs, st);
 }
 
 }  // namespace peqa
