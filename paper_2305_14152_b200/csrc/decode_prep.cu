@@ -227,18 +227,22 @@ decode_prep_kernel(const PrepParams p) {
   __syncwarp();
 
   // ---- this warp's steps of a chunk: [bound(w), bound(w+1)) of the pair-major list, cut so
-  // that the warps' costs are equal (a step of a full pair costs 2, of a half pair 1)
+  // that the warps' costs are equal (a step of a full pair costs 4, of a half pair 3)
   auto spc_of = [&](int ch) { return min(p.spc, p.T - ch * p.spc); };
   auto bound = [&](int w, int spc_c) {
-    const int tot = (lead + 2 * F + trail) * spc_c;
+    // measured: a step of a half pair takes about three quarters of a full pair's step (half
+    // the code extraction, the same MMAs and activation reads)
+    constexpr int CF = 4, CH = 3;
+    const int tot = (CH * (lead + trail) + CF * F) * spc_c;
     int b = (int)(((long long)w * tot) / kPWarps);
     int at = 0;
     if (lead) {
-      if (b <= spc_c) return b;
-      b -= spc_c;
+      if (b <= CH * spc_c) return (b + CH / 2) / CH;
+      b -= CH * spc_c;
       at = spc_c;
     }
-    return b <= 2 * F * spc_c ? at + ((b + 1) >> 1) : at + F * spc_c + (b - 2 * F * spc_c);
+    if (b <= CF * F * spc_c) return at + (b + CF / 2) / CF;
+    return at + F * spc_c + (b - CF * F * spc_c + CH / 2) / CH;
   };
   auto pair_full = [&](int lp) { return lp >= lead && lp < lead + F; };
   // first row group of local pair lp (the only one of a half pair)
@@ -719,10 +723,10 @@ int plan_prep(int N, int K, int M, int bits, int gcols, PrepPlan* plan) {
   const int gps = grouped ? kStepCols / gcols : 0;
   auto need = [&](int spc, int slots, int sps, int* maxseg) -> size_t {
     const int nch = (plan->T + spc - 1) / spc;
-    // a warp's share of a chunk is at most `cost` units (a full pair-step costs 2): it touches
-    // at most ceil(cost / (2 * spc)) + 1 full pairs and the half pairs at the ends
-    const int cost = (2 * plan->pairs * spc + kPWarps - 1) / kPWarps + 1;
-    *maxseg = (cost + 2 * spc - 1) / (2 * spc) + 3;
+    // a warp's share of a chunk is at most pairs*spc*4/16 cost units, i.e. at most that / 3 + 2
+    // steps (all of them half-pair steps at cost 3): the pairs it touches
+    const int steps = plan->pairs * spc / 12 + 2;
+    *maxseg = (steps + spc - 1) / spc + 2;
     if (*maxseg > plan->pairs) *maxseg = plan->pairs;
     size_t b = 128 + kPHeadBytes;
     b += (size_t)kPWarps * (*maxseg) * 16 * toks * 4;
