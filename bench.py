@@ -678,7 +678,7 @@ def bench_ds_from_y(torch, binding, dev, peaks, reps=20):
 
 # --------------------------------------------------------------------------- rendering
 def render_md(path):
-    """Markdown tables of a saved JSON line (the results section of the benchmark spec is made this way)."""
+    """Markdown tables of a saved JSON line (the tables of the results write-up are made this way)."""
     with open(path) as f:
         text = f.read()
     doc = None
