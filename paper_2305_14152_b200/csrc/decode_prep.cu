@@ -141,7 +141,7 @@ struct StepRegs {
 template <int BITS, int NT, bool HAS_B, int MM>
 __device__ __forceinline__ void run_mma2(const uint32_t (&wa)[BITS], const uint32_t (&wb)[BITS],
                                          const uint8_t* x0, const uint8_t* x1,
-                                         float (&acc)[NT][4]) {
+                                         float (&acc)[NT][4], float (&acc2)[NT][4]) {
   const uint4 xa = *reinterpret_cast<const uint4*>(x0 + MM * 64);
   uint4 xb = make_uint4(0u, 0u, 0u, 0u);
   if (NT == 2) xb = *reinterpret_cast<const uint4*>(x1 + MM * 64);
@@ -153,11 +153,14 @@ __device__ __forceinline__ void run_mma2(const uint32_t (&wa)[BITS], const uint3
     dq::mma_pairs_stream<BITS, 2 * MM>(wb, f0[1], f0[3]);
     dq::mma_pairs_stream<BITS, 2 * MM + 1>(wb, f1[1], f1[3]);
   }
+  // the two MMAs of a run go to different accumulators, so that consecutive MMAs of a warp do
+  // not wait for one another (a single chain of 32 dependent MMAs per step cost 5 % of the
+  // kernel); the halves are added when the sums are taken off
   pmma_16816(acc[0], f0, xa.x, xa.y);
-  pmma_16816(acc[0], f1, xa.z, xa.w);
+  pmma_16816(acc2[0], f1, xa.z, xa.w);
   if (NT == 2) {
     pmma_16816(acc[1], f0, xb.x, xb.y);
-    pmma_16816(acc[1], f1, xb.z, xb.w);
+    pmma_16816(acc2[1], f1, xb.z, xb.w);
   }
 }
 
@@ -391,12 +394,22 @@ decode_prep_kernel(const PrepParams p) {
     // ---- this warp's steps of the chunk
     const int lo = wbound[warp], hi = wbound[warp + 1];
     int seg = 0, cur_pair = -1;
-    float acc[NT][4], yv[NT][4];
+    float acc[NT][4], acc2[NT][4], yv[NT][4];
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-      for (int e = 0; e < 4; ++e) acc[nt][e] = yv[nt][e] = 0.0f;
+      for (int e = 0; e < 4; ++e) acc[nt][e] = acc2[nt][e] = yv[nt][e] = 0.0f;
+    auto fold = [&]() {
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          acc[nt][e] += acc2[nt][e];
+          acc2[nt][e] = 0.0f;
+        }
+    };
     auto park = [&]() {
+      fold();
       float* mine = part + ((size_t)(warp * p.maxseg + seg) * 16) * toks;
 #pragma unroll
       for (int nt = 0; nt < NT; ++nt) {
@@ -476,6 +489,7 @@ decode_prep_kernel(const PrepParams p) {
         }
         // group gi of the step is complete: take z * sum x + sum bias * x off and scale
         auto flush = [&](int gi) {
+          fold();
           const int gg = gstep0 + gi;                              // group index in the row
           const float* sm = sums + ((size_t)(tl * GPS + gi) * TOKP) * 2;
           if (!p.task_ids) {
@@ -533,17 +547,17 @@ decode_prep_kernel(const PrepParams p) {
           const uint8_t* xs0 = x0 + s * 256;
           const uint8_t* xs1 = x1 + s * 256;
           if (has_b) {
-            run_mma2<BITS, NT, true, 0>(wa, wb, xs0, xs1, acc);
-            run_mma2<BITS, NT, true, 1>(wa, wb, xs0, xs1, acc);
+            run_mma2<BITS, NT, true, 0>(wa, wb, xs0, xs1, acc, acc2);
+            run_mma2<BITS, NT, true, 1>(wa, wb, xs0, xs1, acc, acc2);
             if (GROUPED && RUNS_PER_GROUP == 2) flush(2 * s);
-            run_mma2<BITS, NT, true, 2>(wa, wb, xs0, xs1, acc);
-            run_mma2<BITS, NT, true, 3>(wa, wb, xs0, xs1, acc);
+            run_mma2<BITS, NT, true, 2>(wa, wb, xs0, xs1, acc, acc2);
+            run_mma2<BITS, NT, true, 3>(wa, wb, xs0, xs1, acc, acc2);
           } else {
-            run_mma2<BITS, NT, false, 0>(wa, wb, xs0, xs1, acc);
-            run_mma2<BITS, NT, false, 1>(wa, wb, xs0, xs1, acc);
+            run_mma2<BITS, NT, false, 0>(wa, wb, xs0, xs1, acc, acc2);
+            run_mma2<BITS, NT, false, 1>(wa, wb, xs0, xs1, acc, acc2);
             if (GROUPED && RUNS_PER_GROUP == 2) flush(2 * s);
-            run_mma2<BITS, NT, false, 2>(wa, wb, xs0, xs1, acc);
-            run_mma2<BITS, NT, false, 3>(wa, wb, xs0, xs1, acc);
+            run_mma2<BITS, NT, false, 2>(wa, wb, xs0, xs1, acc, acc2);
+            run_mma2<BITS, NT, false, 3>(wa, wb, xs0, xs1, acc, acc2);
           }
           if (GROUPED && RUNS_PER_GROUP == 2) flush(2 * s + 1);
           if (GROUPED && RUNS_PER_GROUP == 4) flush(s);
