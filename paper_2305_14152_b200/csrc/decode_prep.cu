@@ -198,8 +198,11 @@ decode_prep_kernel(const PrepParams p) {
   // sums, GROUPED: [groups of the chunk][TOKP][2] = (sum x, sum bias*x) per group and token;
   // else [16 warps][TOKP][2]: every warp's share of the chunk's sums, added in warp order
   const int sum_rows = GROUPED ? p.spc * GPS : kPWarps;
+  // cterm (GROUPED): [pairs][16][toks], the part of every output that does not depend on the weights
+  float* cterm = sums + (size_t)sum_rows * TOKP * 2;
   uint8_t* xs = reinterpret_cast<uint8_t*>(
-      (reinterpret_cast<uintptr_t>(sums + (size_t)sum_rows * TOKP * 2) + 127) & ~static_cast<uintptr_t>(127));
+      (reinterpret_cast<uintptr_t>(cterm + (GROUPED ? (size_t)p.pairs_per_cta * 16 * toks : 0)) + 127) &
+      ~static_cast<uintptr_t>(127));
   uint8_t* ring = xs + (((size_t)p.M * p.x_pitch + 127) & ~static_cast<size_t>(127));
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -462,28 +465,37 @@ decode_prep_kernel(const PrepParams p) {
           if (lane == 0) issue_next();
         }
 
-        // scale and zero-point of this lane's rows for the groups of the step (GROUPED)
+        // scales of this lane's two rows for the groups of the step (GROUPED, one task): the
+        // sum of a group is only scaled here; its zero-point and bias terms, which do not depend
+        // on the weights, come off where the rows are finished
         const int rowa = pair_rg(lp) * 8 + r8, rowb = rowa + 8;
-        float gs_a = 0.0f, gs_b = 0.0f, gz_a = 0.0f, gz_b = 0.0f;
-        float gs2_a = 0.0f, gs2_b = 0.0f, gz2_a = 0.0f, gz2_b = 0.0f;
         const int gstep0 = ((ch * p.spc + tl) * GPS);              // first group of the step
+        float gsa[GPS], gsb[GPS];
         if (GROUPED && !p.task_ids) {
-          // lane c4 fetches group c4 % GPS (and, with eight groups a step, group c4 + 4)
-          const int gl = c4 % GPS;
-          if (gstep0 + gl < p.G) {
-            gs_a = __ldg(p.scales + (size_t)rowa * p.G + gstep0 + gl);
-            gz_a = (float)__ldg(p.zeros + (size_t)rowa * p.G + gstep0 + gl);
-            if (has_b) {
-              gs_b = __ldg(p.scales + (size_t)rowb * p.G + gstep0 + gl);
-              gz_b = (float)__ldg(p.zeros + (size_t)rowb * p.G + gstep0 + gl);
+          const float* pa = p.scales + (size_t)rowa * p.G + gstep0;
+          const float* pb = p.scales + (size_t)rowb * p.G + gstep0;
+          if ((p.G % GPS) == 0 && gstep0 < p.G) {
+            // G is a multiple of the groups per step: whole, aligned vectors
+            if (GPS >= 4) {
+#pragma unroll
+              for (int q = 0; q < GPS / 4; ++q) {
+                const float4 va = __ldg(reinterpret_cast<const float4*>(pa) + q);
+                const float4 vb = has_b ? __ldg(reinterpret_cast<const float4*>(pb) + q) : make_float4(0.f, 0.f, 0.f, 0.f);
+                gsa[4 * q + 0] = va.x; gsa[4 * q + 1] = va.y; gsa[4 * q + 2] = va.z; gsa[4 * q + 3] = va.w;
+                gsb[4 * q + 0] = vb.x; gsb[4 * q + 1] = vb.y; gsb[4 * q + 2] = vb.z; gsb[4 * q + 3] = vb.w;
+              }
+            } else {
+              const float2 va = __ldg(reinterpret_cast<const float2*>(pa));
+              const float2 vb = has_b ? __ldg(reinterpret_cast<const float2*>(pb)) : make_float2(0.f, 0.f);
+              gsa[0] = va.x; gsa[GPS - 1] = va.y;
+              gsb[0] = vb.x; gsb[GPS - 1] = vb.y;
             }
-          }
-          if (GPS == 8 && gstep0 + gl + 4 < p.G) {
-            gs2_a = __ldg(p.scales + (size_t)rowa * p.G + gstep0 + gl + 4);
-            gz2_a = (float)__ldg(p.zeros + (size_t)rowa * p.G + gstep0 + gl + 4);
-            if (has_b) {
-              gs2_b = __ldg(p.scales + (size_t)rowb * p.G + gstep0 + gl + 4);
-              gz2_b = (float)__ldg(p.zeros + (size_t)rowb * p.G + gstep0 + gl + 4);
+          } else {
+#pragma unroll
+            for (int q = 0; q < GPS; ++q) {
+              const bool in = gstep0 + q < p.G;
+              gsa[q] = in ? __ldg(pa + q) : 0.0f;
+              gsb[q] = in && has_b ? __ldg(pb + q) : 0.0f;
             }
           }
         }
@@ -493,18 +505,13 @@ decode_prep_kernel(const PrepParams p) {
           const int gg = gstep0 + gi;                              // group index in the row
           const float* sm = sums + ((size_t)(tl * GPS + gi) * TOKP) * 2;
           if (!p.task_ids) {
-            const int src = (lane & ~3) | (gi & 3 & (GPS - 1));
-            const float sa = __shfl_sync(0xffffffffu, gi >= 4 ? gs2_a : gs_a, src);
-            const float sb = __shfl_sync(0xffffffffu, gi >= 4 ? gs2_b : gs_b, src);
-            const float za = __shfl_sync(0xffffffffu, gi >= 4 ? gz2_a : gz_a, src);
-            const float zb = __shfl_sync(0xffffffffu, gi >= 4 ? gz2_b : gz_b, src);
+            const float sa = gsa[gi], sb = gsb[gi];
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) {
-              const float4 sv = *reinterpret_cast<const float4*>(sm + (nt * 8 + c4 * 2) * 2);
-              yv[nt][0] = fmaf(sa, acc[nt][0] - fmaf(za, sv.x, sv.y), yv[nt][0]);
-              yv[nt][1] = fmaf(sa, acc[nt][1] - fmaf(za, sv.z, sv.w), yv[nt][1]);
-              yv[nt][2] = fmaf(sb, acc[nt][2] - fmaf(zb, sv.x, sv.y), yv[nt][2]);
-              yv[nt][3] = fmaf(sb, acc[nt][3] - fmaf(zb, sv.z, sv.w), yv[nt][3]);
+              yv[nt][0] = fmaf(sa, acc[nt][0], yv[nt][0]);
+              yv[nt][1] = fmaf(sa, acc[nt][1], yv[nt][1]);
+              yv[nt][2] = fmaf(sb, acc[nt][2], yv[nt][2]);
+              yv[nt][3] = fmaf(sb, acc[nt][3], yv[nt][3]);
             }
           } else if (gg < p.G) {
             // every token has the scales of its own task (Sec. 3.3)
@@ -573,20 +580,89 @@ decode_prep_kernel(const PrepParams p) {
     if (cur_pair >= 0) park();
     __syncthreads();
 
-    // ---- add the parked sums of every pair in warp order
+    // ---- grouped scales of one task: the terms of the chunk's groups that do not depend on the
+    // weights, per row and token:  sum_g s[row, g] * (z[row, g] * sum x_g + sum bias * x_g).
+    // A warp takes rows warp, warp + 16, ...; the loads of all its rows are issued before the
+    // first is used (this pass is pure latency otherwise), a lane owns four adjacent groups.
     const bool last = ch + 1 == p.nchunks;
+    const bool group_terms = GROUPED && !p.task_ids;
+    if (group_terms) {
+      constexpr int RB = 8;                                        // rows of a warp in flight
+      const int nrows = npairs * 16;
+      const int g0 = ch * p.spc * GPS;
+      const int ng = min(p.G - g0, spc_c * GPS);
+      const bool vec = ((p.G | g0) & 3) == 0;                      // a lane's four scales are 16-byte aligned
+      for (int rbase = warp; rbase < nrows; rbase += kPWarps * RB) {
+        for (int gb = 0; gb < ng; gb += 128) {
+          const int gl = gb + 4 * lane;                            // this lane's first group of the block
+          float4 sv[RB];
+          uint32_t zv[RB];
+#pragma unroll
+          for (int i = 0; i < RB; ++i) {
+            const int r = rbase + i * kPWarps;
+            const int lp = r >> 4, lr = r & 15;
+            sv[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+            zv[i] = 0u;
+            if (r < nrows && (pair_full(lp) || lr < 8) && gl < ng) {
+              const size_t off = (size_t)(pair_rg(lp) * 8 + lr) * p.G + g0 + gl;
+              if (vec && gl + 4 <= ng) {
+                sv[i] = __ldg(reinterpret_cast<const float4*>(p.scales + off));
+                zv[i] = __ldg(reinterpret_cast<const uint32_t*>(p.zeros + off));
+              } else {
+                float t[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                  if (gl + e < ng) {
+                    t[e] = __ldg(p.scales + off + e);
+                    zv[i] |= (uint32_t)__ldg(p.zeros + off + e) << (8 * e);
+                  }
+                sv[i] = make_float4(t[0], t[1], t[2], t[3]);
+              }
+            }
+          }
+          // groups past the chunk's end carry s = 0; the sums read for them are the last group's
+          for (int m = 0; m < p.M; ++m) {
+            float2 sm[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+              sm[e] = *reinterpret_cast<const float2*>(sums + ((size_t)min(gl + e, ng - 1) * TOKP + m) * 2);
+#pragma unroll
+            for (int i = 0; i < RB; ++i) {
+              const int r = rbase + i * kPWarps;
+              if (r >= nrows) break;                               // warp-uniform
+              const float s4[4] = {sv[i].x, sv[i].y, sv[i].z, sv[i].w};
+              float c = 0.0f;
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const float z = (float)((zv[i] >> (8 * e)) & 0xFFu);
+                c = fmaf(s4[e], fmaf(z, sm[e].x, sm[e].y), c);
+              }
+#pragma unroll
+              for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
+              if (lane == 0) {
+                float* ct = cterm + (size_t)r * toks + m;
+                *ct = gb == 0 ? c : *ct + c;
+              }
+            }
+          }
+        }
+      }
+      __syncthreads();
+    }
+
+    // ---- add the parked sums of every pair in warp order
     for (int idx = threadIdx.x; idx < npairs * 16 * p.M; idx += kPThreads) {
       const int lp = idx / (16 * p.M);
       const int rem = idx - lp * 16 * p.M;
       const int m = rem >> 4, lr = rem & 15;
       if (!pair_full(lp) && lr >= 8) continue;                     // a half pair has eight rows
-      float sum = 0.0f;
+      const int row = pair_rg(lp) * 8 + lr;
+      float sum = group_terms ? -cterm[((size_t)lp * 16 + lr) * toks + m] : 0.0f;
       for (int w = 0; w < kPWarps; ++w) {
         const int sg = lp - wfirst[w];
         if (sg < 0 || sg >= p.maxseg || lp > wlast[w]) continue;
         sum += part[((size_t)(w * p.maxseg + sg) * 16 + lr) * toks + m];
       }
-      const int row = pair_rg(lp) * 8 + lr;
       if (!GROUPED) {
         // the chunk lies inside one group: take its zero-point and bias terms off, then scale
         float sx = 0.0f, sb = 0.0f;
@@ -746,6 +822,7 @@ int plan_prep(int N, int K, int M, int bits, int gcols, PrepPlan* plan) {
     b += (size_t)kPWarps * (*maxseg) * 16 * toks * 4;
     if (nch > 1) b += (size_t)plan->pairs * 16 * toks * 4;
     b += (size_t)(grouped ? spc * gps : kPWarps) * TOKP * 2 * 4 + 128;
+    if (grouped) b += (size_t)plan->pairs * 16 * toks * 4;
     b += (((size_t)M * x_pitch_for(spc)) + 127) / 128 * 128;
     b += (size_t)kPWarps * slots * sps * step_bytes;
     return b;
