@@ -300,9 +300,12 @@ decode_prep_kernel(const PrepParams p) {
       issue_seek();
     }
   };
+  // One slot per warp is requested while the preceding kernel drains; the others follow the
+  // activation requests of the first chunk, which would otherwise queue behind a full ring of
+  // weights on their way into this SM (the CTAs that start last wait longest for them).
   if (lane == 0) {
     issue_seek();
-    for (int s = 0; s < p.slots; ++s) issue_next();
+    issue_next();
   }
 
   // everything below reads X or writes Y: the preceding kernel must have completed
@@ -361,6 +364,8 @@ decode_prep_kernel(const PrepParams p) {
         const int gi = idx / p.M, m = idx - gi * p.M;
         for (int pc = 0; pc < gpieces; ++pc) stage_piece(m, gi * gpieces + pc);
       }
+      if (ch == 0 && lane == 0)
+        for (int s = 1; s < p.slots; ++s) issue_next();
       asm volatile("cp.async.wait_all;" ::: "memory");
       for (int idx = threadIdx.x; idx < ngr * p.M; idx += kPThreads) {
         const int gi = idx / p.M, m = idx - gi * p.M;
@@ -375,6 +380,8 @@ decode_prep_kernel(const PrepParams p) {
       // piece pc of a token goes to thread pc % 512: its run % 4 is the same for all of them
       for (int m = 0; m < p.M; ++m)
         for (int pc = threadIdx.x; pc < pieces; pc += kPThreads) stage_piece(m, pc);
+      if (ch == 0 && lane == 0)
+        for (int s = 1; s < p.slots; ++s) issue_next();
       asm volatile("cp.async.wait_all;" ::: "memory");
       for (int m = 0; m < p.M; ++m) {
         float sx = 0.0f, sb = 0.0f;
@@ -393,6 +400,24 @@ decode_prep_kernel(const PrepParams p) {
       }
     }
     __syncthreads();
+
+    // ---- per-row terms: when every output of the CTA has a thread of its own, that thread fetches
+    // the row's zero-point and scale now, so that the final reduce does not wait for them
+    const bool own_output = !GROUPED && npairs * 16 * p.M <= kPThreads;
+    float z_own = 0.0f, s_own = 0.0f;
+    if (own_output && threadIdx.x < npairs * 16 * p.M) {
+      const int lp = threadIdx.x / (16 * p.M);
+      const int rem = threadIdx.x - lp * 16 * p.M;
+      const int m = rem >> 4, lr = rem & 15;
+      if (pair_full(lp) || lr < 8) {
+        const int row = pair_rg(lp) * 8 + lr;
+        const int gg = p.G == 1 ? 0 : col0 / (p.K / p.G);
+        z_own = (float)__ldg(p.zeros + (size_t)row * p.G + gg);
+        const float* tab = p.scales;
+        if (p.task_ids) tab += (size_t)min(max(__ldg(p.task_ids + m), 0), p.n_tasks - 1) * p.N * p.G;
+        s_own = __ldg(tab + (size_t)row * p.G + gg);
+      }
+    }
 
     // ---- this warp's steps of the chunk
     const int lo = wbound[warp], hi = wbound[warp + 1];
@@ -670,12 +695,16 @@ decode_prep_kernel(const PrepParams p) {
           sx += sums[(w * TOKP + m) * 2];
           sb += sums[(w * TOKP + m) * 2 + 1];
         }
-        const int gg = p.G == 1 ? 0 : col0 / (p.K / p.G);
-        const float z = (float)__ldg(p.zeros + (size_t)row * p.G + gg);
+        float z = z_own, sc = s_own;
+        if (!own_output) {
+          const int gg = p.G == 1 ? 0 : col0 / (p.K / p.G);
+          z = (float)__ldg(p.zeros + (size_t)row * p.G + gg);
+          const float* tab = p.scales;
+          if (p.task_ids) tab += (size_t)min(max(__ldg(p.task_ids + m), 0), p.n_tasks - 1) * p.N * p.G;
+          sc = __ldg(tab + (size_t)row * p.G + gg);
+        }
         sum -= fmaf(z, sx, sb);
-        const float* tab = p.scales;
-        if (p.task_ids) tab += (size_t)min(max(__ldg(p.task_ids + m), 0), p.n_tasks - 1) * p.N * p.G;
-        sum *= __ldg(tab + (size_t)row * p.G + gg);
+        sum *= sc;
       }
       if (p.nchunks > 1) {
         float* ya = yacc + ((size_t)lp * 16 + lr) * toks + m;
