@@ -683,10 +683,15 @@ decode_prep_kernel(const PrepParams p) {
       if (!pair_full(lp) && lr >= 8) continue;                     // a half pair has eight rows
       const int row = pair_rg(lp) * 8 + lr;
       float sum = group_terms ? -cterm[((size_t)lp * 16 + lr) * toks + m] : 0.0f;
+      // branch-free and unrolled, so that the sixteen reads do not wait for one another: a warp
+      // that has nothing parked for this pair reads a slot of its own (any value) and adds zero
+#pragma unroll
       for (int w = 0; w < kPWarps; ++w) {
         const int sg = lp - wfirst[w];
-        if (sg < 0 || sg >= p.maxseg || lp > wlast[w]) continue;
-        sum += part[((size_t)(w * p.maxseg + sg) * 16 + lr) * toks + m];
+        const bool has = sg >= 0 && sg < p.maxseg && lp <= wlast[w];
+        const int sgc = min(max(sg, 0), p.maxseg - 1);
+        const float v = part[((size_t)(w * p.maxseg + sgc) * 16 + lr) * toks + m];
+        sum += has ? v : 0.0f;
       }
       if (!GROUPED) {
         // the chunk lies inside one group: take its zero-point and bias terms off, then scale
