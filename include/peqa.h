@@ -310,7 +310,7 @@ int peqa_scale_adamw(float* scales, const float* dS, float* m, float* v, int64_t
  * writable).  Synchronises the stream before returning.  The tokens travel in
  * chunks over two auxiliary streams of the library, so that the copies in, the
  * kernels and the copies out overlap (pinned host buffers are needed for that);
- * those streams (2) and events (34) are created on the first call on a device
+ * those streams (2) and events (35) are created on the first call on a device
  * and kept until the process ends, so make that first call outside any stream
  * capture.  They are shared by all calls on the device: concurrent calls from
  * several host threads are serialised by the library.  Every argument is checked
@@ -325,6 +325,40 @@ int peqa_train_step_host(const peqa_qweight_t* w, int T,
                          float* d_m, float* d_v,
                          float lr, float beta1, float beta2, float eps, float weight_decay,
                          int64_t step, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * The same host-buffer step for several linears in one call (a layer's
+ * projections, as for peqa_layer_train_step): for each linear, in the order
+ * given, what peqa_train_step_host does, with the copies of the next linear
+ * already on their way while the kernels of the current one run, and the copies
+ * out of a linear overlapping the kernels of the next.  For that every linear
+ * brings device staging buffers of its own: d_X, d_dY, d_Y, d_dX of different
+ * linears must not overlap (PEQA_ERR_BAD_SHAPE otherwise); the workspace may be
+ * shared.  The AdamW step (App. A) is applied to each linear's scales with the
+ * same hyper-parameters and step.  Every argument of every linear is checked
+ * before anything is enqueued; the stream is synchronised before returning; the
+ * library's streams and events are those of peqa_train_step_host.
+ */
+typedef struct {
+  peqa_qweight_t w;       /* w.scales is updated in place */
+  const void* h_X;        /* host bf16 [T, K] in */
+  const void* h_dY;       /* host bf16 [T, N] in */
+  void* h_Y;              /* host bf16 [T, N] out */
+  void* h_dX;             /* host bf16 [T, K] out */
+  float* h_dS;            /* host fp32 [N, G] out */
+  void* d_X;              /* device staging, sizes of the host counterparts */
+  void* d_dY;
+  void* d_Y;
+  void* d_dX;
+  float* d_dS;
+  float* d_m;             /* device fp32 [N, G] in/out, AdamW moments */
+  float* d_v;
+  void* workspace;        /* peqa_workspace_bytes(PEQA_OP_BWD, T, &w) bytes, may be shared */
+  size_t workspace_bytes;
+} peqa_layer_host_linear_t;
+int peqa_layer_train_step_host(const peqa_layer_host_linear_t* linears, int n_linears, int T,
+                               float lr, float beta1, float beta2, float eps, float weight_decay,
+                               int64_t step, void* stream);
 
 /*
  * Scale gradient dS alone, for callers that cannot allocate device memory and

@@ -48,6 +48,14 @@ class _LayerLinear(ctypes.Structure):
                 ("v", ctypes.c_void_p), ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t)]
 
 
+class _LayerHostLinear(ctypes.Structure):
+    _fields_ = [("w", _QWeight), ("h_X", ctypes.c_void_p), ("h_dY", ctypes.c_void_p), ("h_Y", ctypes.c_void_p),
+                ("h_dX", ctypes.c_void_p), ("h_dS", ctypes.c_void_p), ("d_X", ctypes.c_void_p),
+                ("d_dY", ctypes.c_void_p), ("d_Y", ctypes.c_void_p), ("d_dX", ctypes.c_void_p),
+                ("d_dS", ctypes.c_void_p), ("d_m", ctypes.c_void_p), ("d_v", ctypes.c_void_p),
+                ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t)]
+
+
 def lib() -> ctypes.CDLL:
     """Load the shared library (built by paper_2305_14152_b200.build); never falls back."""
     global _lib
@@ -105,6 +113,9 @@ def lib() -> ctypes.CDLL:
         L.peqa_layer_train_step.argtypes = [ctypes.POINTER(_LayerLinear), i32, i32, i32, f32, f32, f32, f32, f32,
                                             i64, vp]
         L.peqa_layer_train_step.restype = ctypes.c_int
+        L.peqa_layer_train_step_host.argtypes = [ctypes.POINTER(_LayerHostLinear), i32, i32, f32, f32, f32, f32,
+                                                 f32, i64, vp]
+        L.peqa_layer_train_step_host.restype = ctypes.c_int
         L.peqa_probe_read.argtypes = [vp, sz, vp, sz, vp]
         L.peqa_probe_read.restype = ctypes.c_int
         for name in ("peqa_quantize_rtn", "peqa_pack", "peqa_unpack", "peqa_qlinear_fwd",
@@ -363,6 +374,54 @@ def layer_train_step(linears, lr: float = 0.0, beta1=0.9, beta2=0.999, eps=1e-8,
         a.workspace, a.workspace_bytes = wp, wb
     _check(lib().peqa_layer_train_step(arr, len(linears), T, 1 if apply_adamw else 0, lr, beta1, beta2, eps,
                                        weight_decay, step, _stream()), "peqa_layer_train_step")
+
+
+@dataclass
+class HostLinear:
+    """Buffers of one linear of a host-buffer layer step: h_* are CPU tensors (pinned for the copies
+    to overlap), d_* device staging of the same shapes, not shared with another linear of the call."""
+    w: QWeight
+    h_X: torch.Tensor        # bf16 [T, K] in
+    h_dY: torch.Tensor       # bf16 [T, N] in
+    h_Y: torch.Tensor        # bf16 [T, N] out
+    h_dX: torch.Tensor       # bf16 [T, K] out
+    h_dS: torch.Tensor       # fp32 [N, G] out
+    d_X: torch.Tensor
+    d_dY: torch.Tensor
+    d_Y: torch.Tensor
+    d_dX: torch.Tensor
+    d_dS: torch.Tensor
+    d_m: torch.Tensor
+    d_v: torch.Tensor
+    workspace: torch.Tensor | None = None
+
+
+def layer_train_step_host(linears, lr: float, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.0, step=1) -> None:
+    """The host-buffer training step of every linear of `linears` in one library call; the copies of
+    a linear overlap the kernels of its neighbours."""
+    arr = (_LayerHostLinear * len(linears))()
+    T = linears[0].h_X.shape[0]
+    for a, L in zip(arr, linears):
+        if L.h_X.shape[0] != T or L.h_dY.shape[0] != T:
+            raise ValueError("all linears of a layer step take the same number of tokens")
+        for t in (L.h_X, L.h_dY, L.h_Y, L.h_dX, L.h_dS):
+            if t.is_cuda or not t.is_contiguous():
+                raise ValueError("h_* must be contiguous CPU tensors")
+        for t, dt, nm in ((L.d_X, torch.bfloat16, "d_X"), (L.d_dY, torch.bfloat16, "d_dY"),
+                          (L.d_Y, torch.bfloat16, "d_Y"), (L.d_dX, torch.bfloat16, "d_dX"),
+                          (L.d_dS, torch.float32, "d_dS"), (L.d_m, torch.float32, "d_m"),
+                          (L.d_v, torch.float32, "d_v")):
+            _dev(t, dt, nm)
+        wp, wb = _ws(L.workspace)
+        a.w = L.w.c_struct()
+        a.h_X, a.h_dY, a.h_Y, a.h_dX, a.h_dS = (L.h_X.data_ptr(), L.h_dY.data_ptr(), L.h_Y.data_ptr(),
+                                                L.h_dX.data_ptr(), L.h_dS.data_ptr())
+        a.d_X, a.d_dY, a.d_Y, a.d_dX, a.d_dS = (L.d_X.data_ptr(), L.d_dY.data_ptr(), L.d_Y.data_ptr(),
+                                                L.d_dX.data_ptr(), L.d_dS.data_ptr())
+        a.d_m, a.d_v = L.d_m.data_ptr(), L.d_v.data_ptr()
+        a.workspace, a.workspace_bytes = wp, wb
+    _check(lib().peqa_layer_train_step_host(arr, len(linears), T, lr, beta1, beta2, eps, weight_decay, step,
+                                            _stream()), "peqa_layer_train_step_host")
 
 
 def qlinear_bwd_dsdz(w: QWeight, X: torch.Tensor, dY: torch.Tensor, dS=None, dZ=None, workspace=None):

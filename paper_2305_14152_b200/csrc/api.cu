@@ -370,7 +370,7 @@ namespace {
 constexpr int kHostChunksMax = 8;
 struct HostPipe {
   cudaStream_t in = nullptr, out = nullptr;
-  cudaEvent_t start = nullptr, out_done = nullptr;
+  cudaEvent_t start = nullptr, out_done = nullptr, ds_done = nullptr;
   cudaEvent_t x_landed[kHostChunksMax] = {};
   cudaEvent_t dy_landed[kHostChunksMax] = {};
   cudaEvent_t fwd_done[kHostChunksMax] = {};
@@ -389,7 +389,8 @@ int host_pipe(int dev, HostPipe** out) {
     bool ok = cudaStreamCreateWithFlags(&hp.in, cudaStreamNonBlocking) == cudaSuccess &&
               cudaStreamCreateWithFlags(&hp.out, cudaStreamNonBlocking) == cudaSuccess &&
               cudaEventCreateWithFlags(&hp.start, cudaEventDisableTiming) == cudaSuccess &&
-              cudaEventCreateWithFlags(&hp.out_done, cudaEventDisableTiming) == cudaSuccess;
+              cudaEventCreateWithFlags(&hp.out_done, cudaEventDisableTiming) == cudaSuccess &&
+              cudaEventCreateWithFlags(&hp.ds_done, cudaEventDisableTiming) == cudaSuccess;
     for (int c = 0; ok && c < kHostChunksMax; ++c)
       ok = cudaEventCreateWithFlags(&hp.x_landed[c], cudaEventDisableTiming) == cudaSuccess &&
            cudaEventCreateWithFlags(&hp.dy_landed[c], cudaEventDisableTiming) == cudaSuccess &&
@@ -401,6 +402,7 @@ int host_pipe(int dev, HostPipe** out) {
       if (hp.out) cudaStreamDestroy(hp.out);
       if (hp.start) cudaEventDestroy(hp.start);
       if (hp.out_done) cudaEventDestroy(hp.out_done);
+      if (hp.ds_done) cudaEventDestroy(hp.ds_done);
       for (int c = 0; c < kHostChunksMax; ++c) {
         if (hp.x_landed[c]) cudaEventDestroy(hp.x_landed[c]);
         if (hp.dy_landed[c]) cudaEventDestroy(hp.dy_landed[c]);
@@ -426,14 +428,140 @@ int drain_and_fail(HostPipe* hp, cudaStream_t st, int rc) {
   return rc;
 }
 
-}  // namespace
-
 // The tokens go through in chunks so that the three engines overlap: chunk c+1 is on its
 // way to the device (auxiliary stream `in`) while chunk c runs forward and dX on the
 // caller's stream and chunk c-1 returns Y and dX (auxiliary stream `out`); PCIe carries both
 // directions at once.  dS sums over all tokens, so it runs once after the last chunk, then
 // AdamW.  Forward and dX treat tokens independently, so chunking does not change a bit of
-// their results.
+// their results.  With several linears the copies in of the next linear run while the
+// kernels of the current one are still busy.
+
+// Host-side checks of one linear of a host-buffer step; nothing is enqueued.
+int check_host_linear(const peqa_layer_host_linear_t& L, int T) {
+  int g = 0, G = 0;
+  PEQA_TRY(check_qweight(&L.w, &g, &G));
+  if (!L.h_X || !L.h_dY || !L.h_Y || !L.h_dX || !L.h_dS || !L.d_X || !L.d_dY || !L.d_Y || !L.d_dX ||
+      !L.d_dS || !L.d_m || !L.d_v)
+    return PEQA_ERR_NULL;
+  PEQA_TRY(check_gemm_shape(&L.w, T));
+  if (!aligned16(L.d_X) || !aligned16(L.d_dY) || !aligned16(L.d_Y) || !aligned16(L.d_dX) || !aligned16(L.d_dS))
+    return PEQA_ERR_ALIGNMENT;
+  const size_t need = ds_workspace_bytes(&L.w, g, T);
+  if (need > 0) {
+    if (!L.workspace || L.workspace_bytes < need) return PEQA_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(L.workspace) & 255u) return PEQA_ERR_ALIGNMENT;
+  }
+  return PEQA_OK;
+}
+
+// Enqueues one linear of a host-buffer step: its tokens travel in chunks of whole 512-token
+// tiles, copies in on hp->in, kernels on st, copies out on hp->out.  The caller has checked
+// every argument, holds the device's pipe mutex and has made hp->in and hp->out wait for
+// whatever must precede the first copy.
+int enqueue_host_linear(HostPipe* hp, cudaStream_t st, const peqa_layer_host_linear_t& L, int T,
+                        float lr, float beta1, float beta2, float eps, float weight_decay,
+                        int64_t step) {
+  const peqa_qweight_t* w = &L.w;
+  const size_t N = w->out_features, K = w->in_features;
+  const size_t G = w->group_size == 0 ? 1 : K / (size_t)w->group_size;
+  int chunks = (T + 511) / 512;
+  if (chunks > kHostChunksMax) chunks = kHostChunksMax;
+  const int per = ((T + chunks - 1) / chunks + 7) & ~7;   // rows per chunk, 16-byte aligned slices
+  chunks = (T + per - 1) / per;
+  const char* hX = static_cast<const char*>(L.h_X);
+  const char* hdY = static_cast<const char*>(L.h_dY);
+  char* hY = static_cast<char*>(L.h_Y);
+  char* hdX = static_cast<char*>(L.h_dX);
+  char* dX_in = static_cast<char*>(L.d_X);
+  char* ddY = static_cast<char*>(L.d_dY);
+  char* dY_out = static_cast<char*>(L.d_Y);
+  char* ddX = static_cast<char*>(L.d_dX);
+  void* stream = static_cast<void*>(st);
+  for (int c = 0; c < chunks; ++c) {
+    const size_t t0 = (size_t)c * per;
+    const size_t tc = (size_t)T - t0 < (size_t)per ? (size_t)T - t0 : (size_t)per;
+    PEQA_CUDA(cudaMemcpyAsync(dX_in + t0 * K * 2, hX + t0 * K * 2, tc * K * 2, cudaMemcpyHostToDevice, hp->in));
+    PEQA_CUDA(cudaEventRecord(hp->x_landed[c], hp->in));
+    PEQA_CUDA(cudaMemcpyAsync(ddY + t0 * N * 2, hdY + t0 * N * 2, tc * N * 2, cudaMemcpyHostToDevice, hp->in));
+    PEQA_CUDA(cudaEventRecord(hp->dy_landed[c], hp->in));
+    // the forward needs only X: it runs while dY is still on its way
+    PEQA_CUDA(cudaStreamWaitEvent(st, hp->x_landed[c], 0));
+    PEQA_TRY(peqa_qlinear_fwd(w, dX_in + t0 * K * 2, (int)tc, dY_out + t0 * N * 2, L.workspace,
+                              L.workspace_bytes, stream));
+    PEQA_CUDA(cudaEventRecord(hp->fwd_done[c], st));
+    PEQA_CUDA(cudaStreamWaitEvent(st, hp->dy_landed[c], 0));
+    PEQA_TRY(peqa_qlinear_bwd(w, nullptr, ddY + t0 * N * 2, (int)tc, ddX + t0 * K * 2, nullptr,
+                              L.workspace, L.workspace_bytes, stream));
+    PEQA_CUDA(cudaEventRecord(hp->dx_done[c], st));
+    // Y goes back while dX is still being computed
+    PEQA_CUDA(cudaStreamWaitEvent(hp->out, hp->fwd_done[c], 0));
+    PEQA_CUDA(cudaMemcpyAsync(hY + t0 * N * 2, dY_out + t0 * N * 2, tc * N * 2, cudaMemcpyDeviceToHost, hp->out));
+    PEQA_CUDA(cudaStreamWaitEvent(hp->out, hp->dx_done[c], 0));
+    PEQA_CUDA(cudaMemcpyAsync(hdX + t0 * K * 2, ddX + t0 * K * 2, tc * K * 2, cudaMemcpyDeviceToHost, hp->out));
+  }
+  PEQA_TRY(peqa_qlinear_bwd_ds_adamw(w, L.d_X, L.d_dY, T, L.d_dS, L.d_m, L.d_v, lr, beta1, beta2, eps,
+                                     weight_decay, step, L.workspace, L.workspace_bytes, stream));
+  // dS follows on the copy-out stream, so that the next linear's kernels do not wait for it
+  PEQA_CUDA(cudaEventRecord(hp->ds_done, st));
+  PEQA_CUDA(cudaStreamWaitEvent(hp->out, hp->ds_done, 0));
+  PEQA_CUDA(cudaMemcpyAsync(L.h_dS, L.d_dS, N * G * 4, cudaMemcpyDeviceToHost, hp->out));
+  return PEQA_OK;
+}
+
+bool ranges_overlap(const void* a, size_t na, const void* b, size_t nb) {
+  const uintptr_t x = reinterpret_cast<uintptr_t>(a), y = reinterpret_cast<uintptr_t>(b);
+  return x < y + nb && y < x + na;
+}
+
+}  // namespace
+
+extern "C" int peqa_layer_train_step_host(const peqa_layer_host_linear_t* linears, int n_linears, int T,
+                                          float lr, float beta1, float beta2, float eps,
+                                          float weight_decay, int64_t step, void* stream) {
+  if (!linears) return PEQA_ERR_NULL;
+  if (n_linears < 1 || n_linears > PEQA_LAYER_MAX_LINEARS || T <= 0 || step < 1) return PEQA_ERR_BAD_SHAPE;
+  // every check of every linear before anything is enqueued
+  for (int i = 0; i < n_linears; ++i) PEQA_TRY(check_host_linear(linears[i], T));
+  // the copies of a linear run ahead of the kernels of the linears before it: the device
+  // staging buffers they write must not be buffers an earlier linear still reads
+  for (int i = 0; i < n_linears; ++i) {
+    const size_t xi = (size_t)T * linears[i].w.in_features * 2, yi = (size_t)T * linears[i].w.out_features * 2;
+    for (int j = 0; j < i; ++j) {
+      const size_t xj = (size_t)T * linears[j].w.in_features * 2, yj = (size_t)T * linears[j].w.out_features * 2;
+      const void* bi[4] = {linears[i].d_X, linears[i].d_dY, linears[i].d_Y, linears[i].d_dX};
+      const size_t ni[4] = {xi, yi, yi, xi};
+      const void* bj[4] = {linears[j].d_X, linears[j].d_dY, linears[j].d_Y, linears[j].d_dX};
+      const size_t nj[4] = {xj, yj, yj, xj};
+      for (int a = 0; a < 4; ++a)
+        for (int b = 0; b < 4; ++b)
+          if (ranges_overlap(bi[a], ni[a], bj[b], nj[b])) return PEQA_ERR_BAD_SHAPE;
+    }
+  }
+  PEQA_TRY(check_arch());
+  cudaStream_t st = as_stream(stream);
+  int dev = 0;
+  PEQA_CUDA(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return PEQA_ERR_TOO_LARGE;
+  // the auxiliary streams and events are shared by all calls on the device: one call at a time
+  std::lock_guard<std::mutex> lock(g_pipe_mutex[dev]);
+  HostPipe* hp = nullptr;
+  PEQA_TRY(host_pipe(dev, &hp));
+  // the auxiliary streams start after whatever the caller's stream already holds
+  cudaError_t e = cudaEventRecord(hp->start, st);
+  if (e == cudaSuccess) e = cudaStreamWaitEvent(hp->in, hp->start, 0);
+  if (e == cudaSuccess) e = cudaStreamWaitEvent(hp->out, hp->start, 0);
+  if (e != cudaSuccess) return drain_and_fail(hp, st, cuda_fail(e));
+  for (int i = 0; i < n_linears; ++i) {
+    const int rc = enqueue_host_linear(hp, st, linears[i], T, lr, beta1, beta2, eps, weight_decay, step);
+    if (rc != PEQA_OK) return drain_and_fail(hp, st, rc);
+  }
+  e = cudaEventRecord(hp->out_done, hp->out);
+  if (e == cudaSuccess) e = cudaStreamWaitEvent(st, hp->out_done, 0);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  if (e != cudaSuccess) return drain_and_fail(hp, st, cuda_fail(e));
+  return PEQA_OK;
+}
+
 extern "C" int peqa_train_step_host(const peqa_qweight_t* w, int T,
                                     const void* h_X, const void* h_dY,
                                     void* h_Y, void* h_dX, float* h_dS,
@@ -442,89 +570,14 @@ extern "C" int peqa_train_step_host(const peqa_qweight_t* w, int T,
                                     float lr, float beta1, float beta2, float eps,
                                     float weight_decay, int64_t step,
                                     void* workspace, size_t workspace_bytes, void* stream) {
-  int g = 0, G = 0;
-  PEQA_TRY(check_qweight(w, &g, &G));
-  if (!h_X || !h_dY || !h_Y || !h_dX || !h_dS || !d_X || !d_dY || !d_Y || !d_dX || !d_dS ||
-      !d_m || !d_v)
-    return PEQA_ERR_NULL;
-  if (T <= 0 || step < 1) return PEQA_ERR_BAD_SHAPE;
-  PEQA_TRY(check_gemm_shape(w, T));
-  // every check the inner calls would make, before anything is enqueued
-  if (!aligned16(d_X) || !aligned16(d_dY) || !aligned16(d_Y) || !aligned16(d_dX) || !aligned16(d_dS))
-    return PEQA_ERR_ALIGNMENT;
-  const size_t need = ds_workspace_bytes(w, g, T);
-  if (need > 0) {
-    if (!workspace || workspace_bytes < need) return PEQA_ERR_WORKSPACE;
-    if (reinterpret_cast<uintptr_t>(workspace) & 255u) return PEQA_ERR_ALIGNMENT;
-  }
-  PEQA_TRY(check_arch());
-  cudaStream_t st = as_stream(stream);
-  const size_t N = w->out_features, K = w->in_features;
-  // chunks of whole 512-token tiles, at most kHostChunksMax of them
-  int chunks = (T + 511) / 512;
-  if (chunks > kHostChunksMax) chunks = kHostChunksMax;
-  const int per = ((T + chunks - 1) / chunks + 7) & ~7;   // rows per chunk, 16-byte aligned slices
-  chunks = (T + per - 1) / per;
-  int dev = 0;
-  PEQA_CUDA(cudaGetDevice(&dev));
-  if (dev < 0 || dev >= 64) return PEQA_ERR_TOO_LARGE;
-  // the auxiliary streams and events are shared by all calls on the device: one call at a time
-  std::lock_guard<std::mutex> lock(g_pipe_mutex[dev]);
-  HostPipe* hp = nullptr;
-  PEQA_TRY(host_pipe(dev, &hp));
-  const char* hX = static_cast<const char*>(h_X);
-  const char* hdY = static_cast<const char*>(h_dY);
-  char* hY = static_cast<char*>(h_Y);
-  char* hdX = static_cast<char*>(h_dX);
-  char* dX_in = static_cast<char*>(d_X);
-  char* ddY = static_cast<char*>(d_dY);
-  char* dY_out = static_cast<char*>(d_Y);
-  char* ddX = static_cast<char*>(d_dX);
-#define PIPE_CUDA(expr)                                                        \
-  do {                                                                         \
-    cudaError_t _e = (expr);                                                   \
-    if (_e != cudaSuccess) return drain_and_fail(hp, st, cuda_fail(_e));       \
-  } while (0)
-#define PIPE_TRY(expr)                                                         \
-  do {                                                                         \
-    int _s = (expr);                                                           \
-    if (_s != PEQA_OK) return drain_and_fail(hp, st, _s);                      \
-  } while (0)
-  // the auxiliary streams start after whatever the caller's stream already holds
-  PIPE_CUDA(cudaEventRecord(hp->start, st));
-  PIPE_CUDA(cudaStreamWaitEvent(hp->in, hp->start, 0));
-  PIPE_CUDA(cudaStreamWaitEvent(hp->out, hp->start, 0));
-  for (int c = 0; c < chunks; ++c) {
-    const size_t t0 = (size_t)c * per;
-    const size_t tc = (size_t)T - t0 < (size_t)per ? (size_t)T - t0 : (size_t)per;
-    PIPE_CUDA(cudaMemcpyAsync(dX_in + t0 * K * 2, hX + t0 * K * 2, tc * K * 2, cudaMemcpyHostToDevice, hp->in));
-    PIPE_CUDA(cudaEventRecord(hp->x_landed[c], hp->in));
-    PIPE_CUDA(cudaMemcpyAsync(ddY + t0 * N * 2, hdY + t0 * N * 2, tc * N * 2, cudaMemcpyHostToDevice, hp->in));
-    PIPE_CUDA(cudaEventRecord(hp->dy_landed[c], hp->in));
-    // the forward needs only X: it runs while dY is still on its way
-    PIPE_CUDA(cudaStreamWaitEvent(st, hp->x_landed[c], 0));
-    PIPE_TRY(peqa_qlinear_fwd(w, dX_in + t0 * K * 2, (int)tc, dY_out + t0 * N * 2, workspace,
-                              workspace_bytes, stream));
-    PIPE_CUDA(cudaEventRecord(hp->fwd_done[c], st));
-    PIPE_CUDA(cudaStreamWaitEvent(st, hp->dy_landed[c], 0));
-    PIPE_TRY(peqa_qlinear_bwd(w, nullptr, ddY + t0 * N * 2, (int)tc, ddX + t0 * K * 2, nullptr,
-                              workspace, workspace_bytes, stream));
-    PIPE_CUDA(cudaEventRecord(hp->dx_done[c], st));
-    // Y goes back while dX is still being computed
-    PIPE_CUDA(cudaStreamWaitEvent(hp->out, hp->fwd_done[c], 0));
-    PIPE_CUDA(cudaMemcpyAsync(hY + t0 * N * 2, dY_out + t0 * N * 2, tc * N * 2, cudaMemcpyDeviceToHost, hp->out));
-    PIPE_CUDA(cudaStreamWaitEvent(hp->out, hp->dx_done[c], 0));
-    PIPE_CUDA(cudaMemcpyAsync(hdX + t0 * K * 2, ddX + t0 * K * 2, tc * K * 2, cudaMemcpyDeviceToHost, hp->out));
-  }
-  PIPE_CUDA(cudaEventRecord(hp->out_done, hp->out));
-  PIPE_TRY(peqa_qlinear_bwd_ds_adamw(w, d_X, d_dY, T, d_dS, d_m, d_v, lr, beta1, beta2, eps,
-                                     weight_decay, step, workspace, workspace_bytes, stream));
-  PIPE_CUDA(cudaMemcpyAsync(h_dS, d_dS, N * (size_t)G * 4, cudaMemcpyDeviceToHost, st));
-  PIPE_CUDA(cudaStreamWaitEvent(st, hp->out_done, 0));
-  PIPE_CUDA(cudaStreamSynchronize(st));
-#undef PIPE_CUDA
-#undef PIPE_TRY
-  return PEQA_OK;
+  if (!w) return PEQA_ERR_NULL;
+  peqa_layer_host_linear_t L = {};
+  L.w = *w;
+  L.h_X = h_X; L.h_dY = h_dY; L.h_Y = h_Y; L.h_dX = h_dX; L.h_dS = h_dS;
+  L.d_X = d_X; L.d_dY = d_dY; L.d_Y = d_Y; L.d_dX = d_dX; L.d_dS = d_dS;
+  L.d_m = d_m; L.d_v = d_v;
+  L.workspace = workspace; L.workspace_bytes = workspace_bytes;
+  return peqa_layer_train_step_host(&L, 1, T, lr, beta1, beta2, eps, weight_decay, step, stream);
 }
 
 extern "C" int peqa_check_status(void* stream) {

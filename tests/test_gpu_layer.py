@@ -103,3 +103,61 @@ def test_arguments_are_checked_before_anything_runs():
     assert torch.equal(layers[0].Y, sentinel)           # the first linear did not run either
     with pytest.raises(binding.PeqaError):
         binding.layer_train_step(layers[:3], LR, step=0)
+
+
+def _host_linears(layers, T, shared_staging=False):
+    out = []
+    stage = None
+    for L in layers:
+        N, K, G = L.w.N, L.w.K, L.w.G
+        pin = lambda t: t.cpu().pin_memory()
+        if shared_staging and stage is not None:
+            d_X = stage                                   # the first linear's buffer again
+        else:
+            d_X = torch.empty((T, K), dtype=torch.bfloat16, device="cuda")
+            stage = stage if stage is not None else d_X
+        out.append(binding.HostLinear(
+            w=L.w, h_X=pin(L.X), h_dY=pin(L.dY),
+            h_Y=torch.empty((T, N), dtype=torch.bfloat16).pin_memory(),
+            h_dX=torch.empty((T, K), dtype=torch.bfloat16).pin_memory(),
+            h_dS=torch.empty((N, G), dtype=torch.float32).pin_memory(),
+            d_X=d_X, d_dY=torch.empty((T, N), dtype=torch.bfloat16, device="cuda"),
+            d_Y=torch.empty((T, N), dtype=torch.bfloat16, device="cuda"),
+            d_dX=torch.empty((T, K), dtype=torch.bfloat16, device="cuda"),
+            d_dS=torch.empty((N, G), dtype=torch.float32, device="cuda"),
+            d_m=L.m, d_v=L.v, workspace=L.workspace))
+    return out
+
+
+@pytest.mark.parametrize("T", [300, 1100])
+def test_layer_step_with_host_buffers(T):
+    """peqa_layer_train_step_host: every linear's Y, dX, dS come back to the host and its scales
+    take the AdamW step, bit-identical to the device-buffer layer call (chunking the tokens
+    changes neither the forward nor dX; dS runs once over all tokens)."""
+    layers, host = _build(T)
+    ref, _ = _build(T)
+    hl = _host_linears(layers, T)
+    binding.layer_train_step_host(hl, LR, step=1)
+    binding.check_status()
+    binding.layer_train_step(ref, LR, step=1)
+    torch.cuda.synchronize()
+    for H, R, (d, zeros, scales, packed, bits, g) in zip(hl, ref, host):
+        assert torch.equal(H.h_Y, R.Y.cpu()) and torch.equal(H.h_dX, R.dX.cpu())
+        assert torch.equal(H.h_dS, R.dS.cpu())
+        assert torch.equal(H.w.scales, R.w.scales) and torch.equal(H.d_m, R.m) and torch.equal(H.d_v, R.v)
+        assert_close(H.h_Y.double().numpy(), oracle.fwd(d["X"], packed, zeros, scales, bits, g), "Y")
+
+
+def test_layer_host_step_rejects_shared_staging_buffers():
+    """The copies of a linear run ahead of the kernels of the one before: staging buffers that
+    overlap between linears are refused before anything is enqueued."""
+    T = 64
+    layers, _ = _build(T)
+    layers = [layers[0], layers[2]]                       # both K = 384: the same d_X size
+    hl = _host_linears(layers, T, shared_staging=True)
+    before = [L.w.scales.clone() for L in layers]
+    with pytest.raises(binding.PeqaError):
+        binding.layer_train_step_host(hl, LR, step=1)
+    torch.cuda.synchronize()
+    for L, b in zip(layers, before):
+        assert torch.equal(L.w.scales, b)

@@ -73,6 +73,27 @@ def test_argument_validation_needs_no_gpu(L):
     assert L.peqa_qlinear_decode_multitask(ctypes.byref(wg), p16, 2, p16, p16, 1, p16, 0) == -3
     assert L.peqa_qlinear_decode_multitask(ctypes.byref(w), p16, 0, p16, p16, 1, p16, 0) == -3
     assert L.peqa_qlinear_decode_multitask(ctypes.byref(w), p16, 2, p16, p16, 17, p16, 0) == -3
+    # the host-buffer layer step: null list, empty list, a linear without host buffers, and two
+    # linears whose device staging buffers overlap
+    f = (1e-3, 0.9, 0.999, 1e-8, 0.0)
+    assert L.peqa_layer_train_step_host(None, 1, 8, *f, 1, 0) == -1
+    one = (binding._LayerHostLinear * 1)()
+    assert L.peqa_layer_train_step_host(one, 0, 8, *f, 1, 0) == -3
+    one[0].w = w
+    assert L.peqa_layer_train_step_host(one, 1, 8, *f, 1, 0) == -1
+    big = ctypes.create_string_buffer(1 << 16)
+    q = (ctypes.addressof(big) + 255) & ~255
+    two = (binding._LayerHostLinear * 2)()
+    for i in range(2):
+        two[i].w = w
+        two[i].workspace, two[i].workspace_bytes = q + 40960, 8192
+        for name in ("h_X", "h_dY", "h_Y", "h_dX", "h_dS", "d_dS", "d_m", "d_v"):
+            setattr(two[i], name, q)
+        # T = 8 tokens: X, dX take 8*256*2 = 4096 bytes, dY, Y 8*128*2 = 2048 bytes
+        two[i].d_X, two[i].d_dX, two[i].d_dY, two[i].d_Y = (q + i * 16384, q + i * 16384 + 4096,
+                                                             q + i * 16384 + 8192, q + i * 16384 + 10240)
+    two[1].d_dY = two[0].d_X + 4080                                  # 16 bytes into linear 0's d_X
+    assert L.peqa_layer_train_step_host(two, 2, 8, *f, 1, 0) == -3
 
 
 def test_workspace_query(L):
