@@ -377,25 +377,34 @@ decode_prep_kernel(const PrepParams p) {
         sums[((size_t)gi * TOKP + m) * 2 + 1] = sb;
       }
     } else {
-      // piece pc of a token goes to thread pc % 512: its run % 4 is the same for all of them
-      for (int m = 0; m < p.M; ++m)
-        for (int pc = threadIdx.x; pc < pieces; pc += kPThreads) stage_piece(m, pc);
+      // A token belongs to 16 / Mp warps (Mp: M rounded up to a power of two); a warp copies
+      // every (16 / Mp)-th block of 32 pieces of its token and sums what it copied itself, so
+      // it needs no other warp's copies and reduces once.  run % 4 of a lane's pieces is fixed.
+      int mp = 1;
+      while (mp < p.M) mp <<= 1;
+      const int wpt = kPWarps / mp;                                // warps per token
+      const int tok = warp / wpt, sub = warp - tok * wpt;
+      if (tok < p.M)
+        for (int pc = sub * 32 + lane; pc < pieces; pc += wpt * 32) stage_piece(tok, pc);
       if (ch == 0 && lane == 0)
         for (int s = 1; s < p.slots; ++s) issue_next();
+      // this warp's row of the table: zero but for its own token
+      for (int i = lane; i < TOKP * 2; i += 32) sums[warp * TOKP * 2 + i] = 0.0f;
       asm volatile("cp.async.wait_all;" ::: "memory");
-      for (int m = 0; m < p.M; ++m) {
+      __syncwarp();
+      if (tok < p.M) {
         float sx = 0.0f, sb = 0.0f;
-        const uint8_t* row = xs + (size_t)m * p.x_pitch;
-        for (int pc = threadIdx.x; pc < pieces; pc += kPThreads)
-          piece_sums(row + pc * 16, (threadIdx.x >> 2) & 3, sx, sb);
+        const uint8_t* row = xs + (size_t)tok * p.x_pitch;
+        for (int pc = sub * 32 + lane; pc < pieces; pc += wpt * 32)
+          piece_sums(row + pc * 16, (lane >> 2) & 3, sx, sb);
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
           sx += __shfl_xor_sync(0xffffffffu, sx, o);
           sb += __shfl_xor_sync(0xffffffffu, sb, o);
         }
         if (lane == 0) {
-          sums[(warp * TOKP + m) * 2] = sx;
-          sums[(warp * TOKP + m) * 2 + 1] = sb;
+          sums[(warp * TOKP + tok) * 2] = sx;
+          sums[(warp * TOKP + tok) * 2 + 1] = sb;
         }
       }
     }
