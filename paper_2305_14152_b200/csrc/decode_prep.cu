@@ -76,6 +76,9 @@ constexpr int kPBarBytes = kPWarps * kPMaxSlots * 8;              // the warps' 
 // + abort flag, wait limit and, per warp, the bounds of its steps and its first and last pair
 constexpr int kPHeadBytes = (kPBarBytes + 32 + 3 * (kPWarps + 1) * 4 + 127) / 128 * 128;
 
+// Pitch (floats) of a row's tokens in the per-output tables of shared memory.
+__host__ __device__ inline int tok_pitch(int toks) { return toks + ((6 - (toks & 3)) & 3); }
+
 struct PrepParams {
   const uint8_t* P;         // prepared weights
   const uint8_t* zeros;     // [N, G]
@@ -192,16 +195,19 @@ decode_prep_kernel(const PrepParams p) {
   int* wfirst = wbound + kPWarps + 1;                                        // [warps] first pair of the range
   int* wlast = wfirst + kPWarps + 1;                                         // [warps] last pair, -1: no steps
   const int toks = (p.M + 1) & ~1;                                           // tokens kept of a tile
-  float* part = reinterpret_cast<float*>(base + kPHeadBytes);                // [warps][maxseg][16][toks]
-  float* yacc = part + (size_t)kPWarps * p.maxseg * 16 * toks;               // [pairs][16][toks]
-  float* sums = yacc + (p.nchunks > 1 ? (size_t)p.pairs_per_cta * 16 * toks : 0);
+  // pitch of a row's tokens in the per-output tables: toks rounded up to 2 mod 4, so that the
+  // sixteen rows a warp reads for one token fall into sixteen different banks
+  const int tp = tok_pitch(toks);
+  float* part = reinterpret_cast<float*>(base + kPHeadBytes);                // [warps][maxseg][16][tp]
+  float* yacc = part + (size_t)kPWarps * p.maxseg * 16 * tp;                 // [pairs][16][tp]
+  float* sums = yacc + (p.nchunks > 1 ? (size_t)p.pairs_per_cta * 16 * tp : 0);
   // sums, GROUPED: [groups of the chunk][TOKP][2] = (sum x, sum bias*x) per group and token;
   // else [16 warps][TOKP][2]: every warp's share of the chunk's sums, added in warp order
   const int sum_rows = GROUPED ? p.spc * GPS : kPWarps;
-  // cterm (GROUPED): [pairs][16][toks], the part of every output that does not depend on the weights
+  // cterm (GROUPED): [pairs][16][tp], the part of every output that does not depend on the weights
   float* cterm = sums + (size_t)sum_rows * TOKP * 2;
   uint8_t* xs = reinterpret_cast<uint8_t*>(
-      (reinterpret_cast<uintptr_t>(cterm + (GROUPED ? (size_t)p.pairs_per_cta * 16 * toks : 0)) + 127) &
+      (reinterpret_cast<uintptr_t>(cterm + (GROUPED ? (size_t)p.pairs_per_cta * 16 * tp : 0)) + 127) &
       ~static_cast<uintptr_t>(127));
   uint8_t* ring = xs + (((size_t)p.M * p.x_pitch + 127) & ~static_cast<size_t>(127));
 
@@ -447,14 +453,14 @@ decode_prep_kernel(const PrepParams p) {
     };
     auto park = [&]() {
       fold();
-      float* mine = part + ((size_t)(warp * p.maxseg + seg) * 16) * toks;
+      float* mine = part + ((size_t)(warp * p.maxseg + seg) * 16) * tp;
 #pragma unroll
       for (int nt = 0; nt < NT; ++nt) {
         const int tk = nt * 8 + c4 * 2;
         const float* v = GROUPED ? yv[nt] : acc[nt];
         if (seg < p.maxseg && tk < toks) {
-          *reinterpret_cast<float2*>(mine + r8 * toks + tk) = make_float2(v[0], v[1]);
-          *reinterpret_cast<float2*>(mine + (r8 + 8) * toks + tk) = make_float2(v[2], v[3]);
+          *reinterpret_cast<float2*>(mine + r8 * tp + tk) = make_float2(v[0], v[1]);
+          *reinterpret_cast<float2*>(mine + (r8 + 8) * tp + tk) = make_float2(v[2], v[3]);
         }
 #pragma unroll
         for (int e = 0; e < 4; ++e) acc[nt][e] = yv[nt][e] = 0.0f;
@@ -674,7 +680,7 @@ decode_prep_kernel(const PrepParams p) {
 #pragma unroll
               for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
               if (lane == 0) {
-                float* ct = cterm + (size_t)r * toks + m;
+                float* ct = cterm + (size_t)r * tp + m;
                 *ct = gb == 0 ? c : *ct + c;
               }
             }
@@ -691,7 +697,7 @@ decode_prep_kernel(const PrepParams p) {
       const int m = rem >> 4, lr = rem & 15;
       if (!pair_full(lp) && lr >= 8) continue;                     // a half pair has eight rows
       const int row = pair_rg(lp) * 8 + lr;
-      float sum = group_terms ? -cterm[((size_t)lp * 16 + lr) * toks + m] : 0.0f;
+      float sum = group_terms ? -cterm[((size_t)lp * 16 + lr) * tp + m] : 0.0f;
       // branch-free and unrolled, so that the sixteen reads do not wait for one another: a warp
       // that has nothing parked for this pair reads a slot of its own (any value) and adds zero
 #pragma unroll
@@ -699,7 +705,7 @@ decode_prep_kernel(const PrepParams p) {
         const int sg = lp - wfirst[w];
         const bool has = sg >= 0 && sg < p.maxseg && lp <= wlast[w];
         const int sgc = min(max(sg, 0), p.maxseg - 1);
-        const float v = part[((size_t)(w * p.maxseg + sgc) * 16 + lr) * toks + m];
+        const float v = part[((size_t)(w * p.maxseg + sgc) * 16 + lr) * tp + m];
         sum += has ? v : 0.0f;
       }
       if (!GROUPED) {
@@ -721,7 +727,7 @@ decode_prep_kernel(const PrepParams p) {
         sum *= sc;
       }
       if (p.nchunks > 1) {
-        float* ya = yacc + ((size_t)lp * 16 + lr) * toks + m;
+        float* ya = yacc + ((size_t)lp * 16 + lr) * tp + m;
         if (ch > 0) sum += *ya;
         if (!last) {
           *ya = sum;
@@ -846,7 +852,7 @@ int plan_prep(int N, int K, int M, int bits, int gcols, PrepPlan* plan) {
   const int sms = sm_count_or(148);
   const int rgs = N / 8;
   const int NT = M <= 8 ? 1 : 2, TOKP = 8 * NT;
-  const int toks = (M + 1) & ~1;
+  const int tp = tok_pitch((M + 1) & ~1);
   const int step_bytes = 2 * bits * 512;
   plan->T = (K + kStepCols - 1) / kStepCols;
   plan->rg_per_cta = (rgs + sms - 1) / sms;
@@ -862,10 +868,10 @@ int plan_prep(int N, int K, int M, int bits, int gcols, PrepPlan* plan) {
     *maxseg = (steps + spc - 1) / spc + 2;
     if (*maxseg > plan->pairs) *maxseg = plan->pairs;
     size_t b = 128 + kPHeadBytes;
-    b += (size_t)kPWarps * (*maxseg) * 16 * toks * 4;
-    if (nch > 1) b += (size_t)plan->pairs * 16 * toks * 4;
+    b += (size_t)kPWarps * (*maxseg) * 16 * tp * 4;
+    if (nch > 1) b += (size_t)plan->pairs * 16 * tp * 4;
     b += (size_t)(grouped ? spc * gps : kPWarps) * TOKP * 2 * 4 + 128;
-    if (grouped) b += (size_t)plan->pairs * 16 * toks * 4;
+    if (grouped) b += (size_t)plan->pairs * 16 * tp * 4;
     b += (((size_t)M * x_pitch_for(spc)) + 127) / 128 * 128;
     b += (size_t)kPWarps * slots * sps * step_bytes;
     return b;
