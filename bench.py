@@ -468,11 +468,8 @@ def bench_layer_call(args, binding, torch, layers, peaks, warmup):
             "peak_kind": which, "frac_of_peak": tf / peak, "frac_of_nominal_2250": tf / NOMINAL_BF16_TFLOPS}
 
 
-def bench_e2e(args, binding, torch, layers, Y, dX, dist, dev, world, flop_step):
-    """Same metric through peqa_layer_train_step_host, one call per step: every step copies each
-    linear's X and dY from pinned host memory and returns Y, dX and dS to pinned host memory;
-    every linear has device staging buffers of its own, so its copies overlap its neighbours'
-    kernels."""
+def host_linears(torch, binding, dev, layers):
+    """Pinned host buffers and per-linear device staging buffers for peqa_layer_train_step_host."""
     hl = []
     for L in layers:
         hX = torch.empty((L.T, L.K), dtype=torch.bfloat16).pin_memory()
@@ -489,7 +486,11 @@ def bench_e2e(args, binding, torch, layers, Y, dX, dist, dev, world, flop_step):
             d_Y=torch.empty((L.T, L.N), dtype=torch.bfloat16, device=dev),
             d_dX=torch.empty((L.T, L.K), dtype=torch.bfloat16, device=dev),
             d_dS=L.dS, d_m=L.m, d_v=L.v, workspace=L.ws))
-    steps = max(2, min(args.steps, 5))
+    return hl
+
+
+def time_host_step(torch, binding, hl, steps, dist=None, dev=None):
+    """ms per peqa_layer_train_step_host call (max over ranks), bytes copied each way, clocks."""
     binding.layer_train_step_host(hl, LR, step=1)
     torch.cuda.synchronize()
     if dist is not None:
@@ -498,12 +499,23 @@ def bench_e2e(args, binding, torch, layers, Y, dX, dist, dev, world, flop_step):
         for k in range(steps):
             binding.layer_train_step_host(hl, LR, step=k + 2)
     ms = aggregate_max(tm.ms / steps, dist, dev)
-    return {"value": world * flop_step / (ms * 1e-3) / 1e12, "unit": "TFLOP/s",
-            "h2d_bytes_per_step": int(sum(H.h_X.numel() * 2 + H.h_dY.numel() * 2 for H in hl)),
-            "d2h_bytes_per_step": int(sum(H.h_Y.numel() * 2 + H.h_dX.numel() * 2 + H.h_dS.numel() * 4 for H in hl)),
-            "ms_per_step": ms, "steps": steps, "clocks": tm.clocks,
-            "what": "peqa_layer_train_step_host, one call per step: per linear H2D X,dY; fwd, dX, dS+AdamW; "
-                    "D2H Y,dX,dS; the copies of a linear overlap the kernels of its neighbours"}
+    return ms, {"h2d_bytes_per_step": int(sum(H.h_X.numel() * 2 + H.h_dY.numel() * 2 for H in hl)),
+                "d2h_bytes_per_step": int(sum(H.h_Y.numel() * 2 + H.h_dX.numel() * 2 + H.h_dS.numel() * 4 for H in hl)),
+                "ms_per_step": ms, "steps": steps, "clocks": tm.clocks}
+
+
+def bench_e2e(args, binding, torch, layers, Y, dX, dist, dev, world, flop_step):
+    """Same metric through peqa_layer_train_step_host, one call per step: every step copies each
+    linear's X and dY from pinned host memory and returns Y, dX and dS to pinned host memory;
+    every linear has device staging buffers of its own, so its copies overlap its neighbours'
+    kernels."""
+    hl = host_linears(torch, binding, dev, layers)
+    ms, rec = time_host_step(torch, binding, hl, max(2, min(args.steps, 5)), dist, dev)
+    out = {"value": world * flop_step / (ms * 1e-3) / 1e12, "unit": "TFLOP/s"}
+    out.update(rec)
+    out["what"] = ("peqa_layer_train_step_host, one call per step: per linear H2D X,dY; fwd, dX, dS+AdamW; "
+                   "D2H Y,dX,dS; the copies of a linear overlap the kernels of its neighbours")
+    return out
 
 
 def bench_small_workload(torch, binding, dev, peaks, name, steps, n_sets):
@@ -553,7 +565,12 @@ def bench_small_workload(torch, binding, dev, peaks, name, steps, n_sets):
         tf = 3.0 * L.flop / (sum(stage_ms[li][1:4]) * 1e-3) / 1e12
         r.update({"fwd_dx_ds_tflops": tf, "frac_of_peak": tf / peak, "frac_of_nominal_2250": tf / NOMINAL_BF16_TFLOPS})
         rec["per_linear"][L.spec.name] = r
-    del sets
+    # the same workload end to end from pinned host buffers (copies both ways inside the time)
+    hl = host_linears(torch, binding, dev, layers)
+    ms, e2e = time_host_step(torch, binding, hl, max(5, steps // 10))
+    e2e.update({"value": flop_step / (ms * 1e-3) / 1e12, "unit": "TFLOP/s"})
+    rec["e2e"] = e2e
+    del sets, hl
     torch.cuda.empty_cache()
     return rec
 
@@ -725,6 +742,12 @@ def render_md(path):
         o.append("")
         o.append(f"End to end ({e['what']}): {e['value']:.0f} TFLOP/s, {e['ms_per_step']:.2f} ms per step, "
                  f"{e['h2d_bytes_per_step'] / 1e6:.0f} MB in and {e['d2h_bytes_per_step'] / 1e6:.0f} MB out per step.")
+    for key in ("c2", "c3"):
+        e = (doc.get(key) or {}).get("e2e")
+        if e:
+            o.append(f"End to end, {key}: {e['value']:.0f} TFLOP/s, {e['ms_per_step']:.3f} ms per step, "
+                     f"{e['h2d_bytes_per_step'] / 1e6:.1f} MB in and {e['d2h_bytes_per_step'] / 1e6:.1f} MB out per step "
+                     f"({(e['h2d_bytes_per_step'] + e['d2h_bytes_per_step']) / e['ms_per_step'] / 1e6:.0f} GB/s over the link, both directions).")
     if doc.get("decode"):
         o.append("")
         o.append("| decode shape | bare read us (GB/s) | M | us | GB/s | of measured copy | of 8 TB/s | bare read / kernel |")

@@ -454,8 +454,8 @@ int check_host_linear(const peqa_layer_host_linear_t& L, int T) {
   return PEQA_OK;
 }
 
-// Enqueues one linear of a host-buffer step: its tokens travel in chunks of whole 512-token
-// tiles, copies in on hp->in, kernels on st, copies out on hp->out.  The caller has checked
+// Enqueues one linear of a host-buffer step: its tokens travel in chunks, copies in on hp->in,
+// kernels on st, copies out on hp->out.  The caller has checked
 // every argument, holds the device's pipe mutex and has made hp->in and hp->out wait for
 // whatever must precede the first copy.
 int enqueue_host_linear(HostPipe* hp, cudaStream_t st, const peqa_layer_host_linear_t& L, int T,
@@ -464,7 +464,9 @@ int enqueue_host_linear(HostPipe* hp, cudaStream_t st, const peqa_layer_host_lin
   const peqa_qweight_t* w = &L.w;
   const size_t N = w->out_features, K = w->in_features;
   const size_t G = w->group_size == 0 ? 1 : K / (size_t)w->group_size;
-  int chunks = (T + 511) / 512;
+  // chunks of 256 tokens or more, at most kHostChunksMax: short chunks shorten the time before
+  // the first kernel can start and after the last one has ended, which is all copy time
+  int chunks = (T + 255) / 256;
   if (chunks > kHostChunksMax) chunks = kHostChunksMax;
   const int per = ((T + chunks - 1) / chunks + 7) & ~7;   // rows per chunk, 16-byte aligned slices
   chunks = (T + per - 1) / per;
