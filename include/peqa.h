@@ -429,7 +429,8 @@ int peqa_decode_unprepare(const peqa_qweight_t* w, const uint32_t* prepared, uin
  * scale_table (fp32 [n_tasks, N, G]): token m is served with the scales of its
  * own task (Sec. 3.3).  w->qweight is not read.
  *   X  in  bf16 [M, K]    Y  out  bf16 [M, N]    task_ids  in  int32 [M] (device)
- * No workspace.  The kernel is launched so that it may begin while earlier work
+ * No workspace.  More than eight tokens are served by two launches of at most
+ * eight tokens each.  The kernel is launched so that it may begin while earlier work
  * on `stream` is still draining: it starts to read `prepared` before that work
  * is known to be complete (X, the zero-points and the scales are read and Y is
  * written only after it has completed).  `prepared` must therefore be final when
