@@ -141,8 +141,8 @@ __device__ __forceinline__ uint32_t quantize_run8(const float (&x)[8], float s, 
 // row are issued before pass 1 of the current one, so that the memory system
 // stays busy while the row is being reduced and encoded.  RUNS == 0 reads the
 // row a second time in pass 3 instead (any K).
-template <int BITS, int RUNS, bool PREFETCH>
-__global__ void __launch_bounds__(kQuantThreads)
+template <int BITS, int RUNS, bool PREFETCH, int THREADS = kQuantThreads>
+__global__ void __launch_bounds__(THREADS)
 quantize_rtn_kernel(const float* __restrict__ W, int N, int K, int g, int cpg_shift,
                     uint32_t* __restrict__ qweight, uint8_t* __restrict__ zeros,
                     float* __restrict__ scales) {
@@ -165,7 +165,7 @@ quantize_rtn_kernel(const float* __restrict__ W, int N, int K, int g, int cpg_sh
     const float4* w4 = row_ptr(row);
 #pragma unroll
     for (int r = 0; r < NR; ++r) {
-      const int v = r * kQuantThreads + threadIdx.x;
+      const int v = r * THREADS + threadIdx.x;
       a[r] = make_float4(0.f, 0.f, 0.f, 0.f);
       b[r] = a[r];
       if (row < N && v < nv8) { a[r] = __ldg(w4 + 2 * v); b[r] = __ldg(w4 + 2 * v + 1); }
@@ -191,11 +191,11 @@ quantize_rtn_kernel(const float* __restrict__ W, int N, int K, int g, int cpg_sh
     if constexpr (RUNS > 0) {
 #pragma unroll
       for (int r = 0; r < RUNS; ++r) {
-        const int v = r * kQuantThreads + threadIdx.x;
+        const int v = r * THREADS + threadIdx.x;
         minmax_run(v, v < nv8, ra[r], rb[r]);
       }
     } else {
-      for (int vb = 0; vb < nv8; vb += kQuantThreads) {
+      for (int vb = 0; vb < nv8; vb += THREADS) {
         const int v = vb + threadIdx.x;
         const bool in = v < nv8;
         float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
@@ -218,7 +218,7 @@ quantize_rtn_kernel(const float* __restrict__ W, int N, int K, int g, int cpg_sh
     };
     if (cpg <= 32) {
       // narrow groups: one thread per group
-      for (int gi = threadIdx.x; gi < G; gi += kQuantThreads) {
+      for (int gi = threadIdx.x; gi < G; gi += THREADS) {
         float mn = INFINITY, mx = -INFINITY;
         for (int c = 0; c < cpg; ++c) {
           mn = fminf(mn, cmin[gi * cpg + c]);
@@ -228,7 +228,7 @@ quantize_rtn_kernel(const float* __restrict__ W, int N, int K, int g, int cpg_sh
       }
     } else {
       // wide groups (per-channel above all): one warp per group
-      for (int gi = warp; gi < G; gi += kQuantWarps) {
+      for (int gi = warp; gi < G; gi += (THREADS / 32)) {
         float mn = INFINITY, mx = -INFINITY;
         for (int c = lane; c < cpg; c += 32) {
           mn = fminf(mn, cmin[gi * cpg + c]);
@@ -263,11 +263,11 @@ quantize_rtn_kernel(const float* __restrict__ W, int N, int K, int g, int cpg_sh
     if constexpr (RUNS > 0) {
 #pragma unroll
       for (int r = 0; r < RUNS; ++r) {
-        const int v = r * kQuantThreads + threadIdx.x;
+        const int v = r * THREADS + threadIdx.x;
         emit_run(v, v < nv8, ra[r], rb[r]);
       }
     } else {
-      for (int vb = 0; vb < nv8; vb += kQuantThreads) {
+      for (int vb = 0; vb < nv8; vb += THREADS) {
         const int v = vb + threadIdx.x;
         const bool in = v < nv8;
         float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
@@ -365,40 +365,41 @@ extern "C" int peqa_quantize_rtn(const float* W, int N, int K, int bits, int gro
   int cpg_shift = -1;
   for (int b = 0; b < 26; ++b)
     if ((32 << b) == g) cpg_shift = b;
-  // rows up to 2048 * RUNS columns stay in registers between the passes; short rows also
-  // prefetch the CTA's next row
+  // rows up to 8 * RUNS * threads columns stay in registers between the passes; rows of up to
+  // 8192 columns (256 threads) and of 12289 to 24576 columns (512 threads) also prefetch the
+  // CTA's next row
   const int runs = K <= 4096 ? 2 : K <= 8192 ? 4 : K <= 12288 ? 6 : K <= 24576 ? 12 : 0;
   const size_t smem = (size_t)(K / g) * (sizeof(GroupConst) + 8) + (size_t)(K >> 5) * 8;
   int sms = 0, dev = 0;
   PEQA_CUDA(cudaGetDevice(&dev));
   PEQA_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-#define PEQA_QUANT_LAUNCH(B, R, P)                                                                     \
+#define PEQA_QUANT_LAUNCH(B, R, P, TH)                                                                 \
   do {                                                                                                 \
-    auto kern = quantize_rtn_kernel<B, R, P>;                                                          \
+    auto kern = quantize_rtn_kernel<B, R, P, TH>;                                                      \
     if (smem > 48 * 1024)                                                                              \
       PEQA_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));   \
     int per_sm = 0;                                                                                    \
-    PEQA_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kQuantThreads, smem));      \
+    PEQA_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, TH, smem));                 \
     if (per_sm < 1) per_sm = 1;                                                                        \
     const long long resident = (long long)sms * per_sm;                                                \
     const int grid = (int)(N < resident ? N : resident);                                               \
-    kern<<<grid, kQuantThreads, smem, st>>>(W, N, K, g, cpg_shift, qweight, zeros, scales);            \
+    kern<<<grid, TH, smem, st>>>(W, N, K, g, cpg_shift, qweight, zeros, scales);                       \
   } while (0)
   if (bits == 4) {
     switch (runs) {
-      case 2: PEQA_QUANT_LAUNCH(4, 2, true); break;
-      case 4: PEQA_QUANT_LAUNCH(4, 4, true); break;
-      case 6: PEQA_QUANT_LAUNCH(4, 6, false); break;
-      case 12: PEQA_QUANT_LAUNCH(4, 12, false); break;
-      default: PEQA_QUANT_LAUNCH(4, 0, false); break;
+      case 2: PEQA_QUANT_LAUNCH(4, 2, true, 256); break;
+      case 4: PEQA_QUANT_LAUNCH(4, 4, true, 256); break;
+      case 6: PEQA_QUANT_LAUNCH(4, 6, false, 256); break;
+      case 12: PEQA_QUANT_LAUNCH(4, 6, true, 512); break;   // 512 threads: the next row is prefetched
+      default: PEQA_QUANT_LAUNCH(4, 0, false, 256); break;
     }
   } else {
     switch (runs) {
-      case 2: PEQA_QUANT_LAUNCH(3, 2, true); break;
-      case 4: PEQA_QUANT_LAUNCH(3, 4, true); break;
-      case 6: PEQA_QUANT_LAUNCH(3, 6, false); break;
-      case 12: PEQA_QUANT_LAUNCH(3, 12, false); break;
-      default: PEQA_QUANT_LAUNCH(3, 0, false); break;
+      case 2: PEQA_QUANT_LAUNCH(3, 2, true, 256); break;
+      case 4: PEQA_QUANT_LAUNCH(3, 4, true, 256); break;
+      case 6: PEQA_QUANT_LAUNCH(3, 6, false, 256); break;
+      case 12: PEQA_QUANT_LAUNCH(3, 6, true, 512); break;   // 512 threads: the next row is prefetched
+      default: PEQA_QUANT_LAUNCH(3, 0, false, 256); break;
     }
   }
 #undef PEQA_QUANT_LAUNCH
