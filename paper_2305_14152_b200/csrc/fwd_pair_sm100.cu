@@ -121,6 +121,10 @@ qfwd_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
   __syncthreads();
   cluster_sync_all();
   tc_fence_after();
+  // Set-up is done.  The next kernel of the stream may begin its own (programmatic launch);
+  // everything below touches memory that the preceding kernel may still be writing.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const uint32_t tmem_base = bars->tmem_base;
   const int total_tiles = p.items.total_items;      // work items: whole tiles, then halves
   const int pair = blockIdx.x >> 1;
@@ -439,13 +443,16 @@ int launch_pair_t(const CUtensorMap& tx, const CUtensorMap& tq, const CUtensorMa
   cfg.blockDim = dim3(kPairThreads, 1, 1);
   cfg.dynamicSmemBytes = P_SMEM_BYTES;
   cfg.stream = st;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = 2;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  // barrier set-up and the tensor-memory allocation may overlap the tail of the kernel before
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = 2;
   PEQA_CUDA(cudaLaunchKernelEx(&cfg, kern, tx, tq, ty, p));
   return PEQA_OK;
 }

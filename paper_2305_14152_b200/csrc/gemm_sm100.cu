@@ -551,6 +551,10 @@ ds_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_constant__ C
   __syncthreads();
   cluster_sync_all();          // barriers of both CTAs initialised before any remote arrive
   tc_fence_after();
+  // Set-up is done.  The next kernel of the stream may begin its own (programmatic launch);
+  // everything below touches memory that the preceding kernel may still be writing.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const uint32_t tmem_base = bars->tmem_base;
   const int total_tiles = p.i_tiles * p.j_tiles;   // pair tiles (256 x 256)
   const int pair = blockIdx.x >> 1;
@@ -952,13 +956,16 @@ int launch_ds(const peqa_qweight_t* w, const float* zeros_f, int g, const void* 
   cfg.blockDim = dim3(kDsThreads, 1, 1);
   cfg.dynamicSmemBytes = DS_SMEM_BYTES;
   cfg.stream = st;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = 2;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  // barrier set-up and the tensor-memory allocation may overlap the tail of the kernel before
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = 2;
 #define PEQA_DS_LAUNCH(B, Z, A)                                                                       \
   do {                                                                                               \
     auto kern = ds_kernel<B, Z, A>;                                                                  \
